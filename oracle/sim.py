@@ -1,0 +1,104 @@
+"""Sequential fp64 simulator backed by a2cid2_oracle.c -- TEST INFRASTRUCTURE.
+
+Follows Eq. (dynamic) of Sec. 3.2 event by event in time order; see the C file's header for
+the passage behind each step."""
+from __future__ import annotations
+
+import ctypes as C
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        dp, ip = C.POINTER(C.c_double), C.POINTER(C.c_int32)
+        L.a2o_mix_coeff.restype = C.c_double
+        L.a2o_mix_coeff.argtypes = [C.c_double, C.c_double]
+        L.a2o_run.restype = C.c_int
+        L.a2o_run.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_double,
+                              dp, dp, dp, dp, C.c_int32, C.c_int64,
+                              C.c_int64, dp, ip, ip, ip, C.c_int32]
+        L.a2o_consensus.restype = C.c_double
+        L.a2o_consensus.argtypes = [C.c_int32, C.c_int64, C.c_int64, dp]
+        L.a2o_consensus_at.restype = C.c_double
+        L.a2o_consensus_at.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_double, dp, dp, dp, C.c_double]
+        _lib = L
+    return _lib
+
+
+def _dp(a, off=0):
+    return C.cast(a.ctypes.data + 8 * off, C.POINTER(C.c_double))
+
+
+def _ip(a):
+    return a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+class OracleError(RuntimeError):
+    pass
+
+
+class OracleSim:
+    """State: X, Xt of shape [n, d] (fp64), t_last[n]. Initialisation as in Algorithm 1:
+    x~ <- x, t <- 0, unless given."""
+
+    def __init__(self, x0, eta, alpha, alpha_tilde, gamma, grads=None, xt0=None, t0=None, variant=0):
+        self.X = np.array(x0, dtype=np.float64, order="C")
+        self.n, self.d = self.X.shape
+        self.Xt = self.X.copy() if xt0 is None else np.array(xt0, dtype=np.float64, order="C")
+        self.t = np.zeros(self.n) if t0 is None else np.array(t0, dtype=np.float64)
+        self.G = None if grads is None else np.array(grads, dtype=np.float64, order="C")
+        self.eta, self.alpha, self.alpha_tilde, self.gamma = float(eta), float(alpha), float(alpha_tilde), float(gamma)
+        self.variant = int(variant)
+
+    def _run_cols(self, c0, c1, tl, times, wi, wj, slot):
+        G = self.G if self.G is not None else np.zeros((1, self.d))
+        rc = lib().a2o_run(self.n, c1 - c0, self.d, self.eta, self.alpha, self.alpha_tilde, self.gamma,
+                           _dp(self.X, c0), _dp(self.Xt, c0), _dp(tl), _dp(G, c0), G.shape[0], self.d,
+                           len(times), _dp(times), _ip(wi), _ip(wj), _ip(slot), self.variant)
+        return rc
+
+    def apply(self, times, wi, wj, slot, threads=1):
+        """Apply events in the order given. threads > 1 splits the *columns* over threads
+        (columns never interact); every slice still sees the events in the same order."""
+        times = np.ascontiguousarray(times, dtype=np.float64)
+        wi = np.ascontiguousarray(wi, dtype=np.int32)
+        wj = np.ascontiguousarray(wj, dtype=np.int32)
+        slot = np.ascontiguousarray(slot, dtype=np.int32)
+        if len(times) == 0:
+            return
+        if threads <= 1 or self.d < threads:
+            rc = self._run_cols(0, self.d, self.t, times, wi, wj, slot)
+            if rc != 0:
+                raise OracleError(f"a2o_run -> {rc}")
+            return
+        bounds = np.linspace(0, self.d, threads + 1).astype(np.int64)
+        tls = [self.t.copy() for _ in range(threads)]
+        with ThreadPoolExecutor(threads) as ex:
+            rcs = list(ex.map(lambda k: self._run_cols(int(bounds[k]), int(bounds[k + 1]), tls[k],
+                                                       times, wi, wj, slot), range(threads)))
+        if any(rcs):
+            raise OracleError(f"a2o_run -> {rcs}")
+        self.t[:] = tls[0]
+
+    def apply_stream(self, ev, threads=1):
+        self.apply(ev.times, ev.wi, ev.wj, ev.slot, threads=threads)
+
+    def consensus(self, t_eval=None):
+        if t_eval is None:
+            return float(lib().a2o_consensus(self.n, self.d, self.d, _dp(self.X)))
+        return float(lib().a2o_consensus_at(self.n, self.d, self.d, self.eta, _dp(self.X), _dp(self.Xt),
+                                            _dp(self.t), float(t_eval)))
+
+    def flushed(self, t_eval):
+        """(x, x~) of every worker mixed forward to the common time t_eval (copies)."""
+        c = np.array([lib().a2o_mix_coeff(self.eta, float(t_eval) - ti) for ti in self.t])[:, None]
+        dlt = self.X - self.Xt
+        return self.X - c * dlt, self.Xt + c * dlt

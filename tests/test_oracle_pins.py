@@ -1,0 +1,439 @@
+"""Pins for the CPU checker: what the paper and the mathematics fix, independent of the
+checker's own formulas. Each test names the passage it rests on."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import spectral
+from oracle.sim import OracleSim, OracleError, lib
+from oracle.sim_np import NumpySim
+from paper_2306_08289_b200 import workload as W
+
+SIMS = [OracleSim, NumpySim]
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_state(n, d, seed):
+    r = np.random.default_rng(seed)
+    return r.standard_normal((n, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+
+
+def _one(times, wi, wj, slot):
+    return (np.array(times, dtype=np.float64), np.array(wi, dtype=np.int32),
+            np.array(wj, dtype=np.int32), np.array(slot, dtype=np.int32))
+
+
+# ---- mixing flow: drift term of Eq. (dynamic); matrix exponential of Algorithm 1 --------
+@pytest.mark.parametrize("Sim", SIMS)
+def test_mixing_keeps_half_sum_and_shrinks_difference(Sim):
+    x0, xt0, _ = _rand_state(3, 7, 0)
+    eta, dt = 0.37, 1.9
+    s = Sim(x0, eta, 0.5, 0.8, 0.1, grads=np.zeros((3, 7)), xt0=xt0)
+    s.apply(*_one([dt], [1], [-1], [1]))  # zero gradient: only the flow acts on worker 1
+    np.testing.assert_allclose(s.X[1] + s.Xt[1], x0[1] + xt0[1], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(s.X[1] - s.Xt[1], (x0[1] - xt0[1]) * math.exp(-2 * eta * dt), rtol=1e-14)
+    # untouched workers are untouched, bit for bit
+    assert np.array_equal(s.X[[0, 2]], x0[[0, 2]]) and np.array_equal(s.Xt[[0, 2]], xt0[[0, 2]])
+    assert s.t[1] == dt and s.t[0] == 0.0
+
+
+@pytest.mark.parametrize("Sim", SIMS)
+def test_mixing_semigroup(Sim):
+    x0, xt0, _ = _rand_state(2, 5, 1)
+    a = Sim(x0, 0.9, 0.5, 0.5, 0.0, grads=np.zeros((2, 5)), xt0=xt0)
+    b = Sim(x0, 0.9, 0.5, 0.5, 0.0, grads=np.zeros((2, 5)), xt0=xt0)
+    a.apply(*_one([0.4, 1.7], [0, 0], [-1, -1], [0, 0]))
+    b.apply(*_one([1.7], [0], [-1], [0]))
+    np.testing.assert_allclose(a.X, b.X, rtol=1e-14, atol=1e-15)
+    np.testing.assert_allclose(a.Xt, b.Xt, rtol=1e-14, atol=1e-15)
+
+
+def test_mixing_matches_series_of_the_generator():
+    """exp(dt*A) summed from its power series, A = [[-eta, eta],[eta,-eta]] (Algorithm 1)."""
+    eta, dt = 0.6, 0.8
+    A = dt * np.array([[-eta, eta], [eta, -eta]])
+    E, term = np.eye(2), np.eye(2)
+    for k in range(1, 40):
+        term = term @ A / k
+        E = E + term
+    x0, xt0, _ = _rand_state(2, 4, 2)
+    s = OracleSim(x0, eta, 0.5, 0.5, 0.0, grads=np.zeros((1, 4)), xt0=xt0)
+    s.apply(*_one([dt], [0], [-1], [0]))
+    want = E @ np.stack([x0[0], xt0[0]])
+    np.testing.assert_allclose(np.stack([s.X[0], s.Xt[0]]), want, rtol=1e-13, atol=1e-15)
+    assert abs(lib().a2o_mix_coeff(eta, dt) - E[0, 1]) < 1e-15
+
+
+# ---- pairwise jump: communication term of Eq. (dynamic); App. C "in the orthogonal of 1" ---
+@pytest.mark.parametrize("Sim", SIMS)
+def test_comm_keeps_population_sums(Sim):
+    x0, xt0, _ = _rand_state(5, 6, 3)
+    s = Sim(x0, 0.3, 0.5, 2.5, 0.0, xt0=xt0, t0=np.full(5, 1.0))
+    s.apply(*_one([1.0], [1], [3], [-1]))  # dt = 0: the jump alone
+    np.testing.assert_allclose(s.X.sum(0), x0.sum(0), atol=1e-14)
+    np.testing.assert_allclose(s.Xt.sum(0), xt0.sum(0), atol=1e-14)
+    m = x0[1] - x0[3]
+    np.testing.assert_allclose(s.X[1], x0[1] - 0.5 * m, atol=1e-15)
+    np.testing.assert_allclose(s.X[3], x0[3] + 0.5 * m, atol=1e-15)
+    np.testing.assert_allclose(s.Xt[1], xt0[1] - 2.5 * m, atol=1e-14)
+    np.testing.assert_allclose(s.Xt[3], xt0[3] + 2.5 * m, atol=1e-14)
+
+
+@pytest.mark.parametrize("alpha", [0.5, 0.3, 0.9])
+def test_comm_consensus_drop_identity(alpha):
+    """App. C, study of the ||pi x||_F^2 terms: one averaging changes it by
+    2 alpha (alpha - 1) |x_i - x_j|^2."""
+    x0, xt0, _ = _rand_state(6, 9, 4)
+    s = OracleSim(x0, 0.4, alpha, 1.3, 0.0, xt0=xt0, t0=np.full(6, 2.0))
+    c0 = s.consensus()
+    m2 = float(((x0[2] - x0[5]) ** 2).sum())
+    s.apply(*_one([2.0], [2], [5], [-1]))
+    assert abs((s.consensus() - c0) - 2 * alpha * (alpha - 1) * m2) < 1e-12 * max(1.0, c0)
+
+
+@pytest.mark.parametrize("Sim", SIMS)
+def test_two_workers_reach_exact_consensus_in_one_event(Sim):
+    x0 = np.array([[1.0, -2.0, 3.5], [0.25, 4.0, -1.0]])
+    s = Sim(x0, 0.0, 0.5, 0.5, 0.0)
+    s.apply(*_one([0.7], [0], [1], [-1]))
+    assert np.array_equal(s.X[0], s.X[1]) and np.array_equal(s.X[0], x0.mean(0))
+    assert np.array_equal(s.Xt, s.X)
+    assert s.consensus() == 0.0
+
+
+def test_baseline_gossip_on_complete_graph_reaches_consensus():
+    """Sec. 3.3: eta = 0, alpha = alpha~ = 1/2, no gradients: plain pairwise averaging. The
+    consensus distance never increases and goes to zero on a connected graph."""
+    n, d = 8, 11
+    x0 = np.random.default_rng(5).standard_normal((n, d))
+    edges = W.complete_edges(n)
+    ev = W.poisson_events(n, edges, np.ones(len(edges)), 1500, seed=7, grad_rate=0.0)
+    assert np.all(ev.wj >= 0)
+    s = OracleSim(x0, 0.0, 0.5, 0.5, 0.0)
+    prev = s.consensus()
+    start = prev
+    for k in range(0, len(ev), 50):
+        s.apply_stream(ev.slice(k, k + 50))
+        cur = s.consensus()
+        assert cur <= prev * (1 + 1e-12) + 1e-27 * start  # monotone down to the rounding floor
+        prev = cur
+    assert prev < 1e-24 * start
+    np.testing.assert_allclose(s.X, np.broadcast_to(x0.mean(0), (n, d)), atol=1e-12)
+    assert np.array_equal(s.X, s.Xt)
+
+
+@pytest.mark.parametrize("Sim", SIMS)
+def test_baseline_equals_textbook_gossip_sgd(Sim):
+    """Eq. (baselinedynamic): with eta = 0, alpha = alpha~ = 1/2 the momentum buffer is a copy
+    and every event is either a local SGD step or a pairwise average."""
+    cfg = W.CONFIGS["cfg1"].scaled(d=13, n_events=400)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    s = Sim(x0, 0.0, 0.5, 0.5, cfg.gamma, grads=G)
+    s.apply(ev.times, ev.wi, ev.wj, ev.slot)
+    ref = x0.copy()
+    for i, j, sl in zip(ev.wi, ev.wj, ev.slot):
+        if j < 0:
+            ref[i] = ref[i] - cfg.gamma * G[sl]
+        else:
+            avg = 0.5 * (ref[i] + ref[j])
+            ref[i] = avg
+            ref[j] = avg.copy()
+    np.testing.assert_allclose(s.X, ref, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(s.Xt, s.X, rtol=0, atol=1e-13)
+
+
+# ---- mean tracker: Eq. (mean) and the remark after (major:delta_f) in App. C -------------
+def test_mean_tracker_identity():
+    cfg = W.CONFIGS["cfg1"].scaled(d=9, n_events=600)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    eta, alpha, at = 0.5, 0.5, 1.7
+    s = OracleSim(x0, eta, alpha, at, cfg.gamma, grads=G)
+    s.apply_stream(ev)
+    gsum = np.zeros(cfg.d)
+    for j, sl in zip(ev.wj, ev.slot):
+        if j < 0:
+            gsum += G[sl]
+    # stored state: the per-worker half-sum (x + x~)/2 is untouched by mixing; sums over workers
+    # are untouched by averaging
+    np.testing.assert_allclose((s.X + s.Xt).sum(0), 2 * x0.sum(0) - 2 * cfg.gamma * gsum, rtol=1e-11, atol=1e-11)
+    # at a common time, mean(x) = mean(x~) = mean(x0) - gamma/n * sum of gradients used
+    xf, xtf = s.flushed(ev.times[-1] + 0.3)
+    want = x0.mean(0) - cfg.gamma / cfg.n * gsum
+    np.testing.assert_allclose(xf.mean(0), want, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(xtf.mean(0), want, rtol=1e-11, atol=1e-12)
+
+
+# ---- brute force: eager integration of the linear ODE with a hand-written matrix exponential
+def _expm_taylor(M):
+    """Scaling and squaring with a plain Taylor series."""
+    nrm = np.abs(M).sum(1).max()
+    s = max(0, int(math.ceil(math.log2(max(nrm, 1e-300)))) + 4)
+    A = M / (2.0 ** s)
+    E, term = np.eye(M.shape[0]), np.eye(M.shape[0])
+    for k in range(1, 30):
+        term = term @ A / k
+        E = E + term
+    for _ in range(s):
+        E = E @ E
+    return E
+
+
+def _brute_force(x0, G, ev, eta, alpha, at, gamma, t_end):
+    """State z = (x_1, x~_1, ..., x_n, x~_n) per column; all workers flow eagerly between
+    consecutive events (Eq. (dynamic)), then the event's jump is applied (App. C, Ito
+    expansion: X - (alpha; alpha~) (e_i - e_j)(e_i - e_j)^T x and X - gamma (g; g))."""
+    n, d = x0.shape
+    gen = np.zeros((2 * n, 2 * n))
+    for w in range(n):
+        gen[2 * w, 2 * w] = -eta
+        gen[2 * w, 2 * w + 1] = eta
+        gen[2 * w + 1, 2 * w] = eta
+        gen[2 * w + 1, 2 * w + 1] = -eta
+    z = np.zeros((2 * n, d))
+    z[0::2] = x0
+    z[1::2] = x0
+    t = 0.0
+    for te, i, j, sl in zip(ev.times, ev.wi, ev.wj, ev.slot):
+        z = _expm_taylor((te - t) * gen) @ z
+        t = te
+        if j < 0:
+            z[2 * i] -= gamma * G[sl]
+            z[2 * i + 1] -= gamma * G[sl]
+        else:
+            m = z[2 * i] - z[2 * j]
+            z[2 * i] -= alpha * m
+            z[2 * i + 1] -= at * m
+            z[2 * j] += alpha * m
+            z[2 * j + 1] += at * m
+    z = _expm_taylor((t_end - t) * gen) @ z
+    return z[0::2], z[1::2]
+
+
+@pytest.mark.parametrize("n,d,graph", [(2, 3, "ring"), (3, 3, "complete"), (5, 2, "ring")])
+@pytest.mark.parametrize("Sim", SIMS)
+def test_brute_force_matrix_exponential(Sim, n, d, graph):
+    r = np.random.default_rng(11)
+    x0 = r.standard_normal((n, d))
+    G = r.standard_normal((n, d))
+    edges = W.make_edges(graph, n)
+    ev = W.poisson_events(n, edges, np.full(len(edges), 0.8), 120, seed=3)
+    eta, alpha, at, gamma = 0.45, 0.5, 1.6, 0.05
+    s = Sim(x0, eta, alpha, at, gamma, grads=G)
+    s.apply(ev.times, ev.wi, ev.wj, ev.slot)
+    t_end = float(ev.times[-1]) + 0.5
+    bx, bxt = _brute_force(x0, G, ev, eta, alpha, at, gamma, t_end)
+    if Sim is OracleSim:
+        fx, fxt = s.flushed(t_end)
+    else:
+        for w in range(n):
+            s.mix(w, t_end)
+        fx, fxt = s.X, s.Xt
+    np.testing.assert_allclose(fx, bx, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(fxt, bxt, rtol=1e-10, atol=1e-11)
+
+
+def test_consensus_at_common_time_matches_flushed_state_and_definition():
+    """App. A: ||pi x||_F^2 with pi = I - 11^T/n, written out as a projection."""
+    cfg = W.CONFIGS["cfg1"].scaled(d=6, n_events=200)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    s = OracleSim(x0, 0.5, 0.5, 1.2, cfg.gamma, grads=G)
+    s.apply_stream(ev)
+    n = cfg.n
+    P = np.eye(n) - np.ones((n, n)) / n
+    assert abs(s.consensus() - np.linalg.norm(P @ s.X, "fro") ** 2) < 1e-11
+    t_eval = float(ev.times[-1]) + 1.0
+    xf, _ = s.flushed(t_eval)
+    assert abs(s.consensus(t_eval) - np.linalg.norm(P @ xf, "fro") ** 2) < 1e-11
+    # flushing to the stored times is the identity only when every worker is already there
+    s2 = OracleSim(x0, 0.5, 0.5, 1.2, cfg.gamma, grads=G)
+    assert s2.consensus(0.0) == s2.consensus()
+
+
+# ---- hand example (closed form worked by hand from Eq. (dynamic)) ------------------------
+@pytest.mark.parametrize("Sim", SIMS)
+def test_hand_example(Sim):
+    # n=2, d=1, eta=.5, alpha=.5, alpha~=1, gamma=.1, x0 = x~0 = (1, 0).
+    # comm(0,1) at t=1: x = x~ so the flow does nothing; m = 1:
+    #   x = (1/2, 1/2), x~ = (1 - 1, 0 + 1) = (0, 1).
+    # gradient g=1 on worker 0 at t=2: dt = 1, e = exp(-1); half-sum 1/4, half-difference 1/4:
+    #   x_0 = 1/4 + e/4 - 1/10,  x~_0 = 1/4 - e/4 - 1/10.
+    s = Sim(np.array([[1.0], [0.0]]), 0.5, 0.5, 1.0, 0.1, grads=np.array([[1.0], [0.0]]))
+    s.apply(*_one([1.0], [0], [1], [-1]))
+    assert np.array_equal(s.X, [[0.5], [0.5]]) and np.array_equal(s.Xt, [[0.0], [1.0]])
+    s.apply(*_one([2.0], [0], [-1], [0]))
+    e = math.exp(-1.0)
+    assert abs(s.X[0, 0] - (0.25 + 0.25 * e - 0.1)) < 1e-15
+    assert abs(s.Xt[0, 0] - (0.25 - 0.25 * e - 0.1)) < 1e-15
+    assert abs(s.X[0, 0] - 0.2419699) < 1e-7 and abs(s.Xt[0, 0] - 0.0580301) < 1e-7
+    assert s.X[1, 0] == 0.5 and s.Xt[1, 0] == 1.0 and list(s.t) == [2.0, 1.0]
+
+
+# ---- structure: locality, column independence, linearity ---------------------------------
+def _levels(ev, n):
+    lvl = np.zeros(n, dtype=np.int64)
+    out = np.zeros(len(ev), dtype=np.int64)
+    for e, (i, j) in enumerate(zip(ev.wi, ev.wj)):
+        l = lvl[i] if j < 0 else max(lvl[i], lvl[j])
+        out[e] = l
+        lvl[i] = l + 1
+        if j >= 0:
+            lvl[j] = l + 1
+    return out
+
+
+def test_order_free_across_disjoint_workers_bit_identical():
+    """Eq. (dynamic) is local to the workers of an event: any reordering that keeps every
+    worker's own order gives the same stored state, bit for bit."""
+    cfg = W.CONFIGS["cfg2"].scaled(d=17, n_events=900)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    par = (0.53, 0.5, 0.7, cfg.gamma)
+    a = OracleSim(x0, *par, grads=G)
+    a.apply_stream(ev)
+    order = np.argsort(_levels(ev, cfg.n), kind="stable")
+    assert not np.array_equal(order, np.arange(len(ev)))
+    b = OracleSim(x0, *par, grads=G)
+    # the checker insists on sorted times within a call: feed level by level, sorted inside
+    lv = _levels(ev, cfg.n)
+    for l in range(lv.max() + 1):
+        idx = np.nonzero(lv == l)[0]
+        b.apply(ev.times[idx], ev.wi[idx], ev.wj[idx], ev.slot[idx])
+    assert np.array_equal(a.X, b.X) and np.array_equal(a.Xt, b.Xt) and np.array_equal(a.t, b.t)
+
+
+def test_columns_do_not_interact_and_thread_split_is_exact():
+    cfg = W.CONFIGS["cfg1"].scaled(d=41, n_events=300)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    par = (0.5, 0.5, 0.9, cfg.gamma)
+    full = OracleSim(x0, *par, grads=G)
+    full.apply_stream(ev)
+    cols = np.array([0, 5, 6, 40])
+    sub = OracleSim(x0[:, cols], *par, grads=G[:, cols])
+    sub.apply_stream(ev)
+    assert np.array_equal(sub.X, full.X[:, cols]) and np.array_equal(sub.Xt, full.Xt[:, cols])
+    thr = OracleSim(x0, *par, grads=G)
+    thr.apply_stream(ev, threads=3)
+    assert np.array_equal(thr.X, full.X) and np.array_equal(thr.Xt, full.Xt) and np.array_equal(thr.t, full.t)
+
+
+def test_linearity_in_x0_and_gradients():
+    cfg = W.CONFIGS["cfg1"].scaled(d=8, n_events=250)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    par = (0.5, 0.5, 1.4, cfg.gamma)
+    a = OracleSim(x0, *par, grads=G)
+    b = OracleSim(2 * x0, *par, grads=2 * G)
+    a.apply_stream(ev)
+    b.apply_stream(ev)
+    assert np.array_equal(2 * a.X, b.X) and np.array_equal(2 * a.Xt, b.Xt)
+    # eta = 0 and zero gradients: x - x~ changes only through (alpha - alpha~) m
+    c = OracleSim(x0, 0.0, 0.5, 0.5, 0.0, grads=0 * G)
+    c.apply_stream(ev)
+    assert np.array_equal(c.X, c.Xt)
+
+
+def test_c_and_numpy_versions_agree_both_orderings():
+    cfg = W.CONFIGS["cfg1"].scaled(d=10, n_events=500)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    for variant in (0, 1):
+        a = OracleSim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=variant)
+        b = NumpySim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=variant)
+        a.apply_stream(ev)
+        b.apply(ev.times, ev.wi, ev.wj, ev.slot)
+        np.testing.assert_allclose(a.X, b.X, rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(a.Xt, b.Xt, rtol=1e-11, atol=1e-12)
+    # the two orderings coincide when eta = 0 and differ otherwise
+    a0 = OracleSim(x0, 0.0, 0.5, 1.3, cfg.gamma, grads=G, variant=0)
+    a1 = OracleSim(x0, 0.0, 0.5, 1.3, cfg.gamma, grads=G, variant=1)
+    a0.apply_stream(ev)
+    a1.apply_stream(ev)
+    np.testing.assert_allclose(a0.X, a1.X, rtol=1e-12, atol=1e-13)
+    b0 = OracleSim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=0)
+    b1 = OracleSim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=1)
+    b0.apply_stream(ev)
+    b1.apply_stream(ev)
+    assert np.abs(b0.X - b1.X).max() > 1e-6
+
+
+def test_checker_rejects_bad_events():
+    x0 = np.zeros((3, 2))
+    s = OracleSim(x0, 0.1, 0.5, 0.5, 0.1, grads=np.zeros((3, 2)), t0=np.array([1.0, 0.0, 0.0]))
+    with pytest.raises(OracleError):
+        s.apply(*_one([0.5], [0], [-1], [0]))  # before the worker's last event
+    with pytest.raises(OracleError):
+        s.apply(*_one([2.0, 1.5], [1, 2], [-1, -1], [1, 2]))  # unsorted
+    with pytest.raises(OracleError):
+        s.apply(*_one([2.0], [1], [1], [-1]))  # i == j
+    with pytest.raises(OracleError):
+        s.apply(*_one([2.0], [1], [-1], [7]))  # slot out of range
+
+
+# ---- spectral quantities: Def. 3.1, Eq. (2), Eq. (3), Prop. 3.6 ---------------------------
+@pytest.mark.parametrize("n,lam", [(4, 1.0), (16, 0.5), (32, 2.0), (64, 0.5)])
+def test_ring_closed_forms(n, lam):
+    e = W.ring_edges(n)
+    L = spectral.laplacian(n, e, np.full(len(e), lam))
+    # eigenvalues of a weighted cycle: lam (2 - 2 cos(2 pi k / n)); effective resistance of
+    # an edge of a cycle of n unit resistors: (n-1)/n
+    assert abs(spectral.chi1(L) - 1.0 / (lam * (2 - 2 * math.cos(2 * math.pi / n)))) < 1e-9 * n * n
+    assert abs(spectral.chi2(L, e) - (n - 1) / (2 * n * lam)) < 1e-12
+
+
+@pytest.mark.parametrize("n,lam", [(4, 1.0), (16, 1 / 15), (9, 0.3)])
+def test_complete_closed_forms(n, lam):
+    e = W.complete_edges(n)
+    L = spectral.laplacian(n, e, np.full(len(e), lam))
+    # Lambda = lam (n I - 11^T): chi_1 = chi_2 = 1/(n lam)  ("chi_1 = chi_2 for the complete graph", Sec. 4.2)
+    assert abs(spectral.chi1(L) - 1 / (n * lam)) < 1e-12
+    assert abs(spectral.chi2(L, e) - 1 / (n * lam)) < 1e-12
+    eta, alpha, at, _, _ = spectral.prescribe(n, e, np.full(len(e), lam))
+    assert abs(at - 0.5) < 1e-12 and abs(eta - n * lam / 2) < 1e-12 and alpha == 0.5
+
+
+def test_laplacian_definition_and_trace():
+    n = 6
+    e = W.exponential_edges(8)[:5]
+    lam = np.array([0.5, 1.0, 2.0, 0.25, 3.0])
+    L = spectral.laplacian(8, e, lam)
+    x = np.random.default_rng(0).standard_normal(8)
+    assert abs(x @ L @ x - sum(l * (x[i] - x[j]) ** 2 for (i, j), l in zip(e, lam))) < 1e-12
+    assert abs(np.trace(L) / 2 - lam.sum()) < 1e-12  # Prop. 3.6: Tr(Lambda)/2 communications per unit time
+    assert np.allclose(L @ np.ones(8), 0)
+
+
+def test_printed_chi_values_n16():
+    want = {}
+    with open(os.path.join(GOLDEN, "chi_n16_topologies.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            g, c1, c2 = line.split()
+            want[g] = (float(c1), float(c2))
+    assert set(want) == {"complete", "exponential", "ring"}
+    for g, (c1, c2) in want.items():
+        e = W.make_edges(g, 16)
+        _, _, _, h1, h2 = spectral.prescribe(16, e, W.edge_rates_per_worker(16, e, 1.0))
+        assert round(h1) == c1 and round(h2) == c2, (g, h1, h2)
+        assert h2 <= h1 * (1 + 1e-12)  # Eq. (3): chi_2 <= chi_1
+
+
+def test_prescription_formulas():
+    e = W.ring_edges(64)
+    eta, alpha, at, c1, c2 = spectral.prescribe(64, e, np.full(64, 0.5))
+    assert abs(eta * 2 * math.sqrt(c1 * c2) - 1) < 1e-12
+    assert abs(at - 0.5 * math.sqrt(c1 / c2)) < 1e-12 and alpha == 0.5
+    assert spectral.prescribe(64, e, np.full(64, 0.5), accelerated=False)[:3] == (0.0, 0.5, 0.5)
