@@ -1,0 +1,245 @@
+/*
+ * a2cid2.h -- C ABI of the A2CiD2 event-update engine (one NVIDIA B200, sm_100a).
+ *
+ * The engine holds a population of n simulated asynchronous workers. Worker i owns a
+ * parameter row x_i and a continuous-momentum row x~_i (stacked [n, d] device buffers) and a
+ * last-event time t_i. Events arrive as a time-sorted stream and are applied as the paper
+ * "A2CiD2: Accelerating Asynchronous Communication in Decentralized Deep Learning" defines
+ * them (Sec. 3.2, Eq. (dynamic); Algorithm 1):
+ *
+ *   mixing    before any update of worker w at time t, (x_w, x~_w) is advanced over t - t_w by
+ *             the flow dx = eta (x~ - x) dt, dx~ = eta (x - x~) dt, in closed form:
+ *             c = (1 - exp(-2 eta (t - t_w))) / 2,  x_w -= c (x_w - x~_w),  x~_w += c (x_w - x~_w).
+ *   gradient  x_i -= gamma g,  x~_i -= gamma g,  t_i = t          (g = one row of the gradient buffer)
+ *   comm      m = x_i - x_j (taken after both are mixed to t);
+ *             x_i -= alpha m,  x~_i -= alpha~ m,  x_j += alpha m,  x~_j += alpha~ m,  t_i = t_j = t.
+ *
+ * and the consensus distance sum_i |x_i - xbar|^2 (App. A) is reduced on the device.
+ *
+ * Conventions
+ *   - Every function returns an int status (A2_OK = 0, negative on error) unless stated.
+ *     No exception, abort or exit crosses this boundary. Invalid input is rejected before any
+ *     device work and leaves the state untouched. a2cid2_last_error() gives the text of the
+ *     last failure on a handle (or of the last failure in a handle-less call, per thread).
+ *   - "host" pointers are ordinary CPU memory, read or written before the call returns.
+ *     "device" pointers are CUDA global memory on the current device and are only borrowed.
+ *   - Device work is issued on the stream given to a2cid2_bind() and is asynchronous: it is
+ *     ordered with other work on that stream. Calls that return results to the host
+ *     (consensus distance, read_state) wait for the stream.
+ *   - A handle is not thread-safe; use it from one thread at a time.
+ *   - There is no CPU path: without a CUDA device every device call fails with A2_ECUDA.
+ */
+#ifndef A2CID2_H
+#define A2CID2_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct a2cid2 a2cid2_t;             /* engine handle; owned by the library            */
+typedef struct a2cid2_sched a2cid2_sched_t; /* host-only schedule of an event stream          */
+typedef struct a2cid2_plan a2cid2_plan_t;   /* a schedule whose descriptors are on the device  */
+
+enum {
+    A2_OK = 0,
+    A2_EINVAL = -1, /* bad argument (NULL, size, alignment, non-finite parameter, bad flag)     */
+    A2_EORDER = -2, /* times decrease within the call, or an event precedes its worker's t_i   */
+    A2_ERANGE = -3, /* worker index or gradient slot out of range, i == j, or both/neither of
+                       (wj, slot) given                                                         */
+    A2_ENOMEM = -4, /* host or device allocation failed                                         */
+    A2_ECUDA = -5,  /* a CUDA call failed (text in a2cid2_last_error)                           */
+    A2_ESTATE = -6  /* call out of sequence: not bound, plan does not match the handle's times  */
+};
+
+enum { A2_F32 = 0, A2_BF16 = 1 }; /* storage type of x, x~ and the gradient buffer; math is fp32 */
+
+/* Scheduling flags. */
+enum {
+    A2_SCHED_FUSE = 1u /* fold the gradient events that directly precede a communication of the
+                          same worker into that communication's item, so their rows are read
+                          and written once (the arithmetic per element is unchanged)           */
+};
+
+/* Kinds of elementary operation inside an item. */
+enum { A2_OP_GRAD_A = 0, A2_OP_GRAD_B = 1, A2_OP_COMM = 2 };
+
+/* Variants of the order of operations at a communication event. */
+enum {
+    A2_MSG_AFTER_MIX = 0, /* message x_i - x_j taken at the event time, as Eq. (dynamic) states */
+    A2_MSG_BEFORE_MIX = 1 /* message taken from the un-mixed buffers, as Algorithm 1 is printed */
+};
+
+/* One item of a batch: all the work done on one worker (b = -1) or one pair of workers. */
+typedef struct a2cid2_item_info {
+    int32_t a, b;           /* worker rows; b = -1 for a gradient-only item                    */
+    int32_t slot_a, slot_b; /* gradient rows read for worker a / b, or -1                       */
+    int64_t first_op;       /* index of the item's first elementary operation                   */
+    int32_t n_ops;          /* operations applied, in order, while the rows sit in registers    */
+    int32_t batch;          /* batch (dependency level) the item belongs to                     */
+} a2cid2_item_info;
+
+/* Counters of one a2cid2_apply_events / a2cid2_plan_run call (all device figures are what the
+ * descriptors imply, not hardware counters). */
+typedef struct a2cid2_stats {
+    int64_t n_events, n_comm, n_grad;
+    int64_t n_batches;  /* dependency levels                                                    */
+    int64_t n_launches; /* event-kernel launches (a batch is split if it exceeds a launch's caps) */
+    int64_t n_items;
+    int64_t bytes_moved;       /* rows read + rows written by the items, times d, times element size */
+    int64_t bytes_one_by_one;  /* the same stream applied one event per item: comm 8 rows, gradient 5 */
+    int64_t descriptor_bytes;  /* host-to-device bytes of the descriptors                        */
+    double host_ms;            /* validation + scheduling + descriptor packing time on the host   */
+} a2cid2_stats;
+
+/* ------------------------------------------------------------------------------------------
+ * Engine
+ * ------------------------------------------------------------------------------------------ */
+
+/* Create an engine for n >= 2 workers of d >= 1 parameters with the hyper-parameters of
+ * Eq. (dynamic) (eta >= 0; all finite). storage_dtype is A2_F32 or A2_BF16. Allocates only
+ * small host/device bookkeeping; the state buffers come from a2cid2_bind. *out receives the
+ * handle, to be released with a2cid2_destroy. Times start at t_i = 0 (Algorithm 1, init). */
+int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_tilde, double gamma,
+                  int32_t storage_dtype, a2cid2_t** out);
+
+/* Select A2_MSG_AFTER_MIX (default) or A2_MSG_BEFORE_MIX for later events. */
+int a2cid2_set_variant(a2cid2_t* h, int32_t variant);
+
+/* Lend the device buffers: x and x_tilde are [n, row_pitch_elems], grads is
+ * [n_grad_slots, row_pitch_elems] (may be NULL with n_grad_slots = 0 if no gradient event is
+ * ever applied), all of the storage type, row-major, 16-byte aligned. row_pitch_elems >= d and
+ * a multiple of 8; the columns between d and the pitch are padding that the library may
+ * overwrite. cuda_stream is a cudaStream_t (NULL = default stream). The caller keeps ownership
+ * and must keep the buffers alive until a2cid2_sync/destroy. May be called again to re-bind. */
+int a2cid2_bind(a2cid2_t* h, void* x, void* x_tilde, void* grads, int32_t n_grad_slots,
+                int64_t row_pitch_elems, void* cuda_stream);
+
+/* Copy a dense host [n, d] array of the storage type into x; x~ from host_x_tilde, or a copy
+ * of x when NULL (Algorithm 1: x~ <- x); times from host_t[n], or zeros when NULL. Waits. */
+int a2cid2_write_state(a2cid2_t* h, const void* host_x, const void* host_x_tilde, const double* host_t);
+
+/* Copy dense host rows [n_slots, d] into gradient rows first_slot.. . Waits. */
+int a2cid2_write_grads(a2cid2_t* h, int32_t first_slot, int32_t n_slots, const void* host_g);
+
+/* Copy x, x~ (dense [n, d], storage type) and t[n] to the host; any pointer may be NULL. Waits. */
+int a2cid2_read_state(a2cid2_t* h, void* host_x, void* host_x_tilde, double* host_t);
+
+/* Copy the workers' last-event times t[n] (kept on the host) without touching the device. */
+int a2cid2_times(const a2cid2_t* h, double* host_t);
+
+/* Overwrite the workers' last-event times (host array t[n], finite) without touching x, x~:
+ * for callers that fill the bound buffers themselves, and for resuming from a checkpoint. */
+int a2cid2_set_times(a2cid2_t* h, const double* host_t);
+
+/* Apply n_events events (host arrays, read before return). Event e happens at times[e]
+ * (finite, non-decreasing, and >= the stored t of its workers). wj[e] >= 0: communication
+ * between wi[e] and wj[e], grad_slot[e] must be -1. wj[e] == -1: gradient event on wi[e]
+ * using gradient row grad_slot[e] >= 0. The stream is validated, packed into batches of
+ * disjoint workers that keep every worker's own order (flags: A2_SCHED_*), and one fused
+ * kernel per batch is queued on the bound stream. stats may be NULL. Asynchronous. */
+int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, const int32_t* wi,
+                        const int32_t* wj, const int32_t* grad_slot, uint32_t flags, a2cid2_stats* stats);
+
+/* Consensus distance sum_i |x_i - xbar|^2, xbar = (1/n) sum_i x_i (App. A). With t_eval = NaN
+ * the stored rows are used as they are (each at its own t_i). With a finite
+ * t_eval >= max_i t_i every row is first mixed forward to t_eval in registers (nothing is
+ * written back). Waits for the stream; *out is a host double. */
+int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out);
+
+/* Wait for all work queued by this handle; returns the first deferred CUDA error, if any. */
+int a2cid2_sync(a2cid2_t* h);
+
+/* Text of the last error on h (h may be NULL: last error of a call that had no handle, for
+ * the calling thread). Never NULL; valid until the next call on the same handle/thread. */
+const char* a2cid2_last_error(const a2cid2_t* h);
+
+/* Release the handle and everything the library allocated for it (waits for the stream).
+ * Plans created from it must be destroyed first. NULL is allowed. */
+void a2cid2_destroy(a2cid2_t* h);
+
+/* ------------------------------------------------------------------------------------------
+ * Plans: schedule once, run later (device-resident descriptors)
+ * ------------------------------------------------------------------------------------------ */
+
+/* Validate and schedule an event stream as a2cid2_apply_events does and upload its
+ * descriptors, but launch nothing. t_start[n] gives the workers' times the stream starts
+ * from (NULL = the handle's current times); a2cid2_plan_run checks them against the handle. */
+int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, const double* times,
+                       const int32_t* wi, const int32_t* wj, const int32_t* grad_slot, uint32_t flags,
+                       a2cid2_plan_t** out);
+
+/* The plan's schedule, for inspection (owned by the plan). */
+const a2cid2_sched_t* a2cid2_plan_sched(const a2cid2_plan_t* p);
+
+/* Queue batches [first_batch, first_batch + n_batches) of the plan; n_batches = -1 means all
+ * remaining. Batches must be run in order, each exactly once, and the handle's times must be
+ * those the plan expects (A2_ESTATE otherwise). Asynchronous. stats may be NULL. */
+int a2cid2_plan_run(a2cid2_t* h, a2cid2_plan_t* p, int64_t first_batch, int64_t n_batches, a2cid2_stats* stats);
+
+void a2cid2_plan_destroy(a2cid2_plan_t* p);
+
+/* ------------------------------------------------------------------------------------------
+ * Host scheduler (no device needed)
+ * ------------------------------------------------------------------------------------------ */
+
+/* Pack a time-sorted event stream into batches. An event's batch is one more than the latest
+ * batch of the workers it touches (greedy, as early as possible), so inside a batch no worker
+ * appears in two items and every worker's events keep their order; since an event only
+ * touches its own workers' rows (Eq. (dynamic) is local), running the batches in order gives
+ * the state of the time-ordered run. With A2_SCHED_FUSE, gradient events of a worker are held
+ * back and applied, in order, inside the next communication item of that worker (or in a
+ * gradient-only item at the end of the stream, or when max_ops_per_item is reached or the
+ * gradient slot changes). t_last[n] are the workers' times at the start (NULL = zeros).
+ * max_ops_per_item <= 0 selects the default. Validation and error codes as in
+ * a2cid2_apply_events. */
+int a2cid2_sched_create(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events,
+                        const double* times, const int32_t* wi, const int32_t* wj, const int32_t* grad_slot,
+                        uint32_t flags, int32_t max_ops_per_item, a2cid2_sched_t** out);
+
+int64_t a2cid2_sched_num_batches(const a2cid2_sched_t* s);
+int64_t a2cid2_sched_num_items(const a2cid2_sched_t* s);
+int64_t a2cid2_sched_num_ops(const a2cid2_sched_t* s);
+
+/* Items of batch b are [*first_item, *first_item + *n_items). */
+int a2cid2_sched_batch_items(const a2cid2_sched_t* s, int64_t b, int64_t* first_item, int64_t* n_items);
+
+int a2cid2_sched_item(const a2cid2_sched_t* s, int64_t item, a2cid2_item_info* out);
+
+/* Operations [first_op, first_op + n_ops): the index of the event each one applies (into the
+ * arrays given to a2cid2_sched_create) and its kind (A2_OP_*). Either output may be NULL. */
+int a2cid2_sched_ops(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, int64_t* event_index, int32_t* kind);
+
+/* Workers' times after the whole schedule has run. */
+int a2cid2_sched_t_final(const a2cid2_sched_t* s, double* t_out);
+
+/* Fill the descriptor-derived counters (events, batches, items, launches, bytes for d columns
+ * of elem_bytes each) for batches [first_batch, first_batch + n_batches); -1 = all remaining. */
+int a2cid2_sched_stats(const a2cid2_sched_t* s, int64_t first_batch, int64_t n_batches, int64_t d,
+                       int32_t elem_bytes, a2cid2_stats* out);
+
+void a2cid2_sched_destroy(a2cid2_sched_t* s);
+
+/* ------------------------------------------------------------------------------------------
+ * Graph quantities and the parameter prescription (host only)
+ * ------------------------------------------------------------------------------------------ */
+
+/* For the graph with n nodes and n_edges edges (ei[k], ej[k]) of rates lambda[k] > 0, form the
+ * Laplacian of Def. 3.1 and return chi_1 = 1 / lambda_2(Lambda) (Eq. (2), algebraic
+ * connectivity) and chi_2 = 1/2 max over edges of the effective resistance
+ * (e_i - e_j)^T Lambda^+ (e_i - e_j) (Eq. (3)). A2_EINVAL if the graph is not connected. */
+int a2cid2_graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda,
+                     double* chi1, double* chi2);
+
+/* Prop. 3.6: accelerated != 0: eta = 1/(2 sqrt(chi1 chi2)), alpha = 1/2,
+ * alpha~ = 1/2 sqrt(chi1/chi2); accelerated == 0: eta = 0, alpha = alpha~ = 1/2. */
+int a2cid2_prescribe(double chi1, double chi2, int32_t accelerated, double* eta, double* alpha, double* alpha_tilde);
+
+/* Library version string. */
+const char* a2cid2_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* A2CID2_H */

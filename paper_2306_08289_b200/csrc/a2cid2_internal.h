@@ -1,0 +1,108 @@
+// Internal declarations shared by the host scheduler, the kernels' launchers and the C ABI.
+#pragma once
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "a2cid2.h"
+
+namespace a2 {
+
+// ---- error text ---------------------------------------------------------------------------
+void set_thread_error(const std::string& msg);
+const char* thread_error();
+
+// ---- host schedule ------------------------------------------------------------------------
+struct SchedOp {
+    int64_t event;    // index into the caller's event arrays
+    int32_t kind;     // A2_OP_*
+    double t;         // event time
+    double t_prev_a;  // time worker a was last updated before this op (GRAD_A, COMM)
+    double t_prev_b;  // same for worker b (GRAD_B, COMM)
+};
+
+struct SchedItem {
+    int32_t a, b, slot_a, slot_b;
+    int64_t first_op;
+    int32_t n_ops;
+    int32_t batch;
+};
+
+}  // namespace a2
+
+struct a2cid2_sched {
+    int32_t n = 0;
+    int32_t n_grad_slots = 0;
+    uint32_t flags = 0;
+    int64_t n_events = 0;
+    std::vector<a2::SchedItem> items;  // sorted by batch, creation order inside a batch
+    std::vector<a2::SchedOp> ops;      // in item order
+    std::vector<int64_t> batch_first;  // items of batch b: [batch_first[b], batch_first[b+1])
+    std::vector<double> t_start, t_final;
+};
+
+namespace a2 {
+
+// Builds a schedule; returns A2_OK or an error code with the text in `err`.
+int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
+                   const int32_t* wi, const int32_t* wj, const int32_t* slot, uint32_t flags,
+                   int32_t max_ops_per_item, a2cid2_sched** out, std::string& err);
+
+void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out);
+
+// ---- device descriptors (layout shared by host packing and the event kernel) ---------------
+struct DevItem {
+    int32_t a, b, slot_a, slot_b;
+    int32_t op_first;  // relative to the launch's first op
+    int32_t op_count;
+};
+
+struct DevOp {
+    int32_t kind;
+    int32_t pad;
+    double t;         // event time
+    double t_prev_a;  // worker a's last-event time before this op
+    double t_prev_b;  // worker b's
+};
+
+constexpr int kMaxItemsPerLaunch = 128;
+constexpr int kMaxOpsPerLaunch = 512;
+constexpr int kDefaultMaxOpsPerItem = 32;
+
+struct EventLaunch {
+    void* x;
+    void* xt;
+    const void* g;
+    int64_t pitch;  // elements
+    int64_t d;
+    const DevItem* items;  // device
+    const DevOp* ops;      // device
+    int32_t n_items;
+    int32_t n_ops;
+    double eta;
+    float alpha, alpha_tilde, gamma;
+    int32_t variant;
+    int32_t dtype;
+};
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int event_ctas_per_sm[2] = {0, 0};  // per storage type
+    int consensus_ctas_per_sm = 0;
+};
+
+// Launchers (kernels.cu). All return a cudaError_t cast to int (0 = success).
+int query_device(DeviceInfo* info);
+int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream);
+// Consensus distance. dt (device, n doubles) is NULL for the stored state; partials is device
+// scratch of n_partials doubles; out is a device double.
+int consensus_grid(const DeviceInfo& dev);
+int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double eta,
+                     const double* dt, double* partials, int n_partials, double* out, void* stream);
+
+// ---- spectral (spectral.cpp) -----------------------------------------------------------------
+int graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda, double* chi1,
+              double* chi2, std::string& err);
+
+}  // namespace a2

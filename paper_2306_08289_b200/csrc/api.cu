@@ -1,0 +1,602 @@
+// C ABI of the engine: handle, plans, validation, descriptor upload, launches.
+#include <cuda_runtime.h>
+
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "a2cid2_internal.h"
+
+namespace a2 {
+
+namespace {
+thread_local std::string g_thread_error = "";
+}
+
+void set_thread_error(const std::string& msg) { g_thread_error = msg; }
+const char* thread_error() { return g_thread_error.c_str(); }
+
+}  // namespace a2
+
+using a2::DevItem;
+using a2::DevOp;
+
+namespace {
+
+struct LaunchRange {
+    int64_t item0, item1;  // items of the plan covered by this launch
+    int64_t op0, op1;
+};
+
+// Grow-only pinned + device buffer pair used to ship the descriptors of one apply_events call.
+struct Arena {
+    void* host = nullptr;  // pinned
+    void* dev = nullptr;
+    size_t cap = 0;
+    cudaEvent_t copied = nullptr;  // recorded after the last H2D copy out of `host`
+    bool in_flight = false;
+};
+
+size_t elem_bytes(int32_t dtype) { return dtype == A2_BF16 ? 2 : 4; }
+
+}  // namespace
+
+struct a2cid2 {
+    int32_t n = 0;
+    int64_t d = 0;
+    double eta = 0, alpha = 0, alpha_tilde = 0, gamma = 0;
+    int32_t dtype = A2_F32;
+    int32_t variant = A2_MSG_AFTER_MIX;
+    // borrowed buffers
+    void* x = nullptr;
+    void* xt = nullptr;
+    void* g = nullptr;
+    int32_t n_slots = 0;
+    int64_t pitch = 0;
+    cudaStream_t stream = nullptr;
+    bool bound = false;
+    int device = -1;
+    // host-side times (authoritative; the kernels get them through the descriptors)
+    std::vector<double> t;
+    // library-owned scratch
+    a2::DeviceInfo dev;
+    bool dev_ok = false;
+    double* d_partials = nullptr;  // consensus_grid doubles + 1 result
+    double* d_dt = nullptr;        // n doubles
+    double* h_pinned = nullptr;    // n + 1 doubles: dt staging and the result
+    Arena arena[2];
+    int arena_next = 0;
+    int64_t live_plans = 0;
+    std::string err;
+};
+
+struct a2cid2_plan {
+    a2cid2* owner = nullptr;
+    a2cid2_sched* sched = nullptr;
+    void* d_desc = nullptr;  // items then ops
+    DevItem* d_items = nullptr;
+    DevOp* d_ops = nullptr;
+    std::vector<LaunchRange> launches;
+    std::vector<int64_t> batch_launch_first;  // launches of batch b: [first[b], first[b+1])
+    int64_t next_batch = 0;
+    bool uses_gradients = false;
+    std::vector<double> t_expect;  // workers' times the next batch expects
+};
+
+namespace {
+
+int fail(a2cid2* h, int code, const std::string& msg) {
+    if (h) h->err = msg;
+    a2::set_thread_error(msg);
+    return code;
+}
+
+int fail_cuda(a2cid2* h, cudaError_t e, const char* what) {
+    std::string m = std::string(what) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
+    return fail(h, A2_ECUDA, m);
+}
+
+#define A2_CUDA(h, call)                                         \
+    do {                                                         \
+        cudaError_t e__ = (call);                                \
+        if (e__ != cudaSuccess) return fail_cuda(h, e__, #call); \
+    } while (0)
+
+int ensure_device(a2cid2* h) {
+    if (h->dev_ok) return A2_OK;
+    int rc = a2::query_device(&h->dev);
+    if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "device query");
+    A2_CUDA(h, cudaGetDevice(&h->device));
+    const int np = a2::consensus_grid(h->dev);
+    A2_CUDA(h, cudaMalloc(&h->d_partials, sizeof(double) * (size_t)(np + 1)));
+    A2_CUDA(h, cudaMalloc(&h->d_dt, sizeof(double) * (size_t)h->n));
+    A2_CUDA(h, cudaMallocHost(&h->h_pinned, sizeof(double) * (size_t)(h->n + 1)));
+    h->dev_ok = true;
+    return A2_OK;
+}
+
+int need_bound(a2cid2* h) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (!h->bound) return fail(h, A2_ESTATE, "no buffers bound (call a2cid2_bind first)");
+    return A2_OK;
+}
+
+// Split every batch into launches that respect the per-launch caps.
+void make_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches, std::vector<int64_t>& batch_first) {
+    const int64_t nb = (int64_t)s.batch_first.size() - 1;
+    batch_first.assign((size_t)nb + 1, 0);
+    for (int64_t b = 0; b < nb; ++b) {
+        batch_first[(size_t)b] = (int64_t)launches.size();
+        int64_t i = s.batch_first[(size_t)b];
+        const int64_t iend = s.batch_first[(size_t)b + 1];
+        while (i < iend) {
+            LaunchRange L{i, i, s.items[(size_t)i].first_op, s.items[(size_t)i].first_op};
+            while (L.item1 < iend && (L.item1 - L.item0) < a2::kMaxItemsPerLaunch &&
+                   (L.op1 - L.op0) + s.items[(size_t)L.item1].n_ops <= a2::kMaxOpsPerLaunch) {
+                L.op1 += s.items[(size_t)L.item1].n_ops;
+                L.item1 += 1;
+            }
+            launches.push_back(L);
+            i = L.item1;
+        }
+    }
+    batch_first[(size_t)nb] = (int64_t)launches.size();
+}
+
+size_t desc_bytes(const a2cid2_sched& s) {
+    const size_t items = (s.items.size() * sizeof(DevItem) + 15) & ~size_t(15);
+    return items + s.ops.size() * sizeof(DevOp);
+}
+
+// Write device descriptors into `dst` (items, then ops at the 16-byte aligned offset returned).
+size_t pack_descriptors(const a2cid2_sched& s, const std::vector<LaunchRange>& launches, void* dst) {
+    DevItem* di = static_cast<DevItem*>(dst);
+    const size_t ops_off = (s.items.size() * sizeof(DevItem) + 15) & ~size_t(15);
+    DevOp* dop = reinterpret_cast<DevOp*>(static_cast<char*>(dst) + ops_off);
+    for (const LaunchRange& L : launches) {
+        for (int64_t k = L.item0; k < L.item1; ++k) {
+            const a2::SchedItem& it = s.items[(size_t)k];
+            di[k] = DevItem{it.a, it.b, it.slot_a, it.slot_b, (int32_t)(it.first_op - L.op0), it.n_ops};
+        }
+    }
+    for (size_t o = 0; o < s.ops.size(); ++o) {
+        const a2::SchedOp& op = s.ops[o];
+        dop[o] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
+    }
+    return ops_off;
+}
+
+int queue_launches(a2cid2* h, const std::vector<LaunchRange>& launches, int64_t l0, int64_t l1, const DevItem* d_items,
+                   const DevOp* d_ops) {
+    for (int64_t l = l0; l < l1; ++l) {
+        const LaunchRange& R = launches[(size_t)l];
+        a2::EventLaunch L;
+        L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
+        L.items = d_items + R.item0;
+        L.ops = d_ops + R.op0;
+        L.n_items = (int32_t)(R.item1 - R.item0);
+        L.n_ops = (int32_t)(R.op1 - R.op0);
+        L.eta = h->eta;
+        L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
+        L.variant = h->variant; L.dtype = h->dtype;
+        const int rc = a2::launch_events(L, h->dev, h->stream);
+        if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
+    }
+    return A2_OK;
+}
+
+// After batches [b0, b1) ran: every worker's time is that of its last operation in them.
+void advance_times(const a2cid2_sched& s, int64_t b0, int64_t b1, std::vector<double>& t) {
+    for (int64_t k = s.batch_first[(size_t)b0]; k < s.batch_first[(size_t)b1]; ++k) {
+        const a2::SchedItem& it = s.items[(size_t)k];
+        for (int32_t o = 0; o < it.n_ops; ++o) {
+            const a2::SchedOp& op = s.ops[(size_t)(it.first_op + o)];
+            if (op.kind != A2_OP_GRAD_B) t[(size_t)it.a] = op.t;
+            if (op.kind != A2_OP_GRAD_A) t[(size_t)it.b] = op.t;
+        }
+    }
+}
+
+bool needs_gradients(const a2cid2_sched& s) {
+    for (const a2::SchedItem& it : s.items)
+        if (it.slot_a >= 0 || it.slot_b >= 0) return true;
+    return false;
+}
+
+double now_ms() {
+    using namespace std::chrono;
+    return duration<double, std::milli>(steady_clock::now().time_since_epoch()).count();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* a2cid2_version(void) { return "a2cid2-b200 0.1 (sm_100a)"; }
+
+const char* a2cid2_last_error(const a2cid2_t* h) { return h ? h->err.c_str() : a2::thread_error(); }
+
+int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_tilde, double gamma,
+                  int32_t storage_dtype, a2cid2_t** out) {
+    if (!out) return fail(nullptr, A2_EINVAL, "out is NULL");
+    *out = nullptr;
+    if (n < 2 || n > 4096) return fail(nullptr, A2_EINVAL, "need 2 <= n <= 4096 workers");
+    if (d < 1 || d > (int64_t(1) << 40)) return fail(nullptr, A2_EINVAL, "need 1 <= d <= 2^40");
+    if (!std::isfinite(eta) || !std::isfinite(alpha) || !std::isfinite(alpha_tilde) || !std::isfinite(gamma))
+        return fail(nullptr, A2_EINVAL, "hyper-parameters must be finite");
+    if (eta < 0) return fail(nullptr, A2_EINVAL, "eta must be >= 0");
+    if (storage_dtype != A2_F32 && storage_dtype != A2_BF16) return fail(nullptr, A2_EINVAL, "unknown storage type");
+    a2cid2* h = new (std::nothrow) a2cid2();
+    if (!h) return fail(nullptr, A2_ENOMEM, "out of host memory");
+    h->n = n; h->d = d; h->eta = eta; h->alpha = alpha; h->alpha_tilde = alpha_tilde; h->gamma = gamma;
+    h->dtype = storage_dtype;
+    h->t.assign((size_t)n, 0.0);
+    *out = h;
+    return A2_OK;
+}
+
+int a2cid2_set_variant(a2cid2_t* h, int32_t variant) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (variant != A2_MSG_AFTER_MIX && variant != A2_MSG_BEFORE_MIX) return fail(h, A2_EINVAL, "unknown variant");
+    h->variant = variant;
+    return A2_OK;
+}
+
+int a2cid2_bind(a2cid2_t* h, void* x, void* x_tilde, void* grads, int32_t n_grad_slots, int64_t row_pitch_elems,
+                void* cuda_stream) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (!x || !x_tilde) return fail(h, A2_EINVAL, "x or x_tilde is NULL");
+    if (n_grad_slots < 0 || (n_grad_slots > 0 && !grads)) return fail(h, A2_EINVAL, "bad gradient buffer");
+    if (row_pitch_elems < h->d || row_pitch_elems % 8 != 0)
+        return fail(h, A2_EINVAL, "row pitch must be >= d and a multiple of 8 elements");
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(x_tilde) | reinterpret_cast<uintptr_t>(grads)) & 15)
+        return fail(h, A2_EINVAL, "buffers must be 16-byte aligned");
+    if (x == x_tilde) return fail(h, A2_EINVAL, "x and x_tilde must be distinct buffers");
+    const int rc = ensure_device(h);
+    if (rc != A2_OK) return rc;
+    h->x = x; h->xt = x_tilde; h->g = n_grad_slots > 0 ? grads : nullptr;
+    h->n_slots = n_grad_slots; h->pitch = row_pitch_elems;
+    h->stream = static_cast<cudaStream_t>(cuda_stream);
+    h->bound = true;
+    return A2_OK;
+}
+
+int a2cid2_write_state(a2cid2_t* h, const void* host_x, const void* host_x_tilde, const double* host_t) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!host_x) return fail(h, A2_EINVAL, "host_x is NULL");
+    if (host_t)
+        for (int32_t w = 0; w < h->n; ++w)
+            if (!std::isfinite(host_t[w])) return fail(h, A2_EINVAL, "non-finite worker time");
+    const size_t eb = elem_bytes(h->dtype);
+    const size_t row = (size_t)h->d * eb, pitch = (size_t)h->pitch * eb;
+    A2_CUDA(h, cudaMemcpy2DAsync(h->x, pitch, host_x, row, row, (size_t)h->n, cudaMemcpyHostToDevice, h->stream));
+    A2_CUDA(h, cudaMemcpy2DAsync(h->xt, pitch, host_x_tilde ? host_x_tilde : host_x, row, row, (size_t)h->n,
+                                 cudaMemcpyHostToDevice, h->stream));
+    A2_CUDA(h, cudaStreamSynchronize(h->stream));
+    for (int32_t w = 0; w < h->n; ++w) h->t[(size_t)w] = host_t ? host_t[w] : 0.0;
+    return A2_OK;
+}
+
+int a2cid2_write_grads(a2cid2_t* h, int32_t first_slot, int32_t n_slots, const void* host_g) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!host_g || first_slot < 0 || n_slots < 0 || first_slot + n_slots > h->n_slots)
+        return fail(h, A2_ERANGE, "gradient slot range out of bounds");
+    if (n_slots == 0) return A2_OK;
+    const size_t eb = elem_bytes(h->dtype);
+    const size_t row = (size_t)h->d * eb, pitch = (size_t)h->pitch * eb;
+    char* dst = static_cast<char*>(h->g) + (size_t)first_slot * pitch;
+    A2_CUDA(h, cudaMemcpy2DAsync(dst, pitch, host_g, row, row, (size_t)n_slots, cudaMemcpyHostToDevice, h->stream));
+    A2_CUDA(h, cudaStreamSynchronize(h->stream));
+    return A2_OK;
+}
+
+int a2cid2_read_state(a2cid2_t* h, void* host_x, void* host_x_tilde, double* host_t) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    const size_t eb = elem_bytes(h->dtype);
+    const size_t row = (size_t)h->d * eb, pitch = (size_t)h->pitch * eb;
+    if (host_x)
+        A2_CUDA(h, cudaMemcpy2DAsync(host_x, row, h->x, pitch, row, (size_t)h->n, cudaMemcpyDeviceToHost, h->stream));
+    if (host_x_tilde)
+        A2_CUDA(h, cudaMemcpy2DAsync(host_x_tilde, row, h->xt, pitch, row, (size_t)h->n, cudaMemcpyDeviceToHost, h->stream));
+    A2_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (host_t) std::memcpy(host_t, h->t.data(), sizeof(double) * (size_t)h->n);
+    return A2_OK;
+}
+
+int a2cid2_times(const a2cid2_t* h, double* host_t) {
+    if (!h || !host_t) return fail(nullptr, A2_EINVAL, "NULL argument");
+    std::memcpy(host_t, h->t.data(), sizeof(double) * (size_t)h->n);
+    return A2_OK;
+}
+
+int a2cid2_set_times(a2cid2_t* h, const double* host_t) {
+    if (!h || !host_t) return fail(h, A2_EINVAL, "NULL argument");
+    for (int32_t w = 0; w < h->n; ++w)
+        if (!std::isfinite(host_t[w])) return fail(h, A2_EINVAL, "non-finite worker time");
+    for (int32_t w = 0; w < h->n; ++w) h->t[(size_t)w] = host_t[w];
+    return A2_OK;
+}
+
+int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, const int32_t* wi, const int32_t* wj,
+                        const int32_t* grad_slot, uint32_t flags, a2cid2_stats* stats) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    const double t0 = now_ms();
+    a2cid2_sched* s = nullptr;
+    std::string err;
+    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, &s, err);
+    if (rc != A2_OK) return fail(h, rc, err);
+    std::vector<LaunchRange> launches;
+    std::vector<int64_t> batch_first;
+    make_launches(*s, launches, batch_first);
+    const int64_t nb = (int64_t)s->batch_first.size() - 1;
+    const size_t bytes = desc_bytes(*s);
+    if (stats) std::memset(stats, 0, sizeof *stats);
+    if (bytes > 0) {
+        Arena& A = h->arena[h->arena_next];
+        h->arena_next ^= 1;
+        if (A.in_flight) {  // the previous copy out of this staging buffer must have finished
+            cudaError_t e = cudaEventSynchronize(A.copied);
+            if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "cudaEventSynchronize"); }
+            A.in_flight = false;
+        }
+        if (A.cap < bytes) {
+            // the device side may still be read by queued kernels: wait before freeing it
+            cudaError_t e = cudaStreamSynchronize(h->stream);
+            if (e == cudaSuccess && A.host) e = cudaFreeHost(A.host);
+            if (e == cudaSuccess && A.dev) e = cudaFree(A.dev);
+            A.host = A.dev = nullptr;
+            A.cap = 0;
+            const size_t cap = bytes + bytes / 2 + 4096;
+            if (e == cudaSuccess) e = cudaMallocHost(&A.host, cap);
+            if (e == cudaSuccess) e = cudaMalloc(&A.dev, cap);
+            if (e == cudaSuccess && !A.copied) e = cudaEventCreateWithFlags(&A.copied, cudaEventDisableTiming);
+            if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "descriptor buffer allocation"); }
+            A.cap = cap;
+        }
+        const size_t ops_off = pack_descriptors(*s, launches, A.host);
+        cudaError_t e = cudaMemcpyAsync(A.dev, A.host, bytes, cudaMemcpyHostToDevice, h->stream);
+        if (e == cudaSuccess) e = cudaEventRecord(A.copied, h->stream);
+        if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "descriptor upload"); }
+        A.in_flight = true;
+        const double t1 = now_ms();
+        rc = queue_launches(h, launches, 0, (int64_t)launches.size(), static_cast<const DevItem*>(A.dev),
+                            reinterpret_cast<const DevOp*>(static_cast<const char*>(A.dev) + ops_off));
+        if (rc != A2_OK) { a2cid2_sched_destroy(s); return rc; }
+        if (stats) {
+            a2::schedule_stats(*s, 0, nb, h->d, (int32_t)elem_bytes(h->dtype), stats);
+            stats->n_launches = (int64_t)launches.size();
+            stats->descriptor_bytes = (int64_t)bytes;
+            stats->host_ms = t1 - t0;
+        }
+    }
+    h->t = s->t_final;
+    a2cid2_sched_destroy(s);
+    return A2_OK;
+}
+
+int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!out) return fail(h, A2_EINVAL, "out is NULL");
+    const bool flush = !std::isnan(t_eval);
+    const int np = a2::consensus_grid(h->dev);
+    if (flush) {
+        if (!std::isfinite(t_eval)) return fail(h, A2_EINVAL, "t_eval must be finite or NaN");
+        for (int32_t w = 0; w < h->n; ++w)
+            if (t_eval < h->t[(size_t)w]) return fail(h, A2_EORDER, "t_eval precedes a worker's last event");
+        // the staging buffer is free: every earlier call waited for the stream before returning
+        for (int32_t w = 0; w < h->n; ++w) h->h_pinned[w] = t_eval - h->t[(size_t)w];
+        A2_CUDA(h, cudaMemcpyAsync(h->d_dt, h->h_pinned, sizeof(double) * (size_t)h->n, cudaMemcpyHostToDevice, h->stream));
+    }
+    const int lrc = a2::launch_consensus(h->x, h->xt, h->pitch, h->n, h->d, h->dtype, h->eta, flush ? h->d_dt : nullptr,
+                                         h->d_partials, np, h->d_partials + np, h->stream);
+    if (lrc != 0) return fail_cuda(h, (cudaError_t)lrc, "consensus kernel launch");
+    A2_CUDA(h, cudaMemcpyAsync(h->h_pinned + h->n, h->d_partials + np, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+    A2_CUDA(h, cudaStreamSynchronize(h->stream));
+    *out = h->h_pinned[h->n];
+    return A2_OK;
+}
+
+int a2cid2_sync(a2cid2_t* h) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (!h->dev_ok) return A2_OK;
+    A2_CUDA(h, cudaStreamSynchronize(h->stream));
+    return A2_OK;
+}
+
+void a2cid2_destroy(a2cid2_t* h) {
+    if (!h) return;
+    if (h->dev_ok) {
+        cudaStreamSynchronize(h->stream);
+        for (Arena& A : h->arena) {
+            if (A.host) cudaFreeHost(A.host);
+            if (A.dev) cudaFree(A.dev);
+            if (A.copied) cudaEventDestroy(A.copied);
+        }
+        if (h->d_partials) cudaFree(h->d_partials);
+        if (h->d_dt) cudaFree(h->d_dt);
+        if (h->h_pinned) cudaFreeHost(h->h_pinned);
+    }
+    delete h;
+}
+
+// ---- plans -----------------------------------------------------------------------------------
+
+int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, const double* times, const int32_t* wi,
+                       const int32_t* wj, const int32_t* grad_slot, uint32_t flags, a2cid2_plan_t** out) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!out) return fail(h, A2_EINVAL, "out is NULL");
+    *out = nullptr;
+    a2cid2_sched* s = nullptr;
+    std::string err;
+    rc = a2::build_schedule(h->n, h->n_slots, t_start ? t_start : h->t.data(), n_events, times, wi, wj, grad_slot, flags,
+                            0, &s, err);
+    if (rc != A2_OK) return fail(h, rc, err);
+    a2cid2_plan* p = new (std::nothrow) a2cid2_plan();
+    if (!p) { a2cid2_sched_destroy(s); return fail(h, A2_ENOMEM, "out of host memory"); }
+    p->owner = h;
+    p->sched = s;
+    p->t_expect = s->t_start;
+    p->uses_gradients = needs_gradients(*s);
+    make_launches(*s, p->launches, p->batch_launch_first);
+    const size_t bytes = desc_bytes(*s);
+    if (bytes > 0) {
+        std::vector<char> staging(bytes);
+        const size_t ops_off = pack_descriptors(*s, p->launches, staging.data());
+        cudaError_t e = cudaMalloc(&p->d_desc, bytes);
+        // pageable source: the copy has left the host buffer when the call returns
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_desc, staging.data(), bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            if (p->d_desc) cudaFree(p->d_desc);
+            a2cid2_sched_destroy(s);
+            delete p;
+            return fail_cuda(h, e, "plan descriptor upload");
+        }
+        p->d_items = static_cast<DevItem*>(p->d_desc);
+        p->d_ops = reinterpret_cast<DevOp*>(static_cast<char*>(p->d_desc) + ops_off);
+    }
+    h->live_plans += 1;
+    *out = p;
+    return A2_OK;
+}
+
+const a2cid2_sched_t* a2cid2_plan_sched(const a2cid2_plan_t* p) { return p ? p->sched : nullptr; }
+
+int a2cid2_plan_run(a2cid2_t* h, a2cid2_plan_t* p, int64_t first_batch, int64_t n_batches, a2cid2_stats* stats) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!p || p->owner != h) return fail(h, A2_EINVAL, "plan is NULL or belongs to another handle");
+    const int64_t nb = (int64_t)p->sched->batch_first.size() - 1;
+    if (n_batches < 0) n_batches = nb - first_batch;
+    if (first_batch != p->next_batch) return fail(h, A2_ESTATE, "plan batches must be run in order, each once");
+    if (first_batch < 0 || n_batches < 0 || first_batch + n_batches > nb) return fail(h, A2_ERANGE, "batch range out of bounds");
+    if (p->t_expect != h->t) return fail(h, A2_ESTATE, "the handle's worker times are not those the plan starts from");
+    if (p->uses_gradients && !h->g) return fail(h, A2_ESTATE, "plan has gradient events but no gradient buffer is bound");
+    const int64_t b1 = first_batch + n_batches;
+    if (n_batches > 0) {
+        rc = queue_launches(h, p->launches, p->batch_launch_first[(size_t)first_batch], p->batch_launch_first[(size_t)b1],
+                            p->d_items, p->d_ops);
+        if (rc != A2_OK) return rc;
+        advance_times(*p->sched, first_batch, b1, h->t);
+    }
+    p->next_batch = b1;
+    p->t_expect = h->t;
+    if (stats) {
+        a2::schedule_stats(*p->sched, first_batch, b1, h->d, (int32_t)elem_bytes(h->dtype), stats);
+        stats->n_launches = p->batch_launch_first[(size_t)b1] - p->batch_launch_first[(size_t)first_batch];
+        stats->descriptor_bytes = 0;
+        stats->host_ms = 0.0;
+    }
+    return A2_OK;
+}
+
+void a2cid2_plan_destroy(a2cid2_plan_t* p) {
+    if (!p) return;
+    if (p->owner) {
+        if (p->owner->dev_ok) cudaStreamSynchronize(p->owner->stream);  // queued kernels may still read the descriptors
+        p->owner->live_plans -= 1;
+    }
+    if (p->d_desc) cudaFree(p->d_desc);
+    a2cid2_sched_destroy(p->sched);
+    delete p;
+}
+
+// ---- host scheduler ----------------------------------------------------------------------------
+
+int a2cid2_sched_create(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
+                        const int32_t* wi, const int32_t* wj, const int32_t* grad_slot, uint32_t flags,
+                        int32_t max_ops_per_item, a2cid2_sched_t** out) {
+    std::string err;
+    const int rc = a2::build_schedule(n, n_grad_slots, t_last, n_events, times, wi, wj, grad_slot, flags, max_ops_per_item,
+                                      out, err);
+    if (rc != A2_OK) a2::set_thread_error(err);
+    return rc;
+}
+
+int64_t a2cid2_sched_num_batches(const a2cid2_sched_t* s) { return s ? (int64_t)s->batch_first.size() - 1 : 0; }
+int64_t a2cid2_sched_num_items(const a2cid2_sched_t* s) { return s ? (int64_t)s->items.size() : 0; }
+int64_t a2cid2_sched_num_ops(const a2cid2_sched_t* s) { return s ? (int64_t)s->ops.size() : 0; }
+
+int a2cid2_sched_batch_items(const a2cid2_sched_t* s, int64_t b, int64_t* first_item, int64_t* n_items) {
+    if (!s || !first_item || !n_items) return fail(nullptr, A2_EINVAL, "NULL argument");
+    if (b < 0 || b + 1 >= (int64_t)s->batch_first.size()) return fail(nullptr, A2_ERANGE, "batch out of range");
+    *first_item = s->batch_first[(size_t)b];
+    *n_items = s->batch_first[(size_t)b + 1] - s->batch_first[(size_t)b];
+    return A2_OK;
+}
+
+int a2cid2_sched_item(const a2cid2_sched_t* s, int64_t item, a2cid2_item_info* out) {
+    if (!s || !out) return fail(nullptr, A2_EINVAL, "NULL argument");
+    if (item < 0 || item >= (int64_t)s->items.size()) return fail(nullptr, A2_ERANGE, "item out of range");
+    const a2::SchedItem& it = s->items[(size_t)item];
+    *out = a2cid2_item_info{it.a, it.b, it.slot_a, it.slot_b, it.first_op, it.n_ops, it.batch};
+    return A2_OK;
+}
+
+int a2cid2_sched_ops(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, int64_t* event_index, int32_t* kind) {
+    if (!s) return fail(nullptr, A2_EINVAL, "NULL argument");
+    if (first_op < 0 || n_ops < 0 || first_op + n_ops > (int64_t)s->ops.size()) return fail(nullptr, A2_ERANGE, "op range out of bounds");
+    for (int64_t k = 0; k < n_ops; ++k) {
+        if (event_index) event_index[k] = s->ops[(size_t)(first_op + k)].event;
+        if (kind) kind[k] = s->ops[(size_t)(first_op + k)].kind;
+    }
+    return A2_OK;
+}
+
+int a2cid2_sched_t_final(const a2cid2_sched_t* s, double* t_out) {
+    if (!s || !t_out) return fail(nullptr, A2_EINVAL, "NULL argument");
+    std::memcpy(t_out, s->t_final.data(), sizeof(double) * (size_t)s->n);
+    return A2_OK;
+}
+
+int a2cid2_sched_stats(const a2cid2_sched_t* s, int64_t first_batch, int64_t n_batches, int64_t d, int32_t elem_bytes_,
+                       a2cid2_stats* out) {
+    if (!s || !out) return fail(nullptr, A2_EINVAL, "NULL argument");
+    const int64_t nb = (int64_t)s->batch_first.size() - 1;
+    if (n_batches < 0) n_batches = nb - first_batch;
+    if (first_batch < 0 || n_batches < 0 || first_batch + n_batches > nb || d < 0 || elem_bytes_ <= 0)
+        return fail(nullptr, A2_ERANGE, "batch range out of bounds");
+    a2::schedule_stats(*s, first_batch, first_batch + n_batches, d, elem_bytes_, out);
+    std::vector<LaunchRange> launches;
+    std::vector<int64_t> bf;
+    make_launches(*s, launches, bf);
+    out->n_launches = bf[(size_t)(first_batch + n_batches)] - bf[(size_t)first_batch];
+    return A2_OK;
+}
+
+void a2cid2_sched_destroy(a2cid2_sched_t* s) { delete s; }
+
+// ---- graph quantities ----------------------------------------------------------------------------
+
+int a2cid2_graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda, double* chi1,
+                     double* chi2) {
+    std::string err;
+    const int rc = a2::graph_chi(n, n_edges, ei, ej, lambda, chi1, chi2, err);
+    if (rc != A2_OK) a2::set_thread_error(err);
+    return rc;
+}
+
+int a2cid2_prescribe(double chi1, double chi2, int32_t accelerated, double* eta, double* alpha, double* alpha_tilde) {
+    if (!eta || !alpha || !alpha_tilde) return fail(nullptr, A2_EINVAL, "NULL output");
+    if (!accelerated) {
+        *eta = 0.0; *alpha = 0.5; *alpha_tilde = 0.5;
+        return A2_OK;
+    }
+    if (!(chi1 > 0) || !(chi2 > 0) || !std::isfinite(chi1) || !std::isfinite(chi2))
+        return fail(nullptr, A2_EINVAL, "chi_1 and chi_2 must be positive and finite");
+    *eta = 1.0 / (2.0 * std::sqrt(chi1 * chi2));
+    *alpha = 0.5;
+    *alpha_tilde = 0.5 * std::sqrt(chi1 / chi2);
+    return A2_OK;
+}
+
+}  // extern "C"

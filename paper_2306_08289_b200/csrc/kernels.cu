@@ -1,0 +1,375 @@
+// Device kernels for sm_100a.
+//
+//   event kernel      one launch per batch of worker-disjoint items. A work unit is (item, column
+//                     tile); a persistent grid strides over the units. For a unit the item's rows
+//                     (x_a, x~_a, x_b, x~_b and the gradient rows it needs) are read once with
+//                     128-bit loads, the item's operations are applied in registers in event
+//                     order, and the state rows are written once. Purely HBM-bound streaming work.
+//   consensus kernel  per column: sum_i (x_i - xbar)^2 from shifted sums, fp64 across columns,
+//                     warp shuffle + block reduce, per-block partials, fixed-order final sum.
+//
+// Per-element arithmetic (fp32, explicit FMAs, identical for fused and unfused schedules):
+//   mixing    dlt = x - x~;  x = fma(-c, dlt, x);  x~ = fma(c, dlt, x~)        (Algorithm 1, matrix exponential)
+//   gradient  x = fma(-gamma, g, x);  x~ = fma(-gamma, g, x~)                  (Eq. (dynamic), dN term)
+//   comm      m = x_a - x_b;  x_a = fma(-alpha, m, x_a);  x~_a = fma(-alpha~, m, x~_a);
+//             x_b = fma(alpha, m, x_b);  x~_b = fma(alpha~, m, x~_b)           (Eq. (dynamic), dM term)
+// The mixing coefficient c = -expm1(-2 eta (t - t_prev)) / 2 is evaluated in fp64 on the device
+// from the event time and the worker's previous time carried by the descriptor, then rounded
+// once to fp32.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "a2cid2_internal.h"
+
+namespace a2 {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------------------------------------
+// 128-bit vector access for the two storage types. Vec<T>::N elements per 16 bytes.
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Vec;
+
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
+        const float4 q = __ldcs(reinterpret_cast<const float4*>(p));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+    }
+    static __device__ __forceinline__ void store(float* p, const float (&v)[4]) {
+        __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
+    }
+};
+
+template <> struct Vec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
+        const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {  // bf16 -> fp32 is a 16-bit shift
+            v[2 * k] = __uint_as_float(w[k] << 16);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {  // round to nearest even
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+            w[k] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+};
+
+__device__ __forceinline__ void mix_elem(float& x, float& xt, float c) {
+    const float dlt = __fsub_rn(x, xt);
+    x = __fmaf_rn(-c, dlt, x);
+    xt = __fmaf_rn(c, dlt, xt);
+}
+
+__device__ __forceinline__ double mix_coeff(double eta, double dt) { return -0.5 * expm1(-2.0 * eta * dt); }
+
+// ---------------------------------------------------------------------------------------------
+// Event kernel
+// ---------------------------------------------------------------------------------------------
+struct EventArgs {
+    void* x;
+    void* xt;
+    const void* g;
+    long long pitch;
+    long long n_vec;  // vectors per row that hold at least one real column
+    const DevItem* items;
+    const DevOp* ops;
+    int n_items;
+    int n_ops;
+    int n_tiles;
+    double eta;
+    float alpha, alpha_tilde, gamma;
+    int msg_before_mix;
+};
+
+template <typename T, int UNROLL>
+__global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
+    constexpr int N = Vec<T>::N;
+    __shared__ DevItem s_items[kMaxItemsPerLaunch];
+    __shared__ float s_ca[kMaxOpsPerLaunch];
+    __shared__ float s_cb[kMaxOpsPerLaunch];
+    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+
+    for (int i = threadIdx.x; i < p.n_items; i += kThreads) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += kThreads) {
+        const DevOp op = p.ops[o];
+        s_kind[o] = (unsigned char)op.kind;
+        s_ca[o] = (op.kind != A2_OP_GRAD_B) ? (float)mix_coeff(p.eta, op.t - op.t_prev_a) : 0.f;
+        s_cb[o] = (op.kind != A2_OP_GRAD_A) ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
+    }
+    __syncthreads();
+
+    T* const X = static_cast<T*>(p.x);
+    T* const Xt = static_cast<T*>(p.xt);
+    const T* const G = static_cast<const T*>(p.g);
+    const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
+    const long long n_units = (long long)p.n_items * p.n_tiles;
+
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int item_idx = (int)(unit % p.n_items);
+        const long long tile = unit / p.n_items;
+        const DevItem it = s_items[item_idx];
+        const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const long long v0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
+
+        T* const pxa = X + (long long)it.a * p.pitch;
+        T* const pxta = Xt + (long long)it.a * p.pitch;
+        T* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
+        T* const pxtb = Xt + (long long)(has_b ? it.b : it.a) * p.pitch;
+        const T* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
+        const T* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+
+        float xa[UNROLL][N], xta[UNROLL][N], xb[UNROLL][N], xtb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N];
+        bool live[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long v = v0 + (long long)u * kThreads;
+            live[u] = v < p.n_vec;
+            const long long off = v * N;
+#pragma unroll
+            for (int k = 0; k < N; ++k) { xb[u][k] = 0.f; xtb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
+            if (live[u]) {
+                Vec<T>::load(pxa + off, xa[u]);
+                Vec<T>::load(pxta + off, xta[u]);
+                if (has_b) {
+                    Vec<T>::load(pxb + off, xb[u]);
+                    Vec<T>::load(pxtb + off, xtb[u]);
+                }
+                if (has_ga) Vec<T>::load(pga + off, ga[u]);
+                if (has_gb) Vec<T>::load(pgb + off, gb[u]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xta[u][k] = 0.f; }
+            }
+        }
+
+        for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
+            const int kind = s_kind[o];
+            if (kind == A2_OP_GRAD_A) {
+                const float c = s_ca[o];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                    for (int k = 0; k < N; ++k) {
+                        mix_elem(xa[u][k], xta[u][k], c);
+                        xa[u][k] = __fmaf_rn(ngamma, ga[u][k], xa[u][k]);
+                        xta[u][k] = __fmaf_rn(ngamma, ga[u][k], xta[u][k]);
+                    }
+            } else if (kind == A2_OP_GRAD_B) {
+                const float c = s_cb[o];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                    for (int k = 0; k < N; ++k) {
+                        mix_elem(xb[u][k], xtb[u][k], c);
+                        xb[u][k] = __fmaf_rn(ngamma, gb[u][k], xb[u][k]);
+                        xtb[u][k] = __fmaf_rn(ngamma, gb[u][k], xtb[u][k]);
+                    }
+            } else {
+                const float ca = s_ca[o], cb = s_cb[o];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                    for (int k = 0; k < N; ++k) {
+                        float m;
+                        if (p.msg_before_mix) {
+                            m = __fsub_rn(xa[u][k], xb[u][k]);
+                            mix_elem(xa[u][k], xta[u][k], ca);
+                            mix_elem(xb[u][k], xtb[u][k], cb);
+                        } else {
+                            mix_elem(xa[u][k], xta[u][k], ca);
+                            mix_elem(xb[u][k], xtb[u][k], cb);
+                            m = __fsub_rn(xa[u][k], xb[u][k]);
+                        }
+                        xa[u][k] = __fmaf_rn(-alpha, m, xa[u][k]);
+                        xta[u][k] = __fmaf_rn(-alpha_t, m, xta[u][k]);
+                        xb[u][k] = __fmaf_rn(alpha, m, xb[u][k]);
+                        xtb[u][k] = __fmaf_rn(alpha_t, m, xtb[u][k]);
+                    }
+            }
+        }
+
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long off = (v0 + (long long)u * kThreads) * N;
+            if (live[u]) {
+                Vec<T>::store(pxa + off, xa[u]);
+                Vec<T>::store(pxta + off, xta[u]);
+                if (has_b) {
+                    Vec<T>::store(pxb + off, xb[u]);
+                    Vec<T>::store(pxtb + off, xtb[u]);
+                }
+            }
+        }
+    }
+}
+
+template <typename T> struct EventCfg;
+template <> struct EventCfg<float> { static constexpr int UNROLL = 2; };
+template <> struct EventCfg<__nv_bfloat16> { static constexpr int UNROLL = 1; };
+
+// ---------------------------------------------------------------------------------------------
+// Consensus kernel
+// ---------------------------------------------------------------------------------------------
+template <typename T, bool FLUSH>
+__global__ void __launch_bounds__(kThreads) k_consensus_partial(const T* __restrict__ X, const T* __restrict__ Xt,
+                                                              long long pitch, int n, long long d, double eta,
+                                                              const double* __restrict__ dt, double* __restrict__ partials) {
+    constexpr int N = Vec<T>::N;
+    extern __shared__ float s_c[];  // FLUSH: mixing coefficient of every worker to the common time
+    __shared__ double s_warp[kThreads / 32];
+    if (FLUSH) {
+        for (int i = threadIdx.x; i < n; i += kThreads) s_c[i] = (float)mix_coeff(eta, dt[i]);
+        __syncthreads();
+    }
+    const long long n_vec = (d + N - 1) / N;
+    const double inv_n = 1.0 / (double)n;
+    double acc = 0.0;
+    for (long long v = (long long)blockIdx.x * kThreads + threadIdx.x; v < n_vec; v += (long long)gridDim.x * kThreads) {
+        const long long off = v * N;
+        float first[N], s1[N], s2[N];
+        Vec<T>::load(X + off, first);
+        if (FLUSH) {
+            float xt0[N];
+            Vec<T>::load(Xt + off, xt0);
+            const float c = s_c[0];
+#pragma unroll
+            for (int k = 0; k < N; ++k) first[k] = __fmaf_rn(-c, __fsub_rn(first[k], xt0[k]), first[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < N; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
+#pragma unroll 4
+        for (int i = 1; i < n; ++i) {
+            float xi[N];
+            Vec<T>::load(X + (long long)i * pitch + off, xi);
+            if (FLUSH) {
+                float xti[N];
+                Vec<T>::load(Xt + (long long)i * pitch + off, xti);
+                const float c = s_c[i];
+#pragma unroll
+                for (int k = 0; k < N; ++k) xi[k] = __fmaf_rn(-c, __fsub_rn(xi[k], xti[k]), xi[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+                const float s = __fsub_rn(xi[k], first[k]);  // shifted by the first row: no large cancellation later
+                s1[k] += s;
+                s2[k] = __fmaf_rn(s, s, s2[k]);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < N; ++k) {
+            if (off + k < d) acc += (double)s2[k] - (double)s1[k] * (double)s1[k] * inv_n;
+        }
+    }
+    // warp shuffle, then block reduce
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, s);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tot = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) tot += s_warp[w];
+        partials[blockIdx.x] = tot;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __restrict__ partials, int n_partials,
+                                                            double* __restrict__ out) {
+    __shared__ double s_warp[kThreads / 32];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n_partials; i += kThreads) acc += partials[i];
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, s);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tot = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) tot += s_warp[w];
+        out[0] = tot;
+    }
+}
+
+template <typename T>
+int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
+    constexpr int U = EventCfg<T>::UNROLL;
+    constexpr int N = Vec<T>::N;
+    EventArgs a;
+    a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
+    a.n_vec = (L.d + N - 1) / N;
+    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
+    const long long vec_per_tile = (long long)kThreads * U;
+    a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
+    a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
+    a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
+    const long long n_units = (long long)a.n_items * a.n_tiles;
+    const int per_sm = dev.event_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0];
+    long long grid = (long long)dev.sm_count * per_sm;
+    if (grid > n_units) grid = n_units;
+    if (grid < 1) return 0;
+    k_apply_events<T, U><<<(unsigned)grid, kThreads, 0, stream>>>(a);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace
+
+int query_device(DeviceInfo* info) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    e = cudaDeviceGetAttribute(&info->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return (int)e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events<float, EventCfg<float>::UNROLL>, kThreads, 0);
+    if (e != cudaSuccess) return (int)e;
+    info->event_ctas_per_sm[0] = occ > 0 ? occ : 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &occ, k_apply_events<__nv_bfloat16, EventCfg<__nv_bfloat16>::UNROLL>, kThreads, 0);
+    if (e != cudaSuccess) return (int)e;
+    info->event_ctas_per_sm[1] = occ > 0 ? occ : 1;
+    info->consensus_ctas_per_sm = 4;
+    return 0;
+}
+
+int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream) {
+    if (L.n_items <= 0) return 0;
+    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16>(L, dev, static_cast<cudaStream_t>(stream));
+    return launch_events_t<float>(L, dev, static_cast<cudaStream_t>(stream));
+}
+
+int consensus_grid(const DeviceInfo& dev) { return dev.sm_count * dev.consensus_ctas_per_sm; }
+
+int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double eta,
+                     const double* dt, double* partials, int n_partials, double* out, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t smem = dt ? (size_t)n * sizeof(float) : 0;
+    if (dtype == A2_BF16) {
+        const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(x);
+        const __nv_bfloat16* Xt = static_cast<const __nv_bfloat16*>(xt);
+        if (dt) k_consensus_partial<__nv_bfloat16, true><<<n_partials, kThreads, smem, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+        else k_consensus_partial<__nv_bfloat16, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+    } else {
+        const float* X = static_cast<const float*>(x);
+        const float* Xt = static_cast<const float*>(xt);
+        if (dt) k_consensus_partial<float, true><<<n_partials, kThreads, smem, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+        else k_consensus_partial<float, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+    k_consensus_final<<<1, kThreads, 0, stream>>>(partials, n_partials, out);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace a2

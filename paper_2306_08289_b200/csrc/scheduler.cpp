@@ -1,0 +1,212 @@
+// Host scheduler: validates a time-sorted event stream and packs it into batches of
+// worker-disjoint items that keep every worker's own event order.
+//
+// Why batches are legal: in Eq. (dynamic) (Sec. 3.2) an event changes only the rows of the
+// workers it names, and needs only those rows and their last-event times. Two events on
+// disjoint workers therefore commute exactly, and any order that keeps each worker's own
+// sequence yields the state of the time-ordered run.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <new>
+
+#include "a2cid2_internal.h"
+
+namespace a2 {
+
+namespace {
+
+struct Pending {
+    std::vector<int64_t> events;  // gradient events held back for this worker, in order
+    int32_t slot = -1;
+};
+
+std::string fmt_event(const char* what, int64_t e) {
+    char buf[160];
+    std::snprintf(buf, sizeof buf, "event %lld: %s", (long long)e, what);
+    return buf;
+}
+
+}  // namespace
+
+int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
+                   const int32_t* wi, const int32_t* wj, const int32_t* slot, uint32_t flags,
+                   int32_t max_ops_per_item, a2cid2_sched** out, std::string& err) {
+    if (!out) { err = "out is NULL"; return A2_EINVAL; }
+    *out = nullptr;
+    if (n < 2) { err = "need n >= 2 workers"; return A2_EINVAL; }
+    if (n_grad_slots < 0 || n_events < 0) { err = "negative size"; return A2_EINVAL; }
+    if (n_events > 0 && (!times || !wi || !wj || !slot)) { err = "event arrays are NULL"; return A2_EINVAL; }
+    if (flags & ~uint32_t(A2_SCHED_FUSE)) { err = "unknown scheduling flag"; return A2_EINVAL; }
+    if (max_ops_per_item <= 0) max_ops_per_item = kDefaultMaxOpsPerItem;
+    if (max_ops_per_item > kMaxOpsPerLaunch) max_ops_per_item = kMaxOpsPerLaunch;
+    const bool fuse = (flags & A2_SCHED_FUSE) != 0 && max_ops_per_item >= 2;
+
+    a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
+    if (!s) { err = "out of host memory"; return A2_ENOMEM; }
+    try {
+        s->n = n;
+        s->n_grad_slots = n_grad_slots;
+        s->flags = flags;
+        s->n_events = n_events;
+        s->t_start.assign((size_t)n, 0.0);
+        if (t_last) {
+            for (int32_t w = 0; w < n; ++w) {
+                if (!std::isfinite(t_last[w])) { err = "non-finite worker time"; delete s; return A2_EINVAL; }
+                s->t_start[(size_t)w] = t_last[w];
+            }
+        }
+
+        // ---- pass 1: validation only (nothing is built from a bad stream) ------------------
+        {
+            std::vector<double> tcur(s->t_start);
+            double prev = -INFINITY;
+            for (int64_t e = 0; e < n_events; ++e) {
+                const double t = times[e];
+                const int32_t i = wi[e], j = wj[e], sl = slot[e];
+                if (!std::isfinite(t)) { err = fmt_event("time is not finite", e); delete s; return A2_EINVAL; }
+                if (t < prev) { err = fmt_event("times decrease", e); delete s; return A2_EORDER; }
+                prev = t;
+                if (i < 0 || i >= n) { err = fmt_event("worker index out of range", e); delete s; return A2_ERANGE; }
+                if (j == -1) {
+                    if (sl < 0 || sl >= n_grad_slots) { err = fmt_event("gradient slot out of range", e); delete s; return A2_ERANGE; }
+                    if (t < tcur[(size_t)i]) { err = fmt_event("precedes the worker's last event", e); delete s; return A2_EORDER; }
+                    tcur[(size_t)i] = t;
+                } else {
+                    if (j < 0 || j >= n || j == i) { err = fmt_event("bad pair", e); delete s; return A2_ERANGE; }
+                    if (sl != -1) { err = fmt_event("communication event with a gradient slot", e); delete s; return A2_ERANGE; }
+                    if (t < tcur[(size_t)i] || t < tcur[(size_t)j]) { err = fmt_event("precedes a worker's last event", e); delete s; return A2_EORDER; }
+                    tcur[(size_t)i] = t;
+                    tcur[(size_t)j] = t;
+                }
+            }
+        }
+
+        // ---- pass 2: greedy level assignment ------------------------------------------------
+        std::vector<SchedItem> items;  // creation order
+        std::vector<SchedOp> ops;      // creation order
+        items.reserve((size_t)n_events);
+        ops.reserve((size_t)n_events);
+        std::vector<int32_t> level((size_t)n, 0);  // first batch in which the worker is free
+        std::vector<double> tcur(s->t_start);
+        std::vector<Pending> pend(fuse ? (size_t)n : 0);
+
+        auto push_grad_ops = [&](int32_t w, int32_t kind, const std::vector<int64_t>& evs) {
+            for (int64_t e : evs) {
+                SchedOp op{e, kind, times[e], 0.0, 0.0};
+                if (kind == A2_OP_GRAD_A) op.t_prev_a = tcur[(size_t)w]; else op.t_prev_b = tcur[(size_t)w];
+                tcur[(size_t)w] = times[e];
+                ops.push_back(op);
+            }
+        };
+        auto flush = [&](int32_t w) {  // gradient-only item for the worker's held-back events
+            Pending& p = pend[(size_t)w];
+            if (p.events.empty()) return;
+            SchedItem it{w, -1, p.slot, -1, (int64_t)ops.size(), (int32_t)p.events.size(), level[(size_t)w]};
+            push_grad_ops(w, A2_OP_GRAD_A, p.events);
+            items.push_back(it);
+            level[(size_t)w] += 1;
+            p.events.clear();
+            p.slot = -1;
+        };
+
+        for (int64_t e = 0; e < n_events; ++e) {
+            const int32_t i = wi[e], j = wj[e];
+            if (j == -1) {
+                if (fuse) {
+                    Pending& p = pend[(size_t)i];
+                    if (!p.events.empty() && (p.slot != slot[e] || (int32_t)p.events.size() >= max_ops_per_item - 1)) flush(i);
+                    p.slot = slot[e];
+                    p.events.push_back(e);
+                } else {
+                    SchedItem it{i, -1, slot[e], -1, (int64_t)ops.size(), 1, level[(size_t)i]};
+                    ops.push_back(SchedOp{e, A2_OP_GRAD_A, times[e], tcur[(size_t)i], 0.0});
+                    tcur[(size_t)i] = times[e];
+                    items.push_back(it);
+                    level[(size_t)i] += 1;
+                }
+            } else {
+                int32_t slot_a = -1, slot_b = -1;
+                if (fuse) {
+                    Pending& pi = pend[(size_t)i];
+                    Pending& pj = pend[(size_t)j];
+                    if ((int64_t)pi.events.size() + (int64_t)pj.events.size() + 1 > max_ops_per_item) {
+                        // too long for one item: spill the longer side first
+                        if (pi.events.size() >= pj.events.size()) flush(i); else flush(j);
+                        if ((int64_t)pi.events.size() + (int64_t)pj.events.size() + 1 > max_ops_per_item) {
+                            flush(i);
+                            flush(j);
+                        }
+                    }
+                    slot_a = pi.events.empty() ? -1 : pi.slot;
+                    slot_b = pj.events.empty() ? -1 : pj.slot;
+                }
+                const int32_t lv = std::max(level[(size_t)i], level[(size_t)j]);
+                SchedItem it{i, j, slot_a, slot_b, (int64_t)ops.size(), 0, lv};
+                if (fuse) {
+                    Pending& pi = pend[(size_t)i];
+                    Pending& pj = pend[(size_t)j];
+                    push_grad_ops(i, A2_OP_GRAD_A, pi.events);
+                    push_grad_ops(j, A2_OP_GRAD_B, pj.events);
+                    pi.events.clear(); pi.slot = -1;
+                    pj.events.clear(); pj.slot = -1;
+                }
+                ops.push_back(SchedOp{e, A2_OP_COMM, times[e], tcur[(size_t)i], tcur[(size_t)j]});
+                tcur[(size_t)i] = times[e];
+                tcur[(size_t)j] = times[e];
+                it.n_ops = (int32_t)((int64_t)ops.size() - it.first_op);
+                items.push_back(it);
+                level[(size_t)i] = lv + 1;
+                level[(size_t)j] = lv + 1;
+            }
+        }
+        if (fuse) for (int32_t w = 0; w < n; ++w) flush(w);
+
+        // ---- order items by batch (stable) and lay the ops out in item order ----------------
+        int32_t n_batches = 0;
+        for (const SchedItem& it : items) n_batches = std::max(n_batches, it.batch + 1);
+        s->batch_first.assign((size_t)n_batches + 1, 0);
+        for (const SchedItem& it : items) s->batch_first[(size_t)it.batch + 1] += 1;
+        for (int32_t b = 0; b < n_batches; ++b) s->batch_first[(size_t)b + 1] += s->batch_first[(size_t)b];
+        std::vector<int64_t> cursor(s->batch_first.begin(), s->batch_first.end() - 1);
+        s->items.resize(items.size());
+        for (const SchedItem& it : items) s->items[(size_t)cursor[(size_t)it.batch]++] = it;
+        s->ops.reserve(ops.size());
+        for (SchedItem& it : s->items) {
+            const int64_t src = it.first_op;
+            it.first_op = (int64_t)s->ops.size();
+            for (int32_t k = 0; k < it.n_ops; ++k) s->ops.push_back(ops[(size_t)(src + k)]);
+        }
+        s->t_final = tcur;
+    } catch (const std::bad_alloc&) {
+        delete s;
+        err = "out of host memory";
+        return A2_ENOMEM;
+    }
+    *out = s;
+    return A2_OK;
+}
+
+void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {
+    a2cid2_stats st{};
+    const int64_t i0 = s.batch_first[(size_t)b0], i1 = s.batch_first[(size_t)b1];
+    int64_t rows_moved = 0, rows_single = 0;
+    for (int64_t k = i0; k < i1; ++k) {
+        const SchedItem& it = s.items[(size_t)k];
+        const int64_t state_rows = it.b >= 0 ? 4 : 2;
+        rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0);
+        for (int32_t o = 0; o < it.n_ops; ++o) {
+            const int32_t kind = s.ops[(size_t)(it.first_op + o)].kind;
+            if (kind == A2_OP_COMM) { st.n_comm += 1; rows_single += 8; }
+            else { st.n_grad += 1; rows_single += 5; }
+        }
+    }
+    st.n_events = st.n_comm + st.n_grad;
+    st.n_batches = b1 - b0;
+    st.n_items = i1 - i0;
+    st.bytes_moved = rows_moved * d * elem_bytes;
+    st.bytes_one_by_one = rows_single * d * elem_bytes;
+    *out = st;
+}
+
+}  // namespace a2
