@@ -1,0 +1,91 @@
+"""The C-ABI library loads without a GPU, exports everything include/a2cid2.h declares, and its
+host-only entry points (graph quantities, parameter prescription, validation) behave."""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import spectral
+from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import build as build_mod
+from paper_2306_08289_b200 import workload as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "a2cid2.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(a2cid2_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported_and_bound():
+    names = _declared()
+    assert len(names) >= 25 and "a2cid2_apply_events" in names and "a2cid2_consensus_distance" in names
+    raw = C.CDLL(B.LIB_PATH)
+    for nm in names:
+        assert hasattr(raw, nm), nm
+    assert set(names) == set(B.SIGNATURES), set(names) ^ set(B.SIGNATURES)
+    assert B.lib().a2cid2_version().startswith(b"a2cid2")
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_graph_quantities_agree_with_checker(name):
+    c = W.CONFIGS[name]
+    c1, c2 = B.graph_chi(c.n, c.edges(), c.rates())
+    eta, alpha, at, o1, o2 = spectral.prescribe(c.n, c.edges(), c.rates())
+    assert abs(c1 - o1) < 1e-10 * o1 and abs(c2 - o2) < 1e-10 * o2
+    e2, a2, at2 = B.prescribe(c1, c2)
+    assert abs(e2 - eta) < 1e-10 * eta and a2 == alpha and abs(at2 - at) < 1e-10 * at
+    assert B.prescribe(c1, c2, accelerated=False) == (0.0, 0.5, 0.5)
+
+
+def test_graph_quantities_irregular_graph_and_errors():
+    # a path with unequal rates: not regular, checks the general code path
+    edges = np.array([[0, 1], [1, 2], [2, 3], [1, 3]], dtype=np.int32)
+    lam = np.array([0.5, 2.0, 1.0, 0.25])
+    c1, c2 = B.graph_chi(4, edges, lam)
+    L = spectral.laplacian(4, edges, lam)
+    assert abs(c1 - spectral.chi1(L)) < 1e-12 and abs(c2 - spectral.chi2(L, edges)) < 1e-12
+    with pytest.raises(B.A2Error) as e:
+        B.graph_chi(4, np.array([[0, 1], [2, 3]], dtype=np.int32), np.ones(2))  # disconnected
+    assert e.value.code == B.A2_EINVAL
+    with pytest.raises(B.A2Error) as e:
+        B.graph_chi(4, np.array([[0, 4]], dtype=np.int32), np.ones(1))
+    assert e.value.code == B.A2_ERANGE
+    with pytest.raises(B.A2Error):
+        B.graph_chi(4, edges, -lam)
+
+
+def test_create_validates_without_a_device():
+    L = B.lib()
+    h = C.c_void_p()
+    assert L.a2cid2_create(1, 10, 0.1, 0.5, 0.5, 0.1, B.A2_F32, C.byref(h)) == B.A2_EINVAL
+    assert L.a2cid2_create(4, 0, 0.1, 0.5, 0.5, 0.1, B.A2_F32, C.byref(h)) == B.A2_EINVAL
+    assert L.a2cid2_create(4, 10, -0.1, 0.5, 0.5, 0.1, B.A2_F32, C.byref(h)) == B.A2_EINVAL
+    assert L.a2cid2_create(4, 10, math.nan, 0.5, 0.5, 0.1, B.A2_F32, C.byref(h)) == B.A2_EINVAL
+    assert L.a2cid2_create(4, 10, 0.1, 0.5, 0.5, 0.1, 7, C.byref(h)) == B.A2_EINVAL
+    assert b"storage" in L.a2cid2_last_error(None)
+    assert L.a2cid2_create(4, 10, 0.1, 0.5, 0.5, 0.1, B.A2_BF16, C.byref(h)) == B.A2_OK and h.value
+    # nothing is bound: every device call refuses instead of touching memory
+    out = C.c_double()
+    assert L.a2cid2_consensus_distance(h, math.nan, C.byref(out)) == B.A2_ESTATE
+    t = np.zeros(1)
+    i = np.zeros(1, dtype=np.int32)
+    assert L.a2cid2_apply_events(h, 0, None, None, None, None, 0, None) == B.A2_ESTATE
+    assert b"bind" in L.a2cid2_last_error(h)
+    tt = np.array([1.0, 2.0, 3.0, 4.0])
+    assert L.a2cid2_set_times(h, tt.ctypes.data_as(C.POINTER(C.c_double))) == B.A2_OK
+    back = np.zeros(4)
+    assert L.a2cid2_times(h, back.ctypes.data_as(C.POINTER(C.c_double))) == B.A2_OK and np.array_equal(back, tt)
+    assert L.a2cid2_sync(h) == B.A2_OK
+    L.a2cid2_destroy(h)
+    L.a2cid2_destroy(None)

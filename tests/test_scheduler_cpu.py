@@ -1,0 +1,154 @@
+"""The host scheduler, without a GPU: its batches replayed through the CPU checker must give
+the time-ordered run bit for bit (events on disjoint workers commute: Eq. (dynamic) is local
+to the workers an event names), with and without gradient fusion; plus validation."""
+import numpy as np
+import pytest
+
+from oracle.sim import OracleSim
+from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import build as build_mod
+from paper_2306_08289_b200 import workload as W
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+
+
+def _replay(cfg, ev, sched, params, x0, G):
+    """Advance the checker batch by batch, events sorted by time inside a batch."""
+    sim = OracleSim(x0, *params, cfg.gamma, grads=G)
+    seen = []
+    for b in range(sched.num_batches):
+        idx = sched.batch_events(b)
+        seen.append(idx)
+        idx = idx[np.argsort(ev.times[idx], kind="stable")]
+        sim.apply(ev.times[idx], ev.wi[idx], ev.wj[idx], ev.slot[idx])
+    return sim, np.concatenate(seen) if seen else np.empty(0, dtype=np.int64)
+
+
+@pytest.mark.parametrize("name,d,n_events", [("cfg1", 7, 2000), ("cfg2", 5, 3000), ("cfg4", 3, 4000), ("cfg5", 3, 4000)])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
+    cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
+    cfg = cfg if cfg.storage == "f32" else W.WorkloadConfig(**{**cfg.__dict__, "storage": "f32"})
+    ev = W.config_events(cfg)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    params = (0.4, 0.5, 1.3)
+    ref = OracleSim(x0, *params, cfg.gamma, grads=G)
+    ref.apply_stream(ev)
+    s = B.Schedule(cfg.n, cfg.n, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+    sim, seen = _replay(cfg, ev, s, params, x0, G)
+    assert np.array_equal(np.sort(seen), np.arange(len(ev)))  # every event exactly once
+    assert np.array_equal(sim.X, ref.X) and np.array_equal(sim.Xt, ref.Xt) and np.array_equal(sim.t, ref.t)
+    assert np.array_equal(s.t_final(cfg.n), ref.t)
+    # structure: items of a batch are worker-disjoint; per-worker event order is kept
+    last_pos = {}
+    pos = 0
+    for b in range(s.num_batches):
+        first, cnt = s.batch_items(b)
+        used = set()
+        for k in range(first, first + cnt):
+            it = s.item(k)
+            assert it.batch == b and it.n_ops >= 1
+            ws = {it.a} | ({it.b} if it.b >= 0 else set())
+            assert not (ws & used)
+            used |= ws
+            evs, kinds = s.ops(it.first_op, it.n_ops)
+            for e, kd in zip(evs, kinds):
+                if kd == B.A2_OP_COMM:
+                    assert (ev.wi[e], ev.wj[e]) == (it.a, it.b)
+                    touched = (it.a, it.b)
+                elif kd == B.A2_OP_GRAD_A:
+                    assert ev.wi[e] == it.a and ev.wj[e] == -1 and ev.slot[e] == it.slot_a
+                    touched = (it.a,)
+                else:
+                    assert ev.wi[e] == it.b and ev.wj[e] == -1 and ev.slot[e] == it.slot_b
+                    touched = (it.b,)
+                for w in touched:
+                    assert last_pos.get(w, -1) < e  # this worker's events come in stream order
+                    last_pos[w] = e
+                pos += 1
+            if not flags:
+                assert it.n_ops == 1
+    assert pos == len(ev)
+    st = s.stats(cfg.d, 4)
+    assert st["n_events"] == len(ev) and st["n_comm"] == int((ev.wj >= 0).sum())
+    assert st["bytes_one_by_one"] == (8 * st["n_comm"] + 5 * st["n_grad"]) * cfg.d * 4
+    if flags:
+        assert st["bytes_moved"] < st["bytes_one_by_one"] and s.num_items < len(ev)
+    else:
+        assert st["bytes_moved"] == st["bytes_one_by_one"] and s.num_items == len(ev)
+
+
+def test_greedy_levels_are_as_early_as_possible():
+    # 0-1 and 2-3 are independent; 1-2 must wait for both; a gradient on 0 fits beside it
+    times = [1.0, 2.0, 3.0, 4.0]
+    s = B.Schedule(4, 4, times, [0, 2, 1, 0], [1, 3, 2, -1], [-1, -1, -1, 0])
+    assert s.num_batches == 2
+    assert sorted(s.batch_events(0)) == [0, 1] and sorted(s.batch_events(1)) == [2, 3]
+
+
+def test_fusion_folds_pending_gradients_and_respects_caps():
+    # gradients on 0,0,1 then comm(0,1), then a trailing gradient on 1
+    times = [1.0, 2.0, 3.0, 4.0, 5.0]
+    wi, wj, sl = [0, 0, 1, 0, 1], [-1, -1, -1, 1, -1], [0, 0, 1, -1, 1]
+    s = B.Schedule(2, 2, times, wi, wj, sl, flags=B.A2_SCHED_FUSE)
+    assert s.num_items == 2 and s.num_batches == 2
+    it = s.item(0)
+    evs, kinds = s.ops(it.first_op, it.n_ops)
+    assert (it.a, it.b, it.slot_a, it.slot_b) == (0, 1, 0, 1)
+    assert list(evs) == [0, 1, 2, 3] and list(kinds) == [B.A2_OP_GRAD_A, B.A2_OP_GRAD_A, B.A2_OP_GRAD_B, B.A2_OP_COMM]
+    tail = s.item(1)
+    assert (tail.a, tail.b, tail.n_ops) == (1, -1, 1)
+    # a cap of 2 operations per item forces spills; a change of gradient slot too
+    s2 = B.Schedule(2, 2, times, wi, wj, sl, flags=B.A2_SCHED_FUSE, max_ops_per_item=2)
+    for k in range(s2.num_items):
+        assert s2.item(k).n_ops <= 2
+    assert sorted(np.concatenate([s2.batch_events(b) for b in range(s2.num_batches)])) == [0, 1, 2, 3, 4]
+    s3 = B.Schedule(2, 2, [1.0, 2.0, 3.0], [0, 0, 0], [-1, -1, 1], [0, 1, -1], flags=B.A2_SCHED_FUSE)
+    assert s3.num_items == 2 and s3.item(0).slot_a == 0 and s3.item(1).slot_a == 1
+
+
+def test_empty_stream_and_start_times():
+    s = B.Schedule(3, 0, [], [], [], [])
+    assert s.num_batches == 0 and s.num_items == 0
+    assert np.array_equal(s.t_final(3), np.zeros(3))
+    s = B.Schedule(3, 1, [5.0], [2], [-1], [0], t_last=[1.0, 2.0, 3.0])
+    assert np.array_equal(s.t_final(3), [1.0, 2.0, 5.0])
+
+
+@pytest.mark.parametrize("times,wi,wj,sl,t_last,code", [
+    ([2.0, 1.0], [0, 1], [-1, -1], [0, 0], None, B.A2_EORDER),            # times decrease
+    ([0.5], [0], [-1], [0], [1.0, 0.0, 0.0], B.A2_EORDER),                # before the worker's time
+    ([1.5], [1], [0], [-1], [2.0, 0.0, 0.0], B.A2_EORDER),                # before the peer's time
+    ([1.0], [3], [-1], [0], None, B.A2_ERANGE),                           # worker out of range
+    ([1.0], [0], [0], [-1], None, B.A2_ERANGE),                           # i == j
+    ([1.0], [0], [-1], [1], None, B.A2_ERANGE),                           # slot out of range (1 slot)
+    ([1.0], [0], [-1], [-1], None, B.A2_ERANGE),                          # neither pair nor slot
+    ([1.0], [0], [1], [0], None, B.A2_ERANGE),                            # both pair and slot
+    ([1.0], [0], [-2], [-1], None, B.A2_ERANGE),                          # bad peer
+    ([float("nan")], [0], [-1], [0], None, B.A2_EINVAL),                  # NaN time
+    ([float("inf")], [0], [1], [-1], None, B.A2_EINVAL),
+])
+def test_malformed_streams_are_rejected(times, wi, wj, sl, t_last, code):
+    with pytest.raises(B.A2Error) as e:
+        B.Schedule(3, 1, times, wi, wj, sl, t_last=t_last)
+    assert e.value.code == code and "event" in str(e.value)
+
+
+def test_bad_arguments():
+    with pytest.raises(B.A2Error) as e:
+        B.Schedule(1, 0, [], [], [], [])
+    assert e.value.code == B.A2_EINVAL
+    with pytest.raises(B.A2Error) as e:
+        B.Schedule(3, 0, [], [], [], [], flags=64)
+    assert e.value.code == B.A2_EINVAL
+    s = B.Schedule(3, 0, [1.0], [0], [1], [-1])
+    with pytest.raises(B.A2Error):
+        s.batch_items(5)
+    with pytest.raises(B.A2Error):
+        s.item(9)
+    with pytest.raises(B.A2Error):
+        s.ops(0, 5)
