@@ -45,6 +45,16 @@ class OracleError(RuntimeError):
     pass
 
 
+def round_to_bf16(a):
+    """Values of `a` (float64) rounded to bfloat16 -- 8 exponent bits, 7 stored mantissa bits,
+    i.e. the upper half of an IEEE binary32 -- with round-to-nearest-even, returned as float64.
+    The value is first rounded to binary32 (also nearest-even). Finite inputs only."""
+    u = np.ascontiguousarray(a, dtype=np.float64).astype(np.float32).view(np.uint32).astype(np.uint64)
+    keep_odd = (u >> np.uint64(16)) & np.uint64(1)
+    u = (u + np.uint64(0x7FFF) + keep_odd) >> np.uint64(16) << np.uint64(16)
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(a))
+
+
 class OracleSim:
     """State: X, Xt of shape [n, d] (fp64), t_last[n]. Initialisation as in Algorithm 1:
     x~ <- x, t <- 0, unless given."""
@@ -90,6 +100,14 @@ class OracleSim:
 
     def apply_stream(self, ev, threads=1):
         self.apply(ev.times, ev.wi, ev.wj, ev.slot, threads=threads)
+
+    def round_rows(self, workers):
+        """Model of bf16 *storage*: the rows of these workers are rounded to bfloat16, as happens
+        whenever an implementation that keeps its state in bf16 writes them back. The arithmetic
+        between two stores stays fp64."""
+        w = np.unique(np.asarray(workers, dtype=np.int64))
+        self.X[w] = round_to_bf16(self.X[w])
+        self.Xt[w] = round_to_bf16(self.Xt[w])
 
     def consensus(self, t_eval=None):
         if t_eval is None:

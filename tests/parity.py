@@ -1,0 +1,128 @@
+"""Helpers of the GPU parity tests: build an engine for a workload, run it batch by batch and
+compare with the CPU checker element by element.
+
+fp32 storage -- bar 1e-5, element-wise, against the plain fp64 run. Metric, per row:
+    max_k |gpu_k - ref_k| / max(|ref_k|, rms(ref row)),
+a relative error whose denominator is floored by the row's root-mean-square, so that elements
+that happen to pass near zero do not blow it up.
+
+bf16 storage -- bar 2e-2, checked two ways:
+  * element-wise (same metric) against the fp64 run *with the storage modelled*: the checker's
+    rows are rounded to bf16 wherever the engine writes them back (after every item);
+  * norm-wise against the plain fp64 run: |gpu_row - ref_row|_2 / |ref_row|_2 per row.
+  The element-wise distance to the plain fp64 run is reported and only sanity-bounded: one bf16
+  store already costs up to 2^-8 = 3.9e-3 of an element, x~ integrates alpha~ times the errors
+  of x at every averaging, and an ideal bf16-storage run (fp64 arithmetic, exact rounding)
+  sits at 3-6e-2 in that metric after a few hundred events.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import spectral
+from oracle.sim import OracleSim
+from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import workload as W
+
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+BF16_ELEMENTWISE_SANITY = 0.3
+TILE_COLS = {"f32": 256 * 2 * 4, "bf16": 256 * 1 * 8}  # columns per work unit of the event kernel
+
+
+def rel_err(gpu, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    gpu = np.asarray(gpu, dtype=np.float64)
+    rms = np.sqrt((ref * ref).mean(axis=1, keepdims=True))
+    den = np.maximum(np.abs(ref), np.maximum(rms, 1e-300))
+    return float((np.abs(gpu - ref) / den).max()) if ref.size else 0.0
+
+
+def row_norm_err(gpu, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    gpu = np.asarray(gpu, dtype=np.float64)
+    num = np.sqrt(((gpu - ref) ** 2).sum(axis=1))
+    den = np.maximum(np.sqrt((ref * ref).sum(axis=1)), 1e-300)
+    return float((num / den).max()) if ref.size else 0.0
+
+
+def widen(a, storage):
+    return W.bf16_bits_to_f32(a).astype(np.float64) if storage == "bf16" else np.asarray(a, dtype=np.float64)
+
+
+def oracle_params(cfg):
+    if cfg.fixed_params is not None:
+        return tuple(float(v) for v in cfg.fixed_params)
+    return tuple(float(v) for v in spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3])
+
+
+class Checker:
+    """The fp64 run, plus (bf16 storage only) a second fp64 run whose rows are rounded to bf16
+    wherever the engine stores them."""
+
+    def __init__(self, x0, params, gamma, grads, storage, variant=0):
+        self.storage = storage
+        self.plain = OracleSim(x0, *params, gamma, grads=grads, variant=variant)
+        self.stored = OracleSim(x0, *params, gamma, grads=grads, variant=variant) if storage == "bf16" else None
+
+    def apply_batch(self, ev, sched, b):
+        idx = sched.batch_events(b)
+        order = idx[np.argsort(ev.times[idx], kind="stable")]
+        self.plain.apply(ev.times[order], ev.wi[order], ev.wj[order], ev.slot[order])
+        if self.stored is not None:
+            first, cnt = sched.batch_items(b)
+            for k in range(first, first + cnt):
+                it = sched.item(k)
+                e, _ = sched.ops(it.first_op, it.n_ops)
+                e = e[np.argsort(ev.times[e], kind="stable")]
+                self.stored.apply(ev.times[e], ev.wi[e], ev.wj[e], ev.slot[e])
+                self.stored.round_rows([it.a] + ([it.b] if it.b >= 0 else []))
+
+    def compare(self, x, xt, t, where="", cols=None):
+        """x, xt: widened device state (optionally only the columns `cols` of the checker)."""
+        pl, st = self.plain, self.stored
+        sel = (lambda a: a) if cols is None else (lambda a: a[:, cols])
+        assert np.array_equal(t, pl.t), f"times differ {where}"
+        out = {"elem_plain": max(rel_err(x, sel(pl.X)), rel_err(xt, sel(pl.Xt)))}
+        if st is None:
+            assert out["elem_plain"] <= TOL["f32"], f"parity {where}: {out}"
+        else:
+            out["elem_stored"] = max(rel_err(x, sel(st.X)), rel_err(xt, sel(st.Xt)))
+            out["norm_plain"] = max(row_norm_err(x, sel(pl.X)), row_norm_err(xt, sel(pl.Xt)))
+            assert out["elem_stored"] <= TOL["bf16"] and out["norm_plain"] <= TOL["bf16"], f"parity {where}: {out}"
+            assert out["elem_plain"] <= BF16_ELEMENTWISE_SANITY, f"parity {where}: {out}"
+        return out
+
+
+def make_small(cfg, variant=0):
+    """Engine + checker for a configuration whose arrays fit the host: same stored inputs on both."""
+    xs, xw = W.x0_matrix(cfg)
+    gs, gw = W.grad_matrix(cfg)
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage)
+    eng.write_state(xs)
+    eng.write_grads(gs)
+    if variant:
+        eng.set_variant(variant)
+    chk = Checker(xw, oracle_params(cfg), cfg.gamma, gw, cfg.storage, variant=variant)
+    return eng, chk
+
+
+def _merge(worst, out):
+    for k, v in out.items():
+        worst[k] = max(worst.get(k, 0.0), v)
+
+
+def run_batches_and_check(eng, chk, ev, flags, every=1):
+    """Plan the stream, run it one batch at a time; advance the checker through the same events
+    (sorted by time inside the batch) and, after every `every`-th batch and the last, compare the
+    whole stored state."""
+    worst = {}
+    plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+    nb = plan.sched.num_batches
+    for b in range(nb):
+        plan.run(b, 1)
+        chk.apply_batch(ev, plan.sched, b)
+        if b % every == 0 or b == nb - 1:
+            x, xt, t = eng.read_state()
+            _merge(worst, chk.compare(widen(x, chk.storage), widen(xt, chk.storage), t, where=f"after batch {b}/{nb}"))
+    plan.close()
+    return worst, nb

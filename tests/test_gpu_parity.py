@@ -1,0 +1,116 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU checker element by
+element on the same seeded inputs, after every batch."""
+import numpy as np
+import pytest
+
+from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import workload as W
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+def test_cfg1_full_every_batch(flags):
+    cfg = W.CONFIGS["cfg1"]
+    eng, chk = P.make_small(cfg)
+    worst, nb = P.run_batches_and_check(eng, chk, W.config_events(cfg), flags)
+    assert nb > 100
+    c_gpu, c_ref = eng.consensus_distance(), chk.plain.consensus()
+    assert abs(c_gpu - c_ref) <= 1e-5 * c_ref
+    eng.close()
+
+
+@pytest.mark.parametrize("name,d,n_events", [
+    ("cfg2", 20_011, 3000),   # several tiles and a ragged tail (d % 4 == 3)
+    ("cfg3", 6_150, 3000),    # d % 4 == 2
+    ("cfg4", 4_097, 4000),    # one column past two tiles
+    ("cfg5", 16_389, 4000),   # bf16: two tiles + 5 columns
+])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+def test_scaled_configs_every_batch(name, d, n_events, flags):
+    cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
+    eng, chk = P.make_small(cfg)
+    worst, nb = P.run_batches_and_check(eng, chk, W.config_events(cfg), flags)
+    print(f"{cfg.name} flags={flags} batches={nb} worst={worst}")
+    eng.close()
+
+
+@pytest.mark.parametrize("n,d", [(2, 1), (2, 3), (3, 8), (5, 9), (4, 2047), (4, 2049)])
+@pytest.mark.parametrize("storage", ["f32", "bf16"])
+def test_degenerate_sizes(n, d, storage):
+    cfg = W.WorkloadConfig(name=f"tiny{n}x{d}", n=n, graph="ring", d=d, storage=storage, n_events=300,
+                           x0_std=1.0, g_std=0.5, gamma=0.05, edge_rate=1.0, fixed_params=(0.7, 0.5, 1.5), seed=77)
+    for flags in (0, B.A2_SCHED_FUSE):
+        eng, chk = P.make_small(cfg)
+        P.run_batches_and_check(eng, chk, W.config_events(cfg), flags, every=7)
+        eng.close()
+
+
+def test_fused_and_unfused_schedules_are_bit_identical():
+    """Fusion only changes which rows share a trip through registers, not the arithmetic."""
+    cfg = W.CONFIGS["cfg4"].scaled(d=10_003, n_events=3000)
+    ev = W.config_events(cfg)
+    out = []
+    for flags in (0, B.A2_SCHED_FUSE):
+        eng, _ = P.make_small(cfg)
+        eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+        out.append(eng.read_state())
+        eng.close()
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    assert np.array_equal(out[0][2], out[1][2])
+
+
+def test_message_before_mix_variant():
+    cfg = W.CONFIGS["cfg3"].scaled(d=5_001, n_events=1500)
+    eng, chk = P.make_small(cfg, variant=B.A2_MSG_BEFORE_MIX)
+    P.run_batches_and_check(eng, chk, W.config_events(cfg), B.A2_SCHED_FUSE, every=5)
+    eng.close()
+
+
+def test_baseline_parameters_keep_momentum_equal_to_x():
+    """eta = 0, alpha = alpha~ = 1/2 (Prop. 3.6, non-accelerated): x~ stays a bit-exact copy of x."""
+    cfg = W.CONFIGS["cfg2"].scaled(d=3_000, n_events=2000)
+    xs, _ = W.x0_matrix(cfg)
+    gs, _ = W.grad_matrix(cfg)
+    eng = B.Engine(cfg.n, cfg.d, *B.prescribe(1.0, 1.0, accelerated=False), cfg.gamma)
+    eng.write_state(xs)
+    eng.write_grads(gs)
+    ev = W.config_events(cfg)
+    eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    x, xt, _ = eng.read_state()
+    assert np.array_equal(x, xt)
+    eng.close()
+
+
+@pytest.mark.parametrize("name,d", [("cfg1", 10_000), ("cfg2", 50_001), ("cfg5", 30_005)])
+def test_consensus_distance_stored_and_at_common_time(name, d):
+    cfg = W.CONFIGS[name].scaled(d=d, n_events=1500)
+    eng, chk = P.make_small(cfg)
+    sim = chk.plain
+    ev = W.config_events(cfg)
+    c0g, c0r = eng.consensus_distance(), sim.consensus()
+    assert abs(c0g - c0r) <= 2e-6 * c0r
+    eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    sim.apply_stream(ev)
+    x, xt, t = eng.read_state()
+    # the reduction itself, on exactly the rows the device holds
+    from oracle.sim import OracleSim
+    on_dev = OracleSim(P.widen(x, cfg.storage), sim.eta, sim.alpha, sim.alpha_tilde, sim.gamma,
+                       xt0=P.widen(xt, cfg.storage), t0=t)
+    assert abs(eng.consensus_distance() - on_dev.consensus()) <= 2e-6 * on_dev.consensus()
+    t_eval = float(ev.times[-1]) + 0.25
+    assert abs(eng.consensus_distance(t_eval) - on_dev.consensus(t_eval)) <= 2e-6 * on_dev.consensus(t_eval)
+    # and end to end against the checker's own state
+    tol = 1e-4 if cfg.storage == "f32" else 5e-2
+    assert abs(eng.consensus_distance() - sim.consensus()) <= tol * sim.consensus()
+    assert abs(eng.consensus_distance(t_eval) - sim.consensus(t_eval)) <= tol * sim.consensus(t_eval)
+    eng.close()
+
+
+def test_exact_consensus_is_zero():
+    eng = B.Engine(4, 1000, 0.0, 0.5, 0.5, 0.0)
+    row = np.random.default_rng(0).standard_normal(1000).astype(np.float32)
+    eng.write_state(np.tile(row, (4, 1)))
+    assert eng.consensus_distance() == 0.0
+    eng.close()

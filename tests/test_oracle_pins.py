@@ -437,3 +437,22 @@ def test_prescription_formulas():
     assert abs(eta * 2 * math.sqrt(c1 * c2) - 1) < 1e-12
     assert abs(at - 0.5 * math.sqrt(c1 / c2)) < 1e-12 and alpha == 0.5
     assert spectral.prescribe(64, e, np.full(64, 0.5), accelerated=False)[:3] == (0.0, 0.5, 0.5)
+
+
+# ---- bf16 storage model -------------------------------------------------------------------
+def test_bf16_rounding_of_the_storage_model():
+    from oracle.sim import round_to_bf16
+
+    # exactly representable values stay; ties go to the even mantissa; spacing is 2^-7 in [1, 2)
+    v = np.array([1.0, -0.5, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, 3.0e-5])
+    r = round_to_bf16(v)
+    assert r[0] == 1.0 and r[1] == -0.5 and r[2] == 1.0 + 2.0 ** -7
+    assert r[3] == 1.0 and r[4] == 1.0 + 2.0 ** -6 and r[5] == 1.0 + 2.0 ** -7
+    assert np.all(np.abs(r - v) <= np.abs(v) * 2.0 ** -8)
+    assert np.array_equal(round_to_bf16(r), r)
+    # agrees with the input generator's independent bit-twiddling on random data
+    a = np.random.default_rng(3).standard_normal(5000) * 0.02
+    assert np.array_equal(round_to_bf16(a), W.bf16_bits_to_f32(W.f32_to_bf16_bits(a.astype(np.float32))).astype(np.float64))
+    s = OracleSim(np.array([[1.0 + 2.0 ** -9, 2.0], [3.0, 1.0 + 2.0 ** -9]]), 0.1, 0.5, 0.5, 0.0)
+    s.round_rows([1])
+    assert s.X[0, 0] == 1.0 + 2.0 ** -9 and s.X[1, 1] == 1.0 and s.Xt[1, 1] == 1.0
