@@ -129,13 +129,22 @@ def fill_engine(eng, cfg, threads):
         stored, _ = (W.x0_row if which == "x" else W.grad_row)(cfg, row)
         return which, row, stored
 
-    jobs = [("x", i) for i in range(cfg.n)] + [("g", i) for i in range(cfg.n)]
+    jobs = [("x", i) for i in range(cfg.n)] + [("g", i) for i in range(cfg.n_grad_slots)]
     with ThreadPoolExecutor(max(1, threads)) as ex:
         for which, row, stored in ex.map(job, jobs):
             eng.fill_row(which, row, stored)
     eng.xt.copy_(eng.x)
     eng.set_times(np.zeros(cfg.n))
     eng.sync()
+
+
+def sample_inputs(cfg, n_cols, threads):
+    """Widened (fp64) first n_cols columns of x0 and of the gradient rows."""
+    cols = np.arange(n_cols)
+    with ThreadPoolExecutor(max(1, threads)) as ex:
+        xw = np.stack(list(ex.map(lambda i: W.x0_row(cfg, i, cols)[1], range(cfg.n))))
+        gw = np.stack(list(ex.map(lambda i: W.grad_row(cfg, i, cols)[1], range(cfg.n_grad_slots))))
+    return xw, gw
 
 
 def cpu_baseline(cfg, ev, n_cols, threads):
@@ -145,9 +154,7 @@ def cpu_baseline(cfg, ev, n_cols, threads):
     from oracle import spectral
     from oracle.sim import OracleSim
 
-    cols = np.arange(n_cols)
-    xw = np.stack([W.x0_row(cfg, i, cols)[1] for i in range(cfg.n)])
-    gw = np.stack([W.grad_row(cfg, i, cols)[1] for i in range(cfg.n)])
+    xw, gw = sample_inputs(cfg, n_cols, threads)
     if cfg.fixed_params is not None:
         params = cfg.fixed_params
     else:
@@ -171,9 +178,7 @@ def run_reference(args, cfg, ranks):
     from oracle import spectral
     from oracle.sim import OracleSim
 
-    cols = np.arange(n_cols)
-    xw = np.stack([W.x0_row(cfg, i, cols)[1] for i in range(cfg.n)])
-    gw = np.stack([W.grad_row(cfg, i, cols)[1] for i in range(cfg.n)])
+    xw, gw = sample_inputs(cfg, n_cols, threads)
     params = cfg.fixed_params if cfg.fixed_params is not None else spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
     sim = OracleSim(xw, *params, cfg.gamma, grads=gw)
     t_timed = 0.0
@@ -232,7 +237,8 @@ def main():
     n_steps = W_ + K
     threads = max(1, min(os.cpu_count() or 1, 32) // max(1, ranks.world))
 
-    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, device=str(device))
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
+                   device=str(device))
     fill_engine(eng, cfg, threads)
     ev_all = W.config_events(cfg, n_events=2 * n_steps * eps)  # first half: resident pass; second: end to end
 
@@ -331,12 +337,12 @@ def main():
 
     if ranks.rank == 0 and ranks.world == 1 and not args.skip_cpu_baseline:
         cores = max(1, min(os.cpu_count() or 1, 32))
-        n_cols = args.cpu_sample_cols or max(1, min(cfg.d, 1_280_000))
-        sample_ev = W.config_events(cfg, n_events=eps)
+        n_cols = args.cpu_sample_cols or max(1, min(cfg.d, 2_560_000))
+        sample_ev = W.config_events(cfg, n_events=4 * eps)
         v, dt, _ = cpu_baseline(cfg, sample_ev, n_cols, cores)
         line["cpu_baseline"] = {
             "value": v, "unit": "events/s", "cores": cores, "kind": "oracle", "seconds": dt,
-            "sample": f"first {n_cols} of {cfg.d} columns, all {cfg.n} workers, {eps} events + one consensus "
+            "sample": f"first {n_cols} of {cfg.d} columns, all {cfg.n} workers, {4 * eps} events + one consensus "
                       f"distance; events/s scaled by the column fraction"}
     eng.close()
     if ranks.rank == 0:

@@ -8,11 +8,18 @@
 //   consensus kernel  per column: sum_i (x_i - xbar)^2 from shifted sums, fp64 across columns,
 //                     warp shuffle + block reduce, per-block partials, fixed-order final sum.
 //
-// Per-element arithmetic (fp32, explicit FMAs, identical for fused and unfused schedules):
-//   mixing    dlt = x - x~;  x = fma(-c, dlt, x);  x~ = fma(c, dlt, x~)        (Algorithm 1, matrix exponential)
-//   gradient  x = fma(-gamma, g, x);  x~ = fma(-gamma, g, x~)                  (Eq. (dynamic), dN term)
-//   comm      m = x_a - x_b;  x_a = fma(-alpha, m, x_a);  x~_a = fma(-alpha~, m, x~_a);
-//             x_b = fma(alpha, m, x_b);  x~_b = fma(alpha~, m, x~_b)           (Eq. (dynamic), dM term)
+// Per-element arithmetic (fp32, explicit FMAs, identical for fused and unfused schedules). Every
+// stored value is updated as value + increment with ONE rounding at the value's own magnitude; the
+// increment collects the mixing term and the jump and is itself small near consensus, so its
+// rounding errors are small too:
+//   gradient  dlt = x - x~;  tg = -gamma g;
+//             x += fma(-c, dlt, tg);  x~ += fma(c, dlt, tg)            (Algorithm 1: matrix exponential, then
+//                                                                       the two -gamma g lines; Eq. (dynamic), dN term)
+//   comm      u_a = -c_a (x_a - x~_a);  u_b = -c_b (x_b - x~_b);         (mixing increments of x; those of x~ are -u)
+//             m = (x_a - x_b) + (u_a - u_b)                             (x_a - x_b after both were mixed to t)
+//             x_a += fma(-alpha, m, u_a);  x~_a += fma(-alpha~, m, -u_a);
+//             x_b += fma( alpha, m, u_b);  x~_b += fma( alpha~, m, -u_b)  (Eq. (dynamic), dM term)
+//   (message-before-mix variant: m = x_a - x_b from the un-mixed rows.)
 // The mixing coefficient c = -expm1(-2 eta (t - t_prev)) / 2 is evaluated in fp64 on the device
 // from the event time and the worker's previous time carried by the descriptor, then rounded
 // once to fp32.
@@ -67,10 +74,25 @@ template <> struct Vec<__nv_bfloat16> {
     }
 };
 
-__device__ __forceinline__ void mix_elem(float& x, float& xt, float c) {
+// Gradient event on one element: mixing over the elapsed time, then -gamma g on both buffers.
+__device__ __forceinline__ void grad_elem(float& x, float& xt, float c, float ngamma, float g) {
     const float dlt = __fsub_rn(x, xt);
-    x = __fmaf_rn(-c, dlt, x);
-    xt = __fmaf_rn(c, dlt, xt);
+    const float tg = __fmul_rn(ngamma, g);
+    x = __fadd_rn(x, __fmaf_rn(-c, dlt, tg));
+    xt = __fadd_rn(xt, __fmaf_rn(c, dlt, tg));
+}
+
+// Communication event on one element of workers a and b.
+__device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, float& xtb, float ca, float cb,
+                                          float alpha, float alpha_t, bool msg_before_mix) {
+    const float ua = __fmul_rn(-ca, __fsub_rn(xa, xta));
+    const float ub = __fmul_rn(-cb, __fsub_rn(xb, xtb));
+    const float raw = __fsub_rn(xa, xb);
+    const float m = msg_before_mix ? raw : __fadd_rn(raw, __fsub_rn(ua, ub));
+    xa = __fadd_rn(xa, __fmaf_rn(-alpha, m, ua));
+    xta = __fadd_rn(xta, __fmaf_rn(-alpha_t, m, -ua));
+    xb = __fadd_rn(xb, __fmaf_rn(alpha, m, ub));
+    xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m, -ub));
 }
 
 __device__ __forceinline__ double mix_coeff(double eta, double dt) { return -0.5 * expm1(-2.0 * eta * dt); }
@@ -162,42 +184,20 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-                    for (int k = 0; k < N; ++k) {
-                        mix_elem(xa[u][k], xta[u][k], c);
-                        xa[u][k] = __fmaf_rn(ngamma, ga[u][k], xa[u][k]);
-                        xta[u][k] = __fmaf_rn(ngamma, ga[u][k], xta[u][k]);
-                    }
+                    for (int k = 0; k < N; ++k) grad_elem(xa[u][k], xta[u][k], c, ngamma, ga[u][k]);
             } else if (kind == A2_OP_GRAD_B) {
                 const float c = s_cb[o];
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-                    for (int k = 0; k < N; ++k) {
-                        mix_elem(xb[u][k], xtb[u][k], c);
-                        xb[u][k] = __fmaf_rn(ngamma, gb[u][k], xb[u][k]);
-                        xtb[u][k] = __fmaf_rn(ngamma, gb[u][k], xtb[u][k]);
-                    }
+                    for (int k = 0; k < N; ++k) grad_elem(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
             } else {
                 const float ca = s_ca[o], cb = s_cb[o];
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-                    for (int k = 0; k < N; ++k) {
-                        float m;
-                        if (p.msg_before_mix) {
-                            m = __fsub_rn(xa[u][k], xb[u][k]);
-                            mix_elem(xa[u][k], xta[u][k], ca);
-                            mix_elem(xb[u][k], xtb[u][k], cb);
-                        } else {
-                            mix_elem(xa[u][k], xta[u][k], ca);
-                            mix_elem(xb[u][k], xtb[u][k], cb);
-                            m = __fsub_rn(xa[u][k], xb[u][k]);
-                        }
-                        xa[u][k] = __fmaf_rn(-alpha, m, xa[u][k]);
-                        xta[u][k] = __fmaf_rn(-alpha_t, m, xta[u][k]);
-                        xb[u][k] = __fmaf_rn(alpha, m, xb[u][k]);
-                        xtb[u][k] = __fmaf_rn(alpha_t, m, xtb[u][k]);
-                    }
+                    for (int k = 0; k < N; ++k)
+                        comm_elem(xa[u][k], xta[u][k], xb[u][k], xtb[u][k], ca, cb, alpha, alpha_t, p.msg_before_mix != 0);
             }
         }
 

@@ -120,8 +120,13 @@ class WorkloadConfig:
     comms_per_grad: float | None = None  # else: averagings per worker per unit time
     fixed_params: tuple | None = None  # (eta, alpha, alpha_tilde) if given outright
     consensus_every: int = 0
+    grad_pool: int = 1  # gradient rows per worker, used round-robin by its gradient events
     seed: int = 0
     note: str = ""
+
+    @property
+    def n_grad_slots(self) -> int:
+        return self.n * self.grad_pool
 
     def edges(self) -> np.ndarray:
         return make_edges(self.graph, self.n)
@@ -148,12 +153,12 @@ CONFIGS = {
     # n=4 ring, unit rate per edge and per worker, all hyper-parameters given outright.
     "cfg1": WorkloadConfig(
         name="cfg1", n=4, graph="ring", d=10_000, storage="f32", n_events=2_000,
-        x0_std=1.0, g_std=1.0, gamma=0.01, edge_rate=1.0, fixed_params=(0.5, 0.5, 0.5),
+        x0_std=1.0, g_std=1.0, gamma=0.01, edge_rate=1.0, fixed_params=(0.5, 0.5, 0.5), grad_pool=16,
         seed=1001, note="n=4 ring, d=1e4 fp32"),
     # n=16 complete, one averaging per worker per gradient step.
     "cfg2": WorkloadConfig(
         name="cfg2", n=16, graph="complete", d=1_000_000, storage="f32", n_events=50_000,
-        x0_std=1.0, g_std=0.1, gamma=0.01, comms_per_grad=1.0,
+        x0_std=1.0, g_std=0.1, gamma=0.01, comms_per_grad=1.0, grad_pool=128,
         seed=1002, note="n=16 complete, d=1e6 fp32"),
     # n=32 ring, ResNet-18-sized flat vector, rate 2 per edge.
     "cfg3": WorkloadConfig(
@@ -200,11 +205,13 @@ def _rng(seed: int, tag: int, row: int = 0) -> np.random.Generator:
 
 
 def poisson_events(n: int, edges: np.ndarray, rates: np.ndarray, n_events: int, seed: int,
-                   grad_rate: float = 1.0, t0: float = 0.0, stream_id: int = 0) -> EventStream:
+                   grad_rate: float = 1.0, t0: float = 0.0, stream_id: int = 0, grad_pool: int = 1) -> EventStream:
     """Superposition of independent Poisson clocks (Assumption 3.1): one clock of rate
     `grad_rate` per worker and one of rate rates[e] per edge. The superposition is a Poisson
     process of rate R = n*grad_rate + sum(rates); each event belongs to a clock with
-    probability rate/R. Worker i's gradient events use gradient slot i."""
+    probability rate/R. Worker i owns the gradient rows i, i + n, ..., i + (grad_pool-1) n and
+    its k-th gradient event uses row i + n (k mod grad_pool): the paper's stochastic gradients
+    are fresh draws at every step (Sec. 3.2), a pool of rows stands in for them."""
     edges = np.asarray(edges, dtype=np.int32).reshape(-1, 2)
     rates = np.asarray(rates, dtype=np.float64)
     if rates.shape[0] != edges.shape[0]:
@@ -222,7 +229,13 @@ def poisson_events(n: int, edges: np.ndarray, rates: np.ndarray, n_events: int, 
     wj = np.full(n_events, -1, dtype=np.int32)
     slot = np.full(n_events, -1, dtype=np.int32)
     wi[is_grad] = which[is_grad]
-    slot[is_grad] = which[is_grad]
+    gw = which[is_grad]
+    # k-th gradient event of each worker -> k (stable sort groups a worker's events in time order)
+    order = np.argsort(gw, kind="stable")
+    starts = np.concatenate([[0], np.cumsum(np.bincount(gw, minlength=n))[:-1]])
+    kth = np.empty(len(gw), dtype=np.int64)
+    kth[order] = np.arange(len(gw)) - starts[gw[order]]
+    slot[is_grad] = gw + n * (kth % max(1, int(grad_pool)))
     e_idx = which[~is_grad] - n
     wi[~is_grad] = edges[e_idx, 0]
     wj[~is_grad] = edges[e_idx, 1]
@@ -233,7 +246,7 @@ def poisson_events(n: int, edges: np.ndarray, rates: np.ndarray, n_events: int, 
 def config_events(cfg: WorkloadConfig, n_events: int | None = None, t0: float = 0.0,
                   stream_id: int = 0) -> EventStream:
     return poisson_events(cfg.n, cfg.edges(), cfg.rates(), cfg.n_events if n_events is None else n_events,
-                          cfg.seed, t0=t0, stream_id=stream_id)
+                          cfg.seed, t0=t0, stream_id=stream_id, grad_pool=cfg.grad_pool)
 
 
 # --------------------------------------------------------------------------------------
@@ -282,7 +295,7 @@ def x0_matrix(cfg: WorkloadConfig):
 
 
 def grad_matrix(cfg: WorkloadConfig):
-    rows = [grad_row(cfg, i) for i in range(cfg.n)]
+    rows = [grad_row(cfg, i) for i in range(cfg.n_grad_slots)]
     return np.stack([r[0] for r in rows]), np.stack([r[1] for r in rows])
 
 

@@ -97,7 +97,7 @@ def make_small(cfg, variant=0):
     """Engine + checker for a configuration whose arrays fit the host: same stored inputs on both."""
     xs, xw = W.x0_matrix(cfg)
     gs, gw = W.grad_matrix(cfg)
-    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage)
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots)
     eng.write_state(xs)
     eng.write_grads(gs)
     if variant:

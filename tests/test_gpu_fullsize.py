@@ -25,8 +25,8 @@ def _fill(eng, cfg, cols):
         return which, row, stored, wide[cols]
 
     xw = np.empty((cfg.n, len(cols)))
-    gw = np.empty((cfg.n, len(cols)))
-    jobs = [("x", i) for i in range(cfg.n)] + [("g", i) for i in range(cfg.n)]
+    gw = np.empty((cfg.n_grad_slots, len(cols)))
+    jobs = [("x", i) for i in range(cfg.n)] + [("g", i) for i in range(cfg.n_grad_slots)]
     with ThreadPoolExecutor(min(16, os.cpu_count() or 1)) as ex:
         for which, row, stored, wide in ex.map(job, jobs):
             eng.fill_row(which, row, stored)
@@ -66,14 +66,13 @@ def test_full_size_sampled_columns_every_batch(name):
     cfg = W.CONFIGS[name]
     cols = W.sample_columns(cfg.d, P.TILE_COLS[cfg.storage], 3000, seed=cfg.seed)
     cols_t = torch.from_numpy(cols).to("cuda:0")
-    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage)
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots)
     xw, gw = _fill(eng, cfg, cols)
     chk = P.Checker(xw, P.oracle_params(cfg), cfg.gamma, gw, cfg.storage)
     ev = W.config_events(cfg)
     plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
     nb = plan.sched.num_batches
     worst = {}
-    every = max(1, cfg.consensus_every) if cfg.consensus_every else 0
     for b in range(nb):
         plan.run(b, 1)
         chk.apply_batch(ev, plan.sched, b)

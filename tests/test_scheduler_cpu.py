@@ -38,7 +38,7 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
     params = (0.4, 0.5, 1.3)
     ref = OracleSim(x0, *params, cfg.gamma, grads=G)
     ref.apply_stream(ev)
-    s = B.Schedule(cfg.n, cfg.n, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+    s = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
     sim, seen = _replay(cfg, ev, s, params, x0, G)
     assert np.array_equal(np.sort(seen), np.arange(len(ev)))  # every event exactly once
     assert np.array_equal(sim.X, ref.X) and np.array_equal(sim.Xt, ref.Xt) and np.array_equal(sim.t, ref.t)

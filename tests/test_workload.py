@@ -43,6 +43,13 @@ def test_event_counts_and_pair_histogram():
     # gradient events are spread evenly over workers and use their own slot
     g = ev.wi[ev.wj < 0]
     assert np.array_equal(ev.slot[ev.wj < 0], g)
+    # with a pool of rows per worker, a worker's gradient events walk its rows round-robin
+    ev4 = W.poisson_events(n, e, rates, 5_000, seed=5, grad_pool=4)
+    ev1 = W.poisson_events(n, e, rates, 5_000, seed=5)
+    assert np.array_equal(ev4.times, ev1.times) and np.array_equal(ev4.wi, ev1.wi) and np.array_equal(ev4.wj, ev1.wj)
+    for w in range(n):
+        sl = ev4.slot[(ev4.wj < 0) & (ev4.wi == w)]
+        assert np.array_equal(sl, w + n * (np.arange(len(sl)) % 4))
     cnt = np.bincount(g, minlength=n)
     assert np.all(np.abs(cnt - n_grad / n) < 5 * np.sqrt(n_grad / n))
     # pairs are proportional to lambda^{ij} and only edges occur
