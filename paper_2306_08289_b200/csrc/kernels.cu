@@ -16,9 +16,11 @@
 //             x += fma(-c, dlt, tg);  x~ += fma(c, dlt, tg)            (Algorithm 1: matrix exponential, then
 //                                                                       the two -gamma g lines; Eq. (dynamic), dN term)
 //   comm      u_a = -c_a (x_a - x~_a);  u_b = -c_b (x_b - x~_b);         (mixing increments of x; those of x~ are -u)
-//             m = (x_a - x_b) + (u_a - u_b)                             (x_a - x_b after both were mixed to t)
-//             x_a += fma(-alpha, m, u_a);  x~_a += fma(-alpha~, m, -u_a);
-//             x_b += fma( alpha, m, u_b);  x~_b += fma( alpha~, m, -u_b)  (Eq. (dynamic), dM term)
+//             m = (x_a - x_b) + (u_a - u_b)                             (x_a - x_b after both were mixed to t),
+//             kept as an unevaluated sum m_hi + m_lo (error-free two-sums), because alpha~ can be
+//             several times alpha and would amplify m's own rounding error into x~;
+//             x_a += -alpha m + u_a;  x~_a += -alpha~ m - u_a;
+//             x_b +=  alpha m + u_b;  x~_b +=  alpha~ m - u_b             (Eq. (dynamic), dM term)
 //   (message-before-mix variant: m = x_a - x_b from the un-mixed rows.)
 // The mixing coefficient c = -expm1(-2 eta (t - t_prev)) / 2 is evaluated in fp64 on the device
 // from the event time and the worker's previous time carried by the descriptor, then rounded
@@ -87,12 +89,24 @@ __device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, floa
                                           float alpha, float alpha_t, bool msg_before_mix) {
     const float ua = __fmul_rn(-ca, __fsub_rn(xa, xta));
     const float ub = __fmul_rn(-cb, __fsub_rn(xb, xtb));
-    const float raw = __fsub_rn(xa, xb);
-    const float m = msg_before_mix ? raw : __fadd_rn(raw, __fsub_rn(ua, ub));
-    xa = __fadd_rn(xa, __fmaf_rn(-alpha, m, ua));
-    xta = __fadd_rn(xta, __fmaf_rn(-alpha_t, m, -ua));
-    xb = __fadd_rn(xb, __fmaf_rn(alpha, m, ub));
-    xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m, -ub));
+    // raw + e_raw == x_a - x_b exactly (two-sum)
+    const float nb = -xb;
+    const float raw = __fadd_rn(xa, nb);
+    float bv = __fsub_rn(raw, xa);
+    float av = __fsub_rn(raw, bv);
+    const float e_raw = __fadd_rn(__fsub_rn(xa, av), __fsub_rn(nb, bv));
+    float m = raw, m_lo = e_raw;
+    if (!msg_before_mix) {  // m + e_m == raw + du exactly
+        const float du = __fsub_rn(ua, ub);
+        m = __fadd_rn(raw, du);
+        bv = __fsub_rn(m, raw);
+        av = __fsub_rn(m, bv);
+        m_lo = __fadd_rn(e_raw, __fadd_rn(__fsub_rn(raw, av), __fsub_rn(du, bv)));
+    }
+    xa = __fadd_rn(xa, __fmaf_rn(-alpha, m, __fmaf_rn(-alpha, m_lo, ua)));
+    xta = __fadd_rn(xta, __fmaf_rn(-alpha_t, m, __fmaf_rn(-alpha_t, m_lo, -ua)));
+    xb = __fadd_rn(xb, __fmaf_rn(alpha, m, __fmaf_rn(alpha, m_lo, ub)));
+    xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m, __fmaf_rn(alpha_t, m_lo, -ub)));
 }
 
 __device__ __forceinline__ double mix_coeff(double eta, double dt) { return -0.5 * expm1(-2.0 * eta * dt); }

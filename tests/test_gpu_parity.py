@@ -73,7 +73,7 @@ def test_baseline_parameters_keep_momentum_equal_to_x():
     cfg = W.CONFIGS["cfg2"].scaled(d=3_000, n_events=2000)
     xs, _ = W.x0_matrix(cfg)
     gs, _ = W.grad_matrix(cfg)
-    eng = B.Engine(cfg.n, cfg.d, *B.prescribe(1.0, 1.0, accelerated=False), cfg.gamma)
+    eng = B.Engine(cfg.n, cfg.d, *B.prescribe(1.0, 1.0, accelerated=False), cfg.gamma, n_grad_slots=cfg.n_grad_slots)
     eng.write_state(xs)
     eng.write_grads(gs)
     ev = W.config_events(cfg)
