@@ -148,6 +148,37 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
  * written back). Waits for the stream; *out is a host double. */
 int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out);
 
+/* The paper has no counterpart for this call; it exists for callers that must not allocate.
+ *
+ * Consensus distance of the stored rows (as a2cid2_consensus_distance with t_eval = NaN) for
+ * programs in which nothing may call cudaMalloc once they are running: for example a trainer
+ * whose own memory pool has already claimed the whole device, so that a raw allocation made by
+ * a library would fail or steal from that pool; or a loop with a latency budget, since
+ * cudaMalloc and cudaFree can stall the whole device. The call needs no handle and obtains no
+ * device or pinned memory, and neither does anything it calls (only a failing call stores an
+ * error text on the host). The per-block
+ * partial sums, which the handle-based call keeps in memory it allocated at bind time, live here
+ * in a fixed array of 4096 doubles (32 KB) inside the library image; every GPU on which the
+ * library is used holds that array until the process exits.
+ *
+ *   x           device, [n, row_pitch_elems] of storage_dtype, 16-byte aligned, only read
+ *   n, d        2 <= n <= 4096; 1 <= d <= 67,108,864 for A2_F32 and 134,217,728 for A2_BF16
+ *               (4096 partials x 4096 vectors of 16 bytes per row); a larger d is rejected with
+ *               A2_ERANGE and a message, nothing is launched
+ *   row_pitch_elems  >= d, multiple of 8
+ *   cuda_stream a cudaStream_t (NULL = default stream); the work is queued there, not waited for
+ *   out_device  device, one double, written by the queued work; the caller owns it
+ *
+ * The first call on each device looks up the device address of the fixed array (with that
+ * device current) and remembers it; make that first call during start-up, outside any stream
+ * capture. All calls on one device share the array: a call overwrites every entry it later
+ * reads, so nothing has to be cleared between calls, but two calls whose work overlaps on the
+ * GPU (different streams, no ordering between them) race on it and give wrong sums. Calls on
+ * one stream, or otherwise ordered, are safe. Errors: A2_EINVAL, A2_ERANGE, A2_ECUDA; the text
+ * is available from a2cid2_last_error(NULL). */
+int a2cid2_consensus_distance_static(const void* x, int32_t n, int64_t d, int64_t row_pitch_elems,
+                                     int32_t storage_dtype, void* cuda_stream, double* out_device);
+
 /* Wait for all work queued by this handle; returns the first deferred CUDA error, if any. */
 int a2cid2_sync(a2cid2_t* h);
 

@@ -64,6 +64,7 @@ SIGNATURES = {
     "a2cid2_set_times": (C.c_int, [_vp, _dp]),
     "a2cid2_apply_events": (C.c_int, [_vp, C.c_int64, _dp, _ip, _ip, _ip, C.c_uint32, C.POINTER(Stats)]),
     "a2cid2_consensus_distance": (C.c_int, [_vp, C.c_double, _dp]),
+    "a2cid2_consensus_distance_static": (C.c_int, [_vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, _vp, _vp]),
     "a2cid2_sync": (C.c_int, [_vp]),
     "a2cid2_last_error": (C.c_char_p, [_vp]),
     "a2cid2_destroy": (None, [_vp]),
@@ -146,6 +147,14 @@ def config_params(cfg):
         return tuple(float(v) for v in cfg.fixed_params)
     c1, c2 = graph_chi(cfg.n, cfg.edges(), cfg.rates())
     return prescribe(c1, c2, True)
+
+
+def consensus_distance_static(x_ptr, n, d, row_pitch_elems, storage_dtype, cuda_stream, out_device_ptr):
+    """a2cid2_consensus_distance_static: consensus distance of the rows at device address x_ptr,
+    queued on cuda_stream, result written to the device double at out_device_ptr. For callers
+    that may not allocate: the call itself allocates nothing (see include/a2cid2.h)."""
+    _check(lib().a2cid2_consensus_distance_static(x_ptr, n, d, row_pitch_elems, storage_dtype, cuda_stream,
+                                                  out_device_ptr))
 
 
 class Schedule:

@@ -101,6 +101,13 @@ int consensus_grid(const DeviceInfo& dev);
 int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double eta,
                      const double* dt, double* partials, int n_partials, double* out, void* stream);
 
+// Consensus distance of the stored state with the partial sums in the library's fixed device
+// array (no allocation anywhere). out_device is a device double. Returns a cudaError_t as int.
+constexpr int kStaticMaxPartials = 4096;
+int launch_consensus_static(const void* x, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double* out_device,
+                            void* stream, int* n_partials_out);
+int64_t consensus_static_max_columns(int32_t dtype);
+
 // ---- spectral (spectral.cpp) -----------------------------------------------------------------
 int graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda, double* chi1,
               double* chi2, std::string& err);

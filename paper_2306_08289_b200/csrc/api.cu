@@ -428,6 +428,30 @@ void a2cid2_destroy(a2cid2_t* h) {
     delete h;
 }
 
+int a2cid2_consensus_distance_static(const void* x, int32_t n, int64_t d, int64_t row_pitch_elems, int32_t storage_dtype,
+                                     void* cuda_stream, double* out_device) {
+    if (!x || !out_device) return fail(nullptr, A2_EINVAL, "x or out_device is NULL");
+    if (storage_dtype != A2_F32 && storage_dtype != A2_BF16) return fail(nullptr, A2_EINVAL, "unknown storage type");
+    if (n < 2 || n > 4096) return fail(nullptr, A2_EINVAL, "need 2 <= n <= 4096 workers");
+    if (d < 1) return fail(nullptr, A2_EINVAL, "need d >= 1");
+    if (row_pitch_elems < d || row_pitch_elems % 8 != 0)
+        return fail(nullptr, A2_EINVAL, "row pitch must be >= d and a multiple of 8 elements");
+    if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(out_device) & 7))
+        return fail(nullptr, A2_EINVAL, "x must be 16-byte aligned and out_device 8-byte aligned");
+    const int64_t max_d = a2::consensus_static_max_columns(storage_dtype);
+    if (d > max_d) {
+        char buf[200];
+        std::snprintf(buf, sizeof buf,
+                      "d = %lld exceeds the %lld columns the fixed scratch array of this entry point covers; "
+                      "use a2cid2_consensus_distance",
+                      (long long)d, (long long)max_d);
+        return fail(nullptr, A2_ERANGE, buf);
+    }
+    const int rc = a2::launch_consensus_static(x, row_pitch_elems, n, d, storage_dtype, out_device, cuda_stream, nullptr);
+    if (rc != 0) return fail_cuda(nullptr, (cudaError_t)rc, "static consensus launch");
+    return A2_OK;
+}
+
 // ---- plans -----------------------------------------------------------------------------------
 
 int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, const double* times, const int32_t* wi,

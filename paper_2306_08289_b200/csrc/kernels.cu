@@ -29,6 +29,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 
 #include "a2cid2_internal.h"
 
@@ -384,6 +385,65 @@ int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, in
     if (e != cudaSuccess) return (int)e;
     k_consensus_final<<<1, kThreads, 0, stream>>>(partials, n_partials, out);
     return (int)cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Consensus distance without any allocation: the per-block partial sums live in a fixed array
+// that is part of the loaded library image instead of in memory obtained at run time.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticVecPerBlock = 4096;  // 128-bit vectors of one row handled by one block
+static __device__ __align__(256) double g_static_partials[kStaticMaxPartials];
+
+// Host code may not hand `g_static_partials` to a kernel: in host code that name is only a
+// stand-in for the device symbol. Its device address is looked up once per device, with that
+// device current, and cached here.
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+double* g_static_addr[kMaxDevices] = {};
+
+}  // namespace
+
+int launch_consensus_static(const void* x, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double* out_device,
+                            void* stream_, int* n_partials_out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= kMaxDevices) return (int)cudaErrorInvalidDevice;
+    double* partials = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_addr[dev]) {
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_static_partials);
+            if (e != cudaSuccess) return (int)e;
+            g_static_addr[dev] = static_cast<double*>(p);
+        }
+        partials = g_static_addr[dev];
+    }
+    const int vec = dtype == A2_BF16 ? 8 : 4;
+    const int64_t n_vec = (d + vec - 1) / vec;
+    const int64_t blocks = (n_vec + kStaticVecPerBlock - 1) / kStaticVecPerBlock;
+    if (blocks < 1 || blocks > kStaticMaxPartials) return (int)cudaErrorInvalidValue;  // checked by the caller too
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // every block overwrites its own partial and the final pass reads exactly `blocks` of them,
+    // so nothing left in the array by an earlier call is ever read
+    if (dtype == A2_BF16)
+        k_consensus_partial<__nv_bfloat16, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(x), nullptr, pitch, n, d, 0.0, nullptr, partials);
+    else
+        k_consensus_partial<float, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
+            static_cast<const float*>(x), nullptr, pitch, n, d, 0.0, nullptr, partials);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+    k_consensus_final<<<1, kThreads, 0, stream>>>(partials, (int)blocks, out_device);
+    if (n_partials_out) *n_partials_out = (int)blocks;
+    return (int)cudaGetLastError();
+}
+
+int64_t consensus_static_max_columns(int32_t dtype) {
+    return (int64_t)kStaticMaxPartials * kStaticVecPerBlock * (dtype == A2_BF16 ? 8 : 4);
 }
 
 }  // namespace a2
