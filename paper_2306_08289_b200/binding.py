@@ -265,7 +265,7 @@ class Engine:
     stream only). x, x~ and the gradient buffer are torch tensors of shape [rows, pitch]."""
 
     def __init__(self, n, d, eta, alpha, alpha_tilde, gamma, storage="f32", n_grad_slots=None, device="cuda:0",
-                 stream=None):
+                 stream=None, rows_16B_only=False):
         import torch
 
         self.torch = torch
@@ -280,12 +280,20 @@ class Engine:
         _check(lib().a2cid2_create(self.n, self.d, eta, alpha, alpha_tilde, gamma, self.dtype_code, C.byref(h)))
         self._h = h
         self.device = torch.device(device)
-        self.pitch = (self.d + 7) // 8 * 8
+        # rows start on 32-byte boundaries so that the kernels can use 256-bit accesses
+        # (rows_16B_only: start them 16 bytes off instead, which is all the ABI requires)
+        q = 32 // self.elem_bytes
+        self.pitch = (self.d + q - 1) // q * q
+        shift = 16 // self.elem_bytes if rows_16B_only else 0
         self.n_slots = self.n if n_grad_slots is None else int(n_grad_slots)
         with torch.cuda.device(self.device):
-            self.x = torch.zeros((self.n, self.pitch), dtype=self.torch_dtype, device=self.device)
-            self.xt = torch.zeros((self.n, self.pitch), dtype=self.torch_dtype, device=self.device)
-            self.g = torch.zeros((max(self.n_slots, 1), self.pitch), dtype=self.torch_dtype, device=self.device)
+            def rows(r):
+                flat = torch.zeros(r * self.pitch + shift, dtype=self.torch_dtype, device=self.device)
+                return flat[shift:].view(r, self.pitch)
+
+            self.x = rows(self.n)
+            self.xt = rows(self.n)
+            self.g = rows(max(self.n_slots, 1))
             self.stream = torch.cuda.current_stream(self.device) if stream is None else stream
             _check(lib().a2cid2_bind(self._h, self.x.data_ptr(), self.xt.data_ptr(),
                                      self.g.data_ptr() if self.n_slots > 0 else None, self.n_slots, self.pitch,

@@ -88,7 +88,7 @@ struct EventLaunch {
 
 struct DeviceInfo {
     int sm_count = 0;
-    int event_ctas_per_sm[2] = {0, 0};  // per storage type
+    int event_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // [storage type][128-bit / 256-bit accesses]
     int consensus_ctas_per_sm = 0;
 };
 

@@ -29,6 +29,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdlib>
 #include <mutex>
 
 #include "a2cid2_internal.h"
@@ -40,40 +41,75 @@ namespace {
 constexpr int kThreads = 256;
 
 // ---------------------------------------------------------------------------------------------
-// 128-bit vector access for the two storage types. Vec<T>::N elements per 16 bytes.
+// Vector access for the two storage types: BYTES = 32 (256-bit ld/st.global.v8, the widest
+// sm_100 offers; needs 32-byte aligned rows) or 16 (128-bit, any row the ABI accepts).
+// Vec<T, BYTES>::N elements per access; streaming (evict-first) cache policy on both sides.
 // ---------------------------------------------------------------------------------------------
-template <typename T> struct Vec;
+__device__ __forceinline__ void ld_u32x4(const void* p, uint32_t (&w)[4]) {
+    const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
+    w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
+}
+__device__ __forceinline__ void st_u32x4(void* p, const uint32_t (&w)[4]) {
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+}
+__device__ __forceinline__ void ld_u32x8(const void* p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void st_u32x8(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
 
-template <> struct Vec<float> {
-    static constexpr int N = 4;
-    static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
-        const float4 q = __ldcs(reinterpret_cast<const float4*>(p));
-        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+template <int WORDS> struct Words;
+template <> struct Words<4> {
+    static __device__ __forceinline__ void ld(const void* p, uint32_t (&w)[4]) { ld_u32x4(p, w); }
+    static __device__ __forceinline__ void st(void* p, const uint32_t (&w)[4]) { st_u32x4(p, w); }
+};
+template <> struct Words<8> {
+    static __device__ __forceinline__ void ld(const void* p, uint32_t (&w)[8]) { ld_u32x8(p, w); }
+    static __device__ __forceinline__ void st(void* p, const uint32_t (&w)[8]) { st_u32x8(p, w); }
+};
+
+template <typename T, int BYTES> struct Vec;
+
+template <int BYTES> struct Vec<float, BYTES> {
+    static constexpr int N = BYTES / 4;
+    static __device__ __forceinline__ void load(const float* p, float (&v)[N]) {
+        uint32_t w[N];
+        Words<N>::ld(p, w);
+#pragma unroll
+        for (int k = 0; k < N; ++k) v[k] = __uint_as_float(w[k]);
     }
-    static __device__ __forceinline__ void store(float* p, const float (&v)[4]) {
-        __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
+    static __device__ __forceinline__ void store(float* p, const float (&v)[N]) {
+        uint32_t w[N];
+#pragma unroll
+        for (int k = 0; k < N; ++k) w[k] = __float_as_uint(v[k]);
+        Words<N>::st(p, w);
     }
 };
 
-template <> struct Vec<__nv_bfloat16> {
-    static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
-        const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+template <int BYTES> struct Vec<__nv_bfloat16, BYTES> {
+    static constexpr int N = BYTES / 2;
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[N]) {
+        uint32_t w[N / 2];
+        Words<N / 2>::ld(p, w);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {  // bf16 -> fp32 is a 16-bit shift
+        for (int k = 0; k < N / 2; ++k) {  // bf16 -> fp32 is a 16-bit shift
             v[2 * k] = __uint_as_float(w[k] << 16);
             v[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
         }
     }
-    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
-        uint32_t w[4];
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[N]) {
+        uint32_t w[N / 2];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {  // round to nearest even
+        for (int k = 0; k < N / 2; ++k) {  // round to nearest even
             const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
             w[k] = *reinterpret_cast<const uint32_t*>(&h);
         }
-        __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+        Words<N / 2>::st(p, w);
     }
 };
 
@@ -85,11 +121,23 @@ __device__ __forceinline__ void grad_elem(float& x, float& xt, float c, float ng
     xt = __fadd_rn(xt, __fmaf_rn(c, dlt, tg));
 }
 
-// Communication event on one element of workers a and b.
+// Communication event on one element of workers a and b. COMPENSATED carries the message as a
+// two-term sum (fp32 storage); with bf16 storage the store's own rounding is five orders of
+// magnitude larger than what the compensation recovers, so the plain difference is used.
+template <bool COMPENSATED>
 __device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, float& xtb, float ca, float cb,
                                           float alpha, float alpha_t, bool msg_before_mix) {
     const float ua = __fmul_rn(-ca, __fsub_rn(xa, xta));
     const float ub = __fmul_rn(-cb, __fsub_rn(xb, xtb));
+    if (!COMPENSATED) {
+        const float d0 = __fsub_rn(xa, xb);
+        const float m0 = msg_before_mix ? d0 : __fadd_rn(d0, __fsub_rn(ua, ub));
+        xa = __fadd_rn(xa, __fmaf_rn(-alpha, m0, ua));
+        xta = __fadd_rn(xta, __fmaf_rn(-alpha_t, m0, -ua));
+        xb = __fadd_rn(xb, __fmaf_rn(alpha, m0, ub));
+        xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m0, -ub));
+        return;
+    }
     // raw + e_raw == x_a - x_b exactly (two-sum)
     const float nb = -xb;
     const float raw = __fadd_rn(xa, nb);
@@ -131,9 +179,10 @@ struct EventArgs {
     int msg_before_mix;
 };
 
-template <typename T, int UNROLL>
+template <typename T, int BYTES, int UNROLL>
 __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
-    constexpr int N = Vec<T>::N;
+    using V = Vec<T, BYTES>;
+    constexpr int N = V::N;
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
     __shared__ float s_ca[kMaxOpsPerLaunch];
     __shared__ float s_cb[kMaxOpsPerLaunch];
@@ -178,14 +227,14 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
 #pragma unroll
             for (int k = 0; k < N; ++k) { xb[u][k] = 0.f; xtb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
             if (live[u]) {
-                Vec<T>::load(pxa + off, xa[u]);
-                Vec<T>::load(pxta + off, xta[u]);
+                V::load(pxa + off, xa[u]);
+                V::load(pxta + off, xta[u]);
                 if (has_b) {
-                    Vec<T>::load(pxb + off, xb[u]);
-                    Vec<T>::load(pxtb + off, xtb[u]);
+                    V::load(pxb + off, xb[u]);
+                    V::load(pxtb + off, xtb[u]);
                 }
-                if (has_ga) Vec<T>::load(pga + off, ga[u]);
-                if (has_gb) Vec<T>::load(pgb + off, gb[u]);
+                if (has_ga) V::load(pga + off, ga[u]);
+                if (has_gb) V::load(pgb + off, gb[u]);
             } else {
 #pragma unroll
                 for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xta[u][k] = 0.f; }
@@ -212,7 +261,8 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
                     for (int k = 0; k < N; ++k)
-                        comm_elem(xa[u][k], xta[u][k], xb[u][k], xtb[u][k], ca, cb, alpha, alpha_t, p.msg_before_mix != 0);
+                        comm_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], xb[u][k], xtb[u][k], ca, cb, alpha, alpha_t,
+                                                  p.msg_before_mix != 0);
             }
         }
 
@@ -220,29 +270,31 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
         for (int u = 0; u < UNROLL; ++u) {
             const long long off = (v0 + (long long)u * kThreads) * N;
             if (live[u]) {
-                Vec<T>::store(pxa + off, xa[u]);
-                Vec<T>::store(pxta + off, xta[u]);
+                V::store(pxa + off, xa[u]);
+                V::store(pxta + off, xta[u]);
                 if (has_b) {
-                    Vec<T>::store(pxb + off, xb[u]);
-                    Vec<T>::store(pxtb + off, xtb[u]);
+                    V::store(pxb + off, xb[u]);
+                    V::store(pxtb + off, xtb[u]);
                 }
             }
         }
     }
 }
 
-template <typename T> struct EventCfg;
-template <> struct EventCfg<float> { static constexpr int UNROLL = 2; };
-template <> struct EventCfg<__nv_bfloat16> { static constexpr int UNROLL = 1; };
+// Vectors per thread and tile. 256-bit accesses: one vector per thread already keeps 4-6 rows x 32 B
+// in flight per thread; 128-bit fp32 uses two.
+template <typename T, int BYTES> struct EventCfg { static constexpr int UNROLL = 1; };
+template <> struct EventCfg<float, 16> { static constexpr int UNROLL = 2; };
 
 // ---------------------------------------------------------------------------------------------
 // Consensus kernel
 // ---------------------------------------------------------------------------------------------
-template <typename T, bool FLUSH>
+template <typename T, int BYTES, bool FLUSH>
 __global__ void __launch_bounds__(kThreads) k_consensus_partial(const T* __restrict__ X, const T* __restrict__ Xt,
                                                               long long pitch, int n, long long d, double eta,
                                                               const double* __restrict__ dt, double* __restrict__ partials) {
-    constexpr int N = Vec<T>::N;
+    using V = Vec<T, BYTES>;
+    constexpr int N = V::N;
     extern __shared__ float s_c[];  // FLUSH: mixing coefficient of every worker to the common time
     __shared__ double s_warp[kThreads / 32];
     if (FLUSH) {
@@ -255,10 +307,10 @@ __global__ void __launch_bounds__(kThreads) k_consensus_partial(const T* __restr
     for (long long v = (long long)blockIdx.x * kThreads + threadIdx.x; v < n_vec; v += (long long)gridDim.x * kThreads) {
         const long long off = v * N;
         float first[N], s1[N], s2[N];
-        Vec<T>::load(X + off, first);
+        V::load(X + off, first);
         if (FLUSH) {
             float xt0[N];
-            Vec<T>::load(Xt + off, xt0);
+            V::load(Xt + off, xt0);
             const float c = s_c[0];
 #pragma unroll
             for (int k = 0; k < N; ++k) first[k] = __fmaf_rn(-c, __fsub_rn(first[k], xt0[k]), first[k]);
@@ -268,10 +320,10 @@ __global__ void __launch_bounds__(kThreads) k_consensus_partial(const T* __restr
 #pragma unroll 4
         for (int i = 1; i < n; ++i) {
             float xi[N];
-            Vec<T>::load(X + (long long)i * pitch + off, xi);
+            V::load(X + (long long)i * pitch + off, xi);
             if (FLUSH) {
                 float xti[N];
-                Vec<T>::load(Xt + (long long)i * pitch + off, xti);
+                V::load(Xt + (long long)i * pitch + off, xti);
                 const float c = s_c[i];
 #pragma unroll
                 for (int k = 0; k < N; ++k) xi[k] = __fmaf_rn(-c, __fsub_rn(xi[k], xti[k]), xi[k]);
@@ -317,10 +369,10 @@ __global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __re
     }
 }
 
-template <typename T>
+template <typename T, int BYTES>
 int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
-    constexpr int U = EventCfg<T>::UNROLL;
-    constexpr int N = Vec<T>::N;
+    constexpr int U = EventCfg<T, BYTES>::UNROLL;
+    constexpr int N = Vec<T, BYTES>::N;
     EventArgs a;
     a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
     a.n_vec = (L.d + N - 1) / N;
@@ -330,12 +382,51 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    const int per_sm = dev.event_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0];
+    const int per_sm = dev.event_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
     long long grid = (long long)dev.sm_count * per_sm;
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events<T, U><<<(unsigned)grid, kThreads, 0, stream>>>(a);
+    k_apply_events<T, BYTES, U><<<(unsigned)grid, kThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
+}
+
+// Resident CTAs per SM the persistent grid is sized for, measured on B200 with 64 rows of 25.6e6
+// columns. fp32 rows, fused ring batches, 256-bit accesses: 1 CTA/SM 5.13 TB/s, 2: 6.33, 3: 6.01,
+// 4: 5.97 -- beyond two CTAs the extra concurrent row streams cost more DRAM locality than the extra
+// loads in flight buy. bf16 rows do twice the arithmetic per byte and want more warps: 128-bit
+// accesses with 2 CTAs/SM 4.91 TB/s, 3: 5.81, 4: 5.84 (256-bit accesses, 127 registers: 5.45).
+template <typename T> struct EventCtas { static constexpr int PER_SM = 2; };
+template <> struct EventCtas<__nv_bfloat16> { static constexpr int PER_SM = 4; };
+
+template <typename T, int BYTES>
+cudaError_t event_occupancy(int* out) {
+    int occ = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL>, kThreads, 0);
+    *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
+    return e;
+}
+
+// 256-bit accesses are used for fp32 rows (bf16 rows are served better by 128-bit ones, see above) and
+// need every row start on a 32-byte boundary.
+bool rows_32B_aligned(const void* a, const void* b, const void* c, int64_t pitch, int32_t dtype) {
+    if (dtype == A2_BF16) return false;
+    static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+    if (force_narrow) return false;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c);
+    const int64_t pitch_bytes = pitch * (dtype == A2_BF16 ? 2 : 4);
+    return (bits % 32 == 0) && (pitch_bytes % 32 == 0);
+}
+
+template <typename T, int BYTES>
+void launch_consensus_partial_t(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, double eta,
+                                const double* dt, double* partials, int n_partials, cudaStream_t stream) {
+    const T* X = static_cast<const T*>(x);
+    const T* Xt = static_cast<const T*>(xt);
+    if (dt)
+        k_consensus_partial<T, BYTES, true><<<n_partials, kThreads, (size_t)n * sizeof(float), stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+    else
+        k_consensus_partial<T, BYTES, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
 }
 
 }  // namespace
@@ -346,22 +437,26 @@ int query_device(DeviceInfo* info) {
     if (e != cudaSuccess) return (int)e;
     e = cudaDeviceGetAttribute(&info->sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return (int)e;
-    int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events<float, EventCfg<float>::UNROLL>, kThreads, 0);
-    if (e != cudaSuccess) return (int)e;
-    info->event_ctas_per_sm[0] = occ > 0 ? occ : 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &occ, k_apply_events<__nv_bfloat16, EventCfg<__nv_bfloat16>::UNROLL>, kThreads, 0);
-    if (e != cudaSuccess) return (int)e;
-    info->event_ctas_per_sm[1] = occ > 0 ? occ : 1;
+    if ((e = event_occupancy<float, 16>(&info->event_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<float, 32>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<__nv_bfloat16, 16>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
+    info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
     info->consensus_ctas_per_sm = 4;
+    if (const char* v = std::getenv("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
+        const int k = std::atoi(v);
+        if (k > 0)
+            for (auto& row : info->event_ctas_per_sm)
+                for (int& c : row) c = k;
+    }
     return 0;
 }
 
-int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream) {
+int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.n_items <= 0) return 0;
-    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16>(L, dev, static_cast<cudaStream_t>(stream));
-    return launch_events_t<float>(L, dev, static_cast<cudaStream_t>(stream));
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
+    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16>(L, dev, stream);
+    return wide ? launch_events_t<float, 32>(L, dev, stream) : launch_events_t<float, 16>(L, dev, stream);
 }
 
 int consensus_grid(const DeviceInfo& dev) { return dev.sm_count * dev.consensus_ctas_per_sm; }
@@ -369,17 +464,12 @@ int consensus_grid(const DeviceInfo& dev) { return dev.sm_count * dev.consensus_
 int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double eta,
                      const double* dt, double* partials, int n_partials, double* out, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const size_t smem = dt ? (size_t)n * sizeof(float) : 0;
+    const bool wide = rows_32B_aligned(x, xt, nullptr, pitch, dtype);
     if (dtype == A2_BF16) {
-        const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(x);
-        const __nv_bfloat16* Xt = static_cast<const __nv_bfloat16*>(xt);
-        if (dt) k_consensus_partial<__nv_bfloat16, true><<<n_partials, kThreads, smem, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
-        else k_consensus_partial<__nv_bfloat16, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+        launch_consensus_partial_t<__nv_bfloat16, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
     } else {
-        const float* X = static_cast<const float*>(x);
-        const float* Xt = static_cast<const float*>(xt);
-        if (dt) k_consensus_partial<float, true><<<n_partials, kThreads, smem, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
-        else k_consensus_partial<float, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+        if (wide) launch_consensus_partial_t<float, 32>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
+        else launch_consensus_partial_t<float, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
@@ -430,10 +520,10 @@ int launch_consensus_static(const void* x, int64_t pitch, int32_t n, int64_t d, 
     // every block overwrites its own partial and the final pass reads exactly `blocks` of them,
     // so nothing left in the array by an earlier call is ever read
     if (dtype == A2_BF16)
-        k_consensus_partial<__nv_bfloat16, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
+        k_consensus_partial<__nv_bfloat16, 16, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
             static_cast<const __nv_bfloat16*>(x), nullptr, pitch, n, d, 0.0, nullptr, partials);
     else
-        k_consensus_partial<float, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
+        k_consensus_partial<float, 16, false><<<(unsigned)blocks, kThreads, 0, stream>>>(
             static_cast<const float*>(x), nullptr, pitch, n, d, 0.0, nullptr, partials);
     e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;

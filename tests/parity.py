@@ -32,7 +32,7 @@ TOL = {"f32": 1e-5, "bf16": 2e-2}
 BF16_ELEM_STORED_BOUND = 5e-2
 BF16_ELEM_PLAIN_BOUND = 0.3
 BF16_NORM_MIN_COLS = 256
-TILE_COLS = {"f32": 256 * 2 * 4, "bf16": 256 * 1 * 8}  # columns per work unit of the event kernel
+TILE_COLS = {"f32": 256 * 8, "bf16": 256 * 8}  # columns per work unit of the event kernel
 
 
 def rel_err(gpu, ref):

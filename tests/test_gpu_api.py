@@ -27,7 +27,7 @@ def test_state_round_trip_and_padding(storage):
     xs, _ = W.x0_matrix(cfg)
     gs, _ = W.grad_matrix(cfg)
     eng = B.Engine(cfg.n, cfg.d, 0.3, 0.5, 1.1, 0.1, storage=storage)
-    assert eng.pitch == 1008
+    assert eng.pitch == (1008 if storage == "f32" else 1008)
     eng.write_state(xs)
     x, xt, t = eng.read_state()
     assert np.array_equal(x, xs) and np.array_equal(xt, xs) and np.array_equal(t, np.zeros(cfg.n))
@@ -179,6 +179,29 @@ def test_bind_rejects_bad_buffers():
                                  i0.ctypes.data_as(ip), 0, None) == B.A2_ERANGE  # gradient event without slots
     assert L.a2cid2_sync(h) == B.A2_OK
     L.a2cid2_destroy(h)
+
+
+@pytest.mark.parametrize("storage", ["f32", "bf16"])
+def test_rows_aligned_to_16_bytes_only_take_the_128_bit_kernels(storage):
+    """Rows on 32-byte boundaries run the 256-bit kernels, rows that are only 16-byte aligned the
+    128-bit ones; the arithmetic per element is the same, so the states agree bit for bit."""
+    cfg = _small(storage, d=5_003, n_events=600)
+    ev = W.config_events(cfg)
+    xs, _ = W.x0_matrix(cfg)
+    gs, _ = W.grad_matrix(cfg)
+    outs = []
+    for narrow in (False, True):
+        eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=storage, rows_16B_only=narrow)
+        assert (eng.x.data_ptr() % 32 == 16) == narrow
+        eng.write_state(xs)
+        eng.write_grads(gs)
+        eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+        t_eval = float(ev.times[-1]) + 0.5
+        outs.append((eng.read_state(), eng.consensus_distance(), eng.consensus_distance(t_eval)))
+        eng.close()
+    (a, ca, cfa), (b, cb, cfb) = outs
+    assert all(np.array_equal(u, v) for u, v in zip(a, b))
+    assert abs(ca - cb) <= 1e-9 * ca and abs(cfa - cfb) <= 1e-9 * cfa
 
 
 def test_non_default_stream():
