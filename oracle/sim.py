@@ -14,10 +14,10 @@ from . import build as _build
 _lib = None
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        L = C.CDLL(_build.build())
+def load(path):
+    """Load a build of the C checker and declare its signatures."""
+    if True:
+        L = C.CDLL(path)
         dp, ip = C.POINTER(C.c_double), C.POINTER(C.c_int32)
         L.a2o_mix_coeff.restype = C.c_double
         L.a2o_mix_coeff.argtypes = [C.c_double, C.c_double]
@@ -29,7 +29,13 @@ def lib():
         L.a2o_consensus.argtypes = [C.c_int32, C.c_int64, C.c_int64, dp]
         L.a2o_consensus_at.restype = C.c_double
         L.a2o_consensus_at.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_double, dp, dp, dp, C.c_double]
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = load(_build.build())
     return _lib
 
 

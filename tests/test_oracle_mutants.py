@@ -1,0 +1,79 @@
+"""Do the pins bite? Plausible mistakes are planted in copies of the C checker (on the CPU, in a
+temporary directory): a dropped term, a wrong sign, swapped coefficients, a wrong index. For each
+mutant at least one of the pins in test_oracle_pins.py must fail."""
+import os
+import subprocess
+
+import pytest
+
+import oracle.sim as sim_mod
+from oracle import build as obuild
+from tests import test_oracle_pins as pins
+
+MUTANTS = {
+    "mix_sign": ("xt[k] = xt[k] + c * dlt;", "xt[k] = xt[k] - c * dlt;"),
+    "mix_rate": ("return -expm1(-2.0 * eta * dt) / 2.0;", "return -expm1(-1.0 * eta * dt) / 2.0;"),
+    "mix_no_half": ("return -expm1(-2.0 * eta * dt) / 2.0;", "return -expm1(-2.0 * eta * dt);"),
+    "grad_only_x": ("xti[k] = xti[k] - gamma * g[k];", "xti[k] = xti[k];"),
+    "grad_sign": ("xi[k] = xi[k] - gamma * g[k];", "xi[k] = xi[k] + gamma * g[k];"),
+    "grad_no_mix": ("a2o_mix(xi, xti, d, eta, t - tl[i]);\n            for (int64_t k = 0; k < d; ++k) {\n                xi[k] = xi[k] - gamma",
+                    "for (int64_t k = 0; k < d; ++k) {\n                xi[k] = xi[k] - gamma"),
+    "comm_j_sign": ("xj[k] = xj[k] + alpha * m;\n                    xtj[k] = xtj[k] + alpha_t * m;\n                }\n            } else {",
+                    "xj[k] = xj[k] - alpha * m;\n                    xtj[k] = xtj[k] + alpha_t * m;\n                }\n            } else {"),
+    "comm_swapped_coeffs": ("xi[k] = xi[k] - alpha * m;\n                    xti[k] = xti[k] - alpha_t * m;\n                    xj[k] = xj[k] + alpha * m;",
+                            "xi[k] = xi[k] - alpha_t * m;\n                    xti[k] = xti[k] - alpha * m;\n                    xj[k] = xj[k] + alpha * m;"),
+    "comm_tilde_uses_own_difference": ("const double m = xi[k] - xj[k];\n                    xi[k] = xi[k] - alpha * m;\n                    xti[k] = xti[k] - alpha_t * m;",
+                                       "const double m = xi[k] - xj[k];\n                    xi[k] = xi[k] - alpha * m;\n                    xti[k] = xti[k] - alpha_t * (xti[k] - xtj[k]);"),
+    "comm_mixes_one_worker": ("a2o_mix(xj, xtj, d, eta, t - tl[j]);\n                for", "for"),
+    "comm_forgets_time_j": ("tl[i] = t;\n            tl[j] = t;", "tl[i] = t;"),
+    "grad_forgets_time": ("xti[k] = xti[k] - gamma * g[k];\n            }\n            tl[i] = t;", "xti[k] = xti[k] - gamma * g[k];\n            }"),
+    "wrong_gradient_row": ("const double* g = G + (size_t)s * ldg;", "const double* g = G + (size_t)i * ldg;"),
+    "consensus_not_centred": ("mean /= (double)n;\n        for (int32_t i = 0; i < n; ++i) {\n            const double dev = X[(size_t)i * ld + k] - mean;",
+                              "mean /= (double)(n + 1);\n        for (int32_t i = 0; i < n; ++i) {\n            const double dev = X[(size_t)i * ld + k] - mean;"),
+    "consensus_at_ignores_flow": ("mean += x - c * (x - xt);", "mean += x;"),
+}
+
+# pins that take the simulator class, and pins that use OracleSim directly
+DETECTORS = [
+    lambda: pins.test_mixing_keeps_half_sum_and_shrinks_difference(pins.OracleSim),
+    lambda: pins.test_mixing_semigroup(pins.OracleSim),
+    lambda: pins.test_mixing_matches_series_of_the_generator(),
+    lambda: pins.test_comm_keeps_population_sums(pins.OracleSim),
+    lambda: pins.test_comm_consensus_drop_identity(0.3),
+    lambda: pins.test_two_workers_reach_exact_consensus_in_one_event(pins.OracleSim),
+    lambda: pins.test_baseline_equals_textbook_gossip_sgd(pins.OracleSim),
+    lambda: pins.test_mean_tracker_identity(),
+    lambda: pins.test_brute_force_matrix_exponential(pins.OracleSim, 3, 3, "complete"),
+    lambda: pins.test_consensus_at_common_time_matches_flushed_state_and_definition(),
+    lambda: pins.test_hand_example(pins.OracleSim),
+]
+
+
+def _caught():
+    failed = []
+    for k, det in enumerate(DETECTORS):
+        try:
+            det()
+        except (AssertionError, sim_mod.OracleError):
+            failed.append(k)
+    return failed
+
+
+def test_unmutated_checker_passes_every_detector():
+    assert _caught() == []
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
+    old, new = MUTANTS[name]
+    src = open(obuild.SRC).read()
+    assert src.count(old) >= 1, f"mutation site for {name} not found"
+    mutated = src.replace(old, new, 1)
+    c = tmp_path / "mutant.c"
+    so = tmp_path / "mutant.so"
+    c.write_text(mutated)
+    subprocess.run(["gcc", "-O1", "-std=c99", "-ffp-contract=off", "-fPIC", "-shared", "-o", str(so), str(c), "-lm"],
+                   check=True)
+    monkeypatch.setattr(sim_mod, "_lib", sim_mod.load(str(so)))
+    caught = _caught()
+    assert caught, f"no pin noticed the planted mistake '{name}'"
