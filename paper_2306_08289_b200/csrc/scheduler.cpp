@@ -37,10 +37,11 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     if (n < 2) { err = "need n >= 2 workers"; return A2_EINVAL; }
     if (n_grad_slots < 0 || n_events < 0) { err = "negative size"; return A2_EINVAL; }
     if (n_events > 0 && (!times || !wi || !wj || !slot)) { err = "event arrays are NULL"; return A2_EINVAL; }
-    if (flags & ~uint32_t(A2_SCHED_FUSE)) { err = "unknown scheduling flag"; return A2_EINVAL; }
+    if (flags & ~uint32_t(A2_SCHED_FUSE | A2_SCHED_RESIDENT)) { err = "unknown scheduling flag"; return A2_EINVAL; }
     if (max_ops_per_item <= 0) max_ops_per_item = kDefaultMaxOpsPerItem;
     if (max_ops_per_item > kMaxOpsPerLaunch) max_ops_per_item = kMaxOpsPerLaunch;
-    const bool fuse = (flags & A2_SCHED_FUSE) != 0 && max_ops_per_item >= 2;
+    const bool resident = (flags & A2_SCHED_RESIDENT) != 0;
+    const bool fuse = !resident && (flags & A2_SCHED_FUSE) != 0 && max_ops_per_item >= 2;
 
     a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
     if (!s) { err = "out of host memory"; return A2_ENOMEM; }
@@ -161,6 +162,8 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             }
         }
         if (fuse) for (int32_t w = 0; w < n; ++w) flush(w);
+        if (resident)  // one batch, every event in stream order (items were created in that order)
+            for (SchedItem& it : items) it.batch = 0;
 
         // ---- order items by batch (stable) and lay the ops out in item order ----------------
         int32_t n_batches = 0;
@@ -185,6 +188,35 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     }
     *out = s;
     return A2_OK;
+}
+
+// Resident mode: cut the stream into chunks whose distinct gradient rows fit `capacity` cache rows.
+// Inside a chunk a gradient row keeps the cache index it was given at first use.
+void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResChunk>& chunks,
+                           std::vector<int32_t>& g_rows, std::vector<int32_t>& cache_idx) {
+    chunks.clear();
+    g_rows.clear();
+    cache_idx.assign(s.items.size(), -1);
+    std::vector<int32_t> where((size_t)std::max(1, s.n_grad_slots), -1);  // slot -> cache index in the open chunk
+    ResChunk cur{0, 0, 0, 0};
+    auto close = [&](int32_t ev_end) {
+        cur.ev_end = ev_end;
+        if (cur.ev_end > cur.ev_begin) chunks.push_back(cur);
+        for (int32_t k = cur.g_begin; k < cur.g_begin + cur.g_count; ++k) where[(size_t)g_rows[(size_t)k]] = -1;
+        cur = ResChunk{ev_end, ev_end, (int32_t)g_rows.size(), 0};
+    };
+    for (size_t e = 0; e < s.items.size(); ++e) {
+        const int32_t slot = s.items[e].slot_a;
+        if (slot < 0) continue;
+        if (where[(size_t)slot] < 0) {
+            if (cur.g_count == capacity) close((int32_t)e);
+            where[(size_t)slot] = cur.g_count;
+            g_rows.push_back(slot);
+            cur.g_count += 1;
+        }
+        cache_idx[e] = where[(size_t)slot];
+    }
+    close((int32_t)s.items.size());
 }
 
 void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {
