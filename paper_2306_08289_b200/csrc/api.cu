@@ -74,14 +74,26 @@ struct a2cid2 {
     std::string err;
 };
 
+// How a schedule is laid out in one descriptor blob, and how it is launched.
+struct Packed {
+    size_t bytes = 0;    // whole blob
+    size_t ops_off = 0;  // DevOp array (the DevItem array sits at offset 0)
+    // batched mode
+    std::vector<LaunchRange> launches;
+    std::vector<int64_t> batch_launch_first;  // launches of batch b: [first[b], first[b+1])
+    // resident mode
+    bool resident = false;
+    int32_t cache_rows = 0;
+    size_t chunks_off = 0, g_rows_off = 0, events_off = 0;
+    std::vector<a2::ResChunk> chunks;
+    std::vector<int32_t> g_rows, cache_idx;
+};
+
 struct a2cid2_plan {
     a2cid2* owner = nullptr;
     a2cid2_sched* sched = nullptr;
-    void* d_desc = nullptr;  // items then ops
-    DevItem* d_items = nullptr;
-    DevOp* d_ops = nullptr;
-    std::vector<LaunchRange> launches;
-    std::vector<int64_t> batch_launch_first;  // launches of batch b: [first[b], first[b+1])
+    void* d_desc = nullptr;  // the descriptor blob on the device
+    Packed pk;
     int64_t next_batch = 0;
     bool uses_gradients = false;
     std::vector<double> t_expect;  // workers' times the next batch expects
@@ -147,33 +159,84 @@ void make_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches, st
     batch_first[(size_t)nb] = (int64_t)launches.size();
 }
 
-size_t desc_bytes(const a2cid2_sched& s) {
-    const size_t items = (s.items.size() * sizeof(DevItem) + 15) & ~size_t(15);
-    return items + s.ops.size() * sizeof(DevOp);
+size_t align16(size_t v) { return (v + 15) & ~size_t(15); }
+
+// Decide how the schedule is launched and lay its descriptors out. Resident schedules need the
+// population to fit shared memory.
+int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
+    pk.resident = (s.flags & A2_SCHED_RESIDENT) != 0;
+    pk.ops_off = align16(s.items.size() * sizeof(DevItem));
+    size_t end = pk.ops_off + s.ops.size() * sizeof(DevOp);
+    if (!pk.resident) {
+        make_launches(s, pk.launches, pk.batch_launch_first);
+    } else {
+        pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
+        if (pk.cache_rows <= 0)
+            return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT: the population does not fit shared memory (need 2 n + 16 <= 216)");
+        a2::build_resident_chunks(s, pk.cache_rows, pk.chunks, pk.g_rows, pk.cache_idx);
+        pk.chunks_off = align16(end);
+        pk.g_rows_off = align16(pk.chunks_off + pk.chunks.size() * sizeof(a2::ResChunk));
+        pk.events_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(int32_t));
+        end = pk.events_off + s.items.size() * sizeof(a2::ResEv);  // this part is written on the device
+    }
+    pk.bytes = s.items.empty() ? 0 : end;
+    return A2_OK;
 }
 
-// Write device descriptors into `dst` (items, then ops at the 16-byte aligned offset returned).
-size_t pack_descriptors(const a2cid2_sched& s, const std::vector<LaunchRange>& launches, void* dst) {
+// Bytes of the blob that have to be copied to the device (the resident event records at its end are
+// produced there).
+size_t upload_bytes(const a2cid2_sched& s, const Packed& pk) {
+    if (s.items.empty()) return 0;
+    return pk.resident ? pk.events_off : pk.bytes;
+}
+
+void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
     DevItem* di = static_cast<DevItem*>(dst);
-    const size_t ops_off = (s.items.size() * sizeof(DevItem) + 15) & ~size_t(15);
-    DevOp* dop = reinterpret_cast<DevOp*>(static_cast<char*>(dst) + ops_off);
-    for (const LaunchRange& L : launches) {
-        for (int64_t k = L.item0; k < L.item1; ++k) {
-            const a2::SchedItem& it = s.items[(size_t)k];
-            di[k] = DevItem{it.a, it.b, it.slot_a, it.slot_b, (int32_t)(it.first_op - L.op0), it.n_ops};
+    DevOp* dop = reinterpret_cast<DevOp*>(static_cast<char*>(dst) + pk.ops_off);
+    if (!pk.resident) {
+        for (const LaunchRange& L : pk.launches)
+            for (int64_t k = L.item0; k < L.item1; ++k) {
+                const a2::SchedItem& it = s.items[(size_t)k];
+                di[k] = DevItem{it.a, it.b, it.slot_a, it.slot_b, (int32_t)(it.first_op - L.op0), it.n_ops};
+            }
+    } else {
+        for (size_t k = 0; k < s.items.size(); ++k) {  // one operation per item; slot_b carries the cache index
+            const a2::SchedItem& it = s.items[k];
+            di[k] = DevItem{it.a, it.b, it.slot_a, pk.cache_idx[k], (int32_t)k, 1};
         }
+        if (!pk.chunks.empty())
+            std::memcpy(static_cast<char*>(dst) + pk.chunks_off, pk.chunks.data(), pk.chunks.size() * sizeof(a2::ResChunk));
+        if (!pk.g_rows.empty())
+            std::memcpy(static_cast<char*>(dst) + pk.g_rows_off, pk.g_rows.data(), pk.g_rows.size() * sizeof(int32_t));
     }
     for (size_t o = 0; o < s.ops.size(); ++o) {
         const a2::SchedOp& op = s.ops[o];
         dop[o] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
     }
-    return ops_off;
 }
 
-int queue_launches(a2cid2* h, const std::vector<LaunchRange>& launches, int64_t l0, int64_t l1, const DevItem* d_items,
-                   const DevOp* d_ops) {
-    for (int64_t l = l0; l < l1; ++l) {
-        const LaunchRange& R = launches[(size_t)l];
+// Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
+int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev, int64_t b0, int64_t b1) {
+    if (b1 <= b0) return A2_OK;
+    char* base = static_cast<char*>(dev);
+    const DevItem* d_items = reinterpret_cast<const DevItem*>(base);
+    const DevOp* d_ops = reinterpret_cast<const DevOp*>(base + pk.ops_off);
+    if (pk.resident) {
+        a2::ResidentLaunch L;
+        L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
+        L.n = h->n; L.dtype = h->dtype; L.variant = h->variant; L.eta = h->eta;
+        L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
+        L.items = d_items; L.ops = d_ops;
+        L.events = reinterpret_cast<a2::ResEv*>(base + pk.events_off);
+        L.chunks = reinterpret_cast<const a2::ResChunk*>(base + pk.chunks_off);
+        L.g_rows = reinterpret_cast<const int32_t*>(base + pk.g_rows_off);
+        L.n_events = (int32_t)s.items.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
+        const int rc = a2::launch_resident(L, h->dev, h->stream);
+        if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
+        return A2_OK;
+    }
+    for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
+        const LaunchRange& R = pk.launches[(size_t)l];
         a2::EventLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.items = d_items + R.item0;
@@ -187,6 +250,18 @@ int queue_launches(a2cid2* h, const std::vector<LaunchRange>& launches, int64_t 
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
     return A2_OK;
+}
+
+// Descriptor-derived counters of batches [b0, b1).
+void fill_stats(const a2cid2* h, const a2cid2_sched& s, const Packed& pk, int64_t b0, int64_t b1, a2cid2_stats* st) {
+    const int32_t eb = (int32_t)elem_bytes(h->dtype);
+    a2::schedule_stats(s, b0, b1, h->d, eb, st);
+    if (pk.resident) {  // the state crosses HBM once each way, every cached gradient row once per chunk
+        st->n_launches = b1 > b0 ? 2 : 0;
+        st->bytes_moved = b1 > b0 ? ((int64_t)4 * h->n + (int64_t)pk.g_rows.size()) * h->d * eb : 0;
+    } else {
+        st->n_launches = pk.batch_launch_first[(size_t)b1] - pk.batch_launch_first[(size_t)b0];
+    }
 }
 
 // After batches [b0, b1) ran: every worker's time is that of its last operation in them.
@@ -333,13 +408,12 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
     std::string err;
     rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
-    std::vector<LaunchRange> launches;
-    std::vector<int64_t> batch_first;
-    make_launches(*s, launches, batch_first);
+    Packed pk;
+    rc = plan_layout(h, *s, pk);
+    if (rc != A2_OK) { a2cid2_sched_destroy(s); return rc; }
     const int64_t nb = (int64_t)s->batch_first.size() - 1;
-    const size_t bytes = desc_bytes(*s);
     if (stats) std::memset(stats, 0, sizeof *stats);
-    if (bytes > 0) {
+    if (pk.bytes > 0) {
         Arena& A = h->arena[h->arena_next];
         h->arena_next ^= 1;
         if (A.in_flight) {  // the previous copy out of this staging buffer must have finished
@@ -347,33 +421,32 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
             if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "cudaEventSynchronize"); }
             A.in_flight = false;
         }
-        if (A.cap < bytes) {
+        if (A.cap < pk.bytes) {
             // the device side may still be read by queued kernels: wait before freeing it
             cudaError_t e = cudaStreamSynchronize(h->stream);
             if (e == cudaSuccess && A.host) e = cudaFreeHost(A.host);
             if (e == cudaSuccess && A.dev) e = cudaFree(A.dev);
             A.host = A.dev = nullptr;
             A.cap = 0;
-            const size_t cap = bytes + bytes / 2 + 4096;
+            const size_t cap = pk.bytes + pk.bytes / 2 + 4096;
             if (e == cudaSuccess) e = cudaMallocHost(&A.host, cap);
             if (e == cudaSuccess) e = cudaMalloc(&A.dev, cap);
             if (e == cudaSuccess && !A.copied) e = cudaEventCreateWithFlags(&A.copied, cudaEventDisableTiming);
             if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "descriptor buffer allocation"); }
             A.cap = cap;
         }
-        const size_t ops_off = pack_descriptors(*s, launches, A.host);
-        cudaError_t e = cudaMemcpyAsync(A.dev, A.host, bytes, cudaMemcpyHostToDevice, h->stream);
+        write_descriptors(*s, pk, A.host);
+        const size_t up = upload_bytes(*s, pk);
+        cudaError_t e = cudaMemcpyAsync(A.dev, A.host, up, cudaMemcpyHostToDevice, h->stream);
         if (e == cudaSuccess) e = cudaEventRecord(A.copied, h->stream);
         if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "descriptor upload"); }
         A.in_flight = true;
         const double t1 = now_ms();
-        rc = queue_launches(h, launches, 0, (int64_t)launches.size(), static_cast<const DevItem*>(A.dev),
-                            reinterpret_cast<const DevOp*>(static_cast<const char*>(A.dev) + ops_off));
+        rc = queue_batches(h, *s, pk, A.dev, 0, nb);
         if (rc != A2_OK) { a2cid2_sched_destroy(s); return rc; }
         if (stats) {
-            a2::schedule_stats(*s, 0, nb, h->d, (int32_t)elem_bytes(h->dtype), stats);
-            stats->n_launches = (int64_t)launches.size();
-            stats->descriptor_bytes = (int64_t)bytes;
+            fill_stats(h, *s, pk, 0, nb, stats);
+            stats->descriptor_bytes = (int64_t)up;
             stats->host_ms = t1 - t0;
         }
     }
@@ -471,22 +544,21 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
     p->sched = s;
     p->t_expect = s->t_start;
     p->uses_gradients = needs_gradients(*s);
-    make_launches(*s, p->launches, p->batch_launch_first);
-    const size_t bytes = desc_bytes(*s);
-    if (bytes > 0) {
-        std::vector<char> staging(bytes);
-        const size_t ops_off = pack_descriptors(*s, p->launches, staging.data());
-        cudaError_t e = cudaMalloc(&p->d_desc, bytes);
+    rc = plan_layout(h, *s, p->pk);
+    if (rc != A2_OK) { a2cid2_sched_destroy(s); delete p; return rc; }
+    if (p->pk.bytes > 0) {
+        const size_t up = upload_bytes(*s, p->pk);
+        std::vector<char> staging(up);
+        write_descriptors(*s, p->pk, staging.data());
+        cudaError_t e = cudaMalloc(&p->d_desc, p->pk.bytes);
         // pageable source: the copy has left the host buffer when the call returns
-        if (e == cudaSuccess) e = cudaMemcpy(p->d_desc, staging.data(), bytes, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_desc, staging.data(), up, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) {
             if (p->d_desc) cudaFree(p->d_desc);
             a2cid2_sched_destroy(s);
             delete p;
             return fail_cuda(h, e, "plan descriptor upload");
         }
-        p->d_items = static_cast<DevItem*>(p->d_desc);
-        p->d_ops = reinterpret_cast<DevOp*>(static_cast<char*>(p->d_desc) + ops_off);
     }
     h->live_plans += 1;
     *out = p;
@@ -507,16 +579,14 @@ int a2cid2_plan_run(a2cid2_t* h, a2cid2_plan_t* p, int64_t first_batch, int64_t 
     if (p->uses_gradients && !h->g) return fail(h, A2_ESTATE, "plan has gradient events but no gradient buffer is bound");
     const int64_t b1 = first_batch + n_batches;
     if (n_batches > 0) {
-        rc = queue_launches(h, p->launches, p->batch_launch_first[(size_t)first_batch], p->batch_launch_first[(size_t)b1],
-                            p->d_items, p->d_ops);
+        rc = queue_batches(h, *p->sched, p->pk, p->d_desc, first_batch, b1);
         if (rc != A2_OK) return rc;
         advance_times(*p->sched, first_batch, b1, h->t);
     }
     p->next_batch = b1;
     p->t_expect = h->t;
     if (stats) {
-        a2::schedule_stats(*p->sched, first_batch, b1, h->d, (int32_t)elem_bytes(h->dtype), stats);
-        stats->n_launches = p->batch_launch_first[(size_t)b1] - p->batch_launch_first[(size_t)first_batch];
+        fill_stats(h, *p->sched, p->pk, first_batch, b1, stats);
         stats->descriptor_bytes = 0;
         stats->host_ms = 0.0;
     }
