@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(HERE, "liba2cid2.so")
 A2_OK, A2_EINVAL, A2_EORDER, A2_ERANGE, A2_ENOMEM, A2_ECUDA, A2_ESTATE = 0, -1, -2, -3, -4, -5, -6
 A2_F32, A2_BF16 = 0, 1
 A2_SCHED_FUSE = 1
+A2_SCHED_RESIDENT = 2
 A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM = 0, 1, 2
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX = 0, 1
 

@@ -114,3 +114,64 @@ def test_exact_consensus_is_zero():
     eng.write_state(np.tile(row, (4, 1)))
     assert eng.consensus_distance() == 0.0
     eng.close()
+
+
+# ---- resident mode: one launch per call, the population's column tile kept in shared memory ----
+@pytest.mark.parametrize("name,d,n_events", [
+    ("cfg1", 10_000, 2000),  # 4 workers, pool of 16 gradient rows per worker: fits one cache fill
+    ("cfg2", 5_003, 6000),   # 16 workers x 128 rows: the cache is refilled chunk by chunk
+    ("cfg4", 4_097, 3000),   # 64 workers: one CTA per SM
+])
+def test_resident_mode_is_bit_identical_to_batches_fp32(name, d, n_events):
+    """Same per-element operations in the same per-worker order, so fp32 states agree bit for bit."""
+    cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
+    ev = W.config_events(cfg)
+    states = []
+    for flags in (B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
+        eng, chk = P.make_small(cfg)
+        for lo in range(0, len(ev), 777):  # several calls, so that resident calls chain on stored state
+            c = ev.slice(lo, lo + 777)
+            st = eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=flags, want_stats=True)
+            if flags == B.A2_SCHED_RESIDENT:
+                assert st["n_launches"] == 2 and st["n_batches"] == 1
+                chk.plain.apply_stream(c)
+                x, xt, t = eng.read_state()
+                chk.compare(P.widen(x, "f32"), P.widen(xt, "f32"), t, where=f"resident {name} after event {lo + len(c)}")
+        states.append(eng.read_state())
+        eng.close()
+    assert all(np.array_equal(u, v) for u, v in zip(states[0], states[1]))
+
+
+def test_resident_mode_bf16_storage():
+    cfg = W.CONFIGS["cfg5"].scaled(d=6_151, n_events=3000)
+    ev = W.config_events(cfg)
+    eng, chk = P.make_small(cfg)
+    for lo in range(0, len(ev), 500):
+        c = ev.slice(lo, lo + 500)
+        eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=B.A2_SCHED_RESIDENT)
+        chk.plain.apply_stream(c)
+        chk.stored.apply_stream(c)  # the tile is held in fp32 during a call and rounded at its end
+        chk.stored.round_rows(np.arange(cfg.n))
+        x, xt, t = eng.read_state()
+        chk.compare(P.widen(x, "bf16"), P.widen(xt, "bf16"), t, where=f"resident bf16 after event {lo + len(c)}")
+    eng.close()
+
+
+def test_resident_mode_plan_variant_and_limits():
+    cfg = W.CONFIGS["cfg3"].scaled(d=2_050, n_events=1200)
+    ev = W.config_events(cfg)
+    eng, chk = P.make_small(cfg, variant=B.A2_MSG_BEFORE_MIX)
+    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_RESIDENT)
+    assert p.sched.num_batches == 1
+    p.run()
+    p.close()
+    chk.plain.apply_stream(ev)
+    x, xt, t = eng.read_state()
+    chk.compare(P.widen(x, "f32"), P.widen(xt, "f32"), t, where="resident, message before mix")
+    eng.close()
+    big = B.Engine(120, 64, 0.1, 0.5, 0.5, 0.1)  # 2 * 120 rows of shared memory are too many
+    with pytest.raises(B.A2Error) as e:
+        big.apply_events([1.0], [0], [1], [-1], flags=B.A2_SCHED_RESIDENT)
+    assert e.value.code == B.A2_EINVAL and "shared memory" in str(e.value)
+    big.apply_events([1.0], [0], [1], [-1])  # the batched path takes any n
+    big.close()
