@@ -61,6 +61,7 @@ def parse_args():
     ap.add_argument("--no-fuse", action="store_true", help="one event per item (no gradient fusion)")
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-resident-mode", action="store_true")
     return ap.parse_args()
 
 
@@ -241,7 +242,8 @@ def main():
     eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
                    device=str(device))
     fill_engine(eng, cfg, threads)
-    ev_all = W.config_events(cfg, n_events=2 * n_steps * eps)  # first half: resident pass; second: end to end
+    # three stretches of the stream: plans resident on the device, end to end, shared-memory-resident mode
+    ev_all = W.config_events(cfg, n_events=3 * n_steps * eps)
 
     # ---- pass 1: descriptors resident on the device ---------------------------------------------
     plans, t_start = [], np.zeros(cfg.n)
@@ -304,6 +306,41 @@ def main():
     if not all(np.isfinite(cons)):
         raise SystemExit("non-finite consensus distance: the run is invalid")
 
+    # ---- pass 3: the shared-memory-resident mode (one launch per step), reported beside the main figure ---
+    resident = None
+    if not args.skip_resident_mode:
+        try:
+            r_plans, t_start = [], eng.times()
+            for s in range(n_steps):
+                c = ev_all.slice((2 * n_steps + s) * eps, (2 * n_steps + s + 1) * eps)
+                p = eng.plan(c.times, c.wi, c.wj, c.slot, flags=B.A2_SCHED_RESIDENT, t_start=t_start)
+                t_start = p.sched.t_final(cfg.n)
+                r_plans.append(p)
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            r_bytes = 0
+            for s in range(n_steps):
+                if s == W_:
+                    torch.cuda.synchronize(device)
+                    ranks.barrier()
+                    r0.record(stream)
+                st = r_plans[s].run(want_stats=True)
+                cons.append(eng.consensus_distance())
+                if s >= W_:
+                    r_bytes += st["bytes_moved"]
+            r1.record(stream)
+            torch.cuda.synchronize(device)
+            ranks.barrier()
+            r_ms = r0.elapsed_time(r1)
+            for p in r_plans:
+                p.close()
+            r_value, r_slow = aggregate_throughput(ranks, K * eps, r_ms / 1e3)
+            resident = {"value": r_value, "unit": "events/s", "ms_per_step": 1e3 * r_slow / K,
+                        "hbm_gbs": r_bytes / (r_ms / 1e3) / 1e9,
+                        "note": "A2_SCHED_RESIDENT: one launch per step, column tile of all workers in shared "
+                                "memory; needs every gradient of the step up front; not HBM-bound"}
+        except B.A2Error as exc:
+            resident = {"unavailable": str(exc)}
+
     # ---- roofline of the event kernel ------------------------------------------------------------
     peak, peak_src = measured_peak()
     achieved = k1_bytes / (k1_ms / 1e3) / 1e9
@@ -334,6 +371,7 @@ def main():
         "gpu_launches": int(k1_launches + 2 * K),
         "consensus_kernel": {"ms": k2_ms / K, "gbs": consensus_gbs, "frac": consensus_gbs / peak},
         "batches_per_step": sum(stats[s]["n_batches"] for s in timed) / K,
+        "resident_mode": resident,
     }
 
     if ranks.rank == 0 and ranks.world == 1 and not args.skip_cpu_baseline:
