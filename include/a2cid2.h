@@ -68,7 +68,7 @@ enum {
                               a CTA the batches are separated by an ordinary block barrier. Only
                               valid when the gradients of the whole stream are known up front (they
                               are rows of the bound buffer), for populations that fit shared memory
-                              (2 n + 16 <= 196 rows of 256 floats; A2_EINVAL otherwise), and a plan
+                              (2 n + 16 <= 216 rows of 256 floats; A2_EINVAL otherwise), and a plan
                               made with it must be run whole (all batches in one a2cid2_plan_run).
                               With bf16 storage the tile is kept in fp32 and rounded once, at the end
                               of the call.                                                     */

@@ -53,24 +53,17 @@ struct ResOp {  // one elementary operation, as the resident kernel reads it (16
 struct ResLevel {
     int32_t item_begin, item_end;  // items that touch disjoint workers
 };
-struct ResChunk {  // a stretch of levels whose descriptors are staged in shared memory together
-    int32_t level_begin, level_end;
-    int32_t item_begin, item_end;
-    int32_t op_begin, op_end;
-    int32_t g_begin, g_count;  // gradient rows to (re)load before it: g_rows[g_begin .. g_begin + g_count)
+struct ResChunk {
+    int32_t level_begin, level_end;  // levels of the chunk
+    int32_t g_begin, g_count;        // its gradient rows: g_rows[g_begin .. g_begin + g_count)
 };
-struct ResGRow {
-    int32_t slot;   // row of the gradient buffer
-    int32_t index;  // cache row it goes to
-};
-constexpr int kResidentCols = 256;            // columns per tile
-constexpr int kResidentThreads = 1024;        // = 4 items of a level in flight per column
-constexpr int kResidentMaxRows = 196;         // 2 n + cache rows, 1 KB of shared memory each
+constexpr int kResidentCols = 256;      // columns per tile
+constexpr int kResidentThreads = 1024;  // = 4 items of a level in flight per column
+constexpr int kResidentMaxRows = 216;   // 2 n + cache rows, 1 KB of shared memory each
 constexpr int kResidentMinCache = 16;
-constexpr int kResidentDescBytes = 28 * 1024;  // shared memory for one chunk's item and operation records
 
 void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResLevel>& levels,
-                           std::vector<ResChunk>& chunks, std::vector<ResGRow>& g_rows,
+                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
                            std::vector<int32_t>& cache_a, std::vector<int32_t>& cache_b);
 
 // Builds a schedule; returns A2_OK or an error code with the text in `err`.
@@ -144,7 +137,7 @@ struct ResidentLaunch {
     ResOp* res_ops;          // device, n_ops (written by the prepare kernel)
     const ResLevel* levels;  // device
     const ResChunk* chunks;  // device
-    const ResGRow* g_rows;   // device
+    const int32_t* g_rows;   // device
     int32_t n_ops, n_chunks, cache_rows;
 };
 int resident_cache_rows(int32_t n, int32_t n_grad_slots);  // 0: the population does not fit

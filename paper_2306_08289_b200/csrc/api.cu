@@ -87,8 +87,7 @@ struct Packed {
     size_t levels_off = 0, chunks_off = 0, g_rows_off = 0, res_ops_off = 0;
     std::vector<a2::ResLevel> levels;
     std::vector<a2::ResChunk> chunks;
-    std::vector<a2::ResGRow> g_rows;
-    std::vector<int32_t> cache_a, cache_b;
+    std::vector<int32_t> g_rows, cache_a, cache_b;
 };
 
 struct a2cid2_plan {
@@ -174,12 +173,12 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
     } else {
         pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
         if (pk.cache_rows <= 0)
-            return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT: the population does not fit shared memory (need 2 n + 16 <= 196)");
+            return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT: the population does not fit shared memory (need 2 n + 16 <= 216)");
         a2::build_resident_chunks(s, pk.cache_rows, pk.levels, pk.chunks, pk.g_rows, pk.cache_a, pk.cache_b);
         pk.levels_off = align16(end);
         pk.chunks_off = align16(pk.levels_off + pk.levels.size() * sizeof(a2::ResLevel));
         pk.g_rows_off = align16(pk.chunks_off + pk.chunks.size() * sizeof(a2::ResChunk));
-        pk.res_ops_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(a2::ResGRow));
+        pk.res_ops_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(int32_t));
         end = pk.res_ops_off + s.ops.size() * sizeof(a2::ResOp);  // this part is written on the device
     }
     pk.bytes = s.items.empty() ? 0 : end;
@@ -212,7 +211,7 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
         if (!pk.chunks.empty())
             std::memcpy(static_cast<char*>(dst) + pk.chunks_off, pk.chunks.data(), pk.chunks.size() * sizeof(a2::ResChunk));
         if (!pk.g_rows.empty())
-            std::memcpy(static_cast<char*>(dst) + pk.g_rows_off, pk.g_rows.data(), pk.g_rows.size() * sizeof(a2::ResGRow));
+            std::memcpy(static_cast<char*>(dst) + pk.g_rows_off, pk.g_rows.data(), pk.g_rows.size() * sizeof(int32_t));
     }
     for (size_t o = 0; o < s.ops.size(); ++o) {
         const a2::SchedOp& op = s.ops[o];
@@ -237,7 +236,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.res_ops = reinterpret_cast<a2::ResOp*>(base + pk.res_ops_off);
         L.levels = reinterpret_cast<const a2::ResLevel*>(base + pk.levels_off);
         L.chunks = reinterpret_cast<const a2::ResChunk*>(base + pk.chunks_off);
-        L.g_rows = reinterpret_cast<const a2::ResGRow*>(base + pk.g_rows_off);
+        L.g_rows = reinterpret_cast<const int32_t*>(base + pk.g_rows_off);
         L.n_ops = (int32_t)s.ops.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
         const int rc = a2::launch_resident(L, h->dev, h->stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");

@@ -523,16 +523,15 @@ struct ResidentArgs {
     const ResOp* ops;
     const ResLevel* levels;
     const ResChunk* chunks;
-    const ResGRow* g_rows;
+    const int* g_rows;
     int n_chunks;
-    int cache_rows;
     float alpha, alpha_tilde, gamma;
     int msg_before_mix;
 };
 
 template <typename T>
 __global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const ResidentArgs p) {
-    extern __shared__ float s_tile[];  // [n][256] x, [n][256] x~, [cache][256] gradient rows, then descriptors
+    extern __shared__ float s_tile[];  // [n][256] x, [n][256] x~, [cache][256] gradient rows
     constexpr int W = kResidentCols;
     constexpr int GROUPS = kResidentThreads / W;
     const int c = threadIdx.x % W;   // column of the tile
@@ -540,7 +539,6 @@ __global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const Resident
     float* const sX = s_tile + c;
     float* const sXt = sX + (size_t)p.n * W;
     float* const sG = sXt + (size_t)p.n * W;
-    uint32_t* const s_desc = reinterpret_cast<uint32_t*>(s_tile + (size_t)(2 * p.n + p.cache_rows) * W);
     T* const X = static_cast<T*>(p.x);
     T* const Xt = static_cast<T*>(p.xt);
     const T* const G = static_cast<const T*>(p.g);
@@ -558,26 +556,15 @@ __global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const Resident
         }
         for (int ck = 0; ck < p.n_chunks; ++ck) {
             const ResChunk ch = p.chunks[ck];
-            __syncthreads();  // the previous chunk's levels are done with the descriptors and the cache
-            // stage the chunk's item and operation records (word by word, coalesced)
-            const int item_words = (ch.item_end - ch.item_begin) * (int)(sizeof(DevItem) / 4);
-            const int op_words = (ch.op_end - ch.op_begin) * (int)(sizeof(ResOp) / 4);
-            const uint32_t* src_items = reinterpret_cast<const uint32_t*>(p.items + ch.item_begin);
-            const uint32_t* src_ops = reinterpret_cast<const uint32_t*>(p.ops + ch.op_begin);
-            for (int w = threadIdx.x; w < item_words; w += kResidentThreads) s_desc[w] = __ldg(src_items + w);
-            for (int w = threadIdx.x; w < op_words; w += kResidentThreads) s_desc[item_words + w] = __ldg(src_ops + w);
-            const DevItem* const s_items = reinterpret_cast<const DevItem*>(s_desc) - ch.item_begin;
-            const ResOp* const s_ops = reinterpret_cast<const ResOp*>(s_desc + item_words) - ch.op_begin;
+            __syncthreads();  // the previous chunk's levels are done with the gradient cache (and the tile is loaded)
 #pragma unroll 4
-            for (int k = q; k < ch.g_count; k += GROUPS) {
-                const ResGRow r = p.g_rows[ch.g_begin + k];
-                sG[r.index * W] = active ? widen1<T>(__ldg(G + (long long)r.slot * p.pitch + col)) : 0.f;
-            }
+            for (int k = q; k < ch.g_count; k += GROUPS)
+                sG[k * W] = active ? widen1<T>(__ldg(G + (long long)p.g_rows[ch.g_begin + k] * p.pitch + col)) : 0.f;
             for (int lv = ch.level_begin; lv < ch.level_end; ++lv) {
                 const ResLevel L = p.levels[lv];
-                __syncthreads();  // every thread passes here once per level: what this level reads has been written
+                __syncthreads();  // every thread passes here once per level: the rows this level reads are written
                 for (int k = L.item_begin + q; k < L.item_end; k += GROUPS) {
-                    const DevItem it = s_items[k];
+                    const DevItem it = p.items[k];
                     const bool has_b = it.b >= 0;
                     const int rb = has_b ? it.b : it.a;
                     float xa = sX[it.a * W], xta = sXt[it.a * W];
@@ -585,7 +572,7 @@ __global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const Resident
                     const float ga = it.slot_a >= 0 ? sG[it.slot_a * W] : 0.f;
                     const float gb = it.slot_b >= 0 ? sG[it.slot_b * W] : 0.f;
                     for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
-                        const ResOp op = s_ops[o];
+                        const ResOp op = p.ops[o];
                         if (op.kind == A2_OP_GRAD_A) grad_elem(xa, xta, op.ca, ngamma, ga);
                         else if (op.kind == A2_OP_GRAD_B) grad_elem(xb, xtb, op.cb, ngamma, gb);
                         else comm_elem<sizeof(T) == 4>(xa, xta, xb, xtb, op.ca, op.cb, p.alpha, p.alpha_tilde, before);
@@ -612,7 +599,7 @@ __global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const Resident
 
 template <typename T>
 int launch_resident_t(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
-    const size_t smem = (size_t)(2 * L.n + L.cache_rows) * kResidentCols * sizeof(float) + kResidentDescBytes;
+    const size_t smem = (size_t)(2 * L.n + L.cache_rows) * kResidentCols * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_resident<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     int occ = 0;
@@ -624,7 +611,6 @@ int launch_resident_t(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream
     a.n_tiles = (L.d + kResidentCols - 1) / kResidentCols;
     a.n = L.n; a.items = L.items; a.ops = L.res_ops; a.levels = L.levels; a.chunks = L.chunks; a.g_rows = L.g_rows;
     a.n_chunks = L.n_chunks;
-    a.cache_rows = L.cache_rows;
     a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     long long grid = (long long)dev.sm_count * occ;

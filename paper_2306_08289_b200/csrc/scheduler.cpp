@@ -188,39 +188,29 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
 }
 
 // Resident mode. The kernel walks "levels" (item ranges whose items touch disjoint workers: the
-// schedule's batches, split further where needed). Levels are grouped into "chunks": the item and
-// operation records of a chunk are staged in shared memory together (kResidentDescBytes), and before a
-// chunk the gradient rows it uses for the first time are loaded into a cache of `capacity` rows. A row
-// keeps its cache index until the cache overflows; then the cache starts over. Items get the cache
-// indices of their rows.
+// schedule's batches, split further where needed) and keeps the gradient rows of a "chunk" of
+// consecutive levels in a cache of `capacity` rows. Items get the cache indices of their rows.
 void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResLevel>& levels,
-                           std::vector<ResChunk>& chunks, std::vector<ResGRow>& g_rows,
+                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
                            std::vector<int32_t>& cache_a, std::vector<int32_t>& cache_b) {
     levels.clear();
     chunks.clear();
     g_rows.clear();
     cache_a.assign(s.items.size(), -1);
     cache_b.assign(s.items.size(), -1);
-    std::vector<int32_t> where((size_t)std::max(1, s.n_grad_slots), -1);  // slot -> cache index, or -1
-    std::vector<int32_t> cached;                                           // slots now in the cache
-    ResChunk cur{};
+    std::vector<int32_t> where((size_t)std::max(1, s.n_grad_slots), -1);  // slot -> cache index in the open chunk
+    ResChunk cur{0, 0, 0, 0};
     ResLevel lev{0, 0};
     auto close_level = [&](int32_t item_end) {
         lev.item_end = item_end;
         if (lev.item_end > lev.item_begin) levels.push_back(lev);
         lev = ResLevel{item_end, item_end};
     };
-    auto close_chunk = [&](int32_t item_end, int32_t op_end) {
+    auto close_chunk = [&]() {
         cur.level_end = (int32_t)levels.size();
-        cur.item_end = item_end;
-        cur.op_end = op_end;
-        cur.g_count = (int32_t)g_rows.size() - cur.g_begin;
         if (cur.level_end > cur.level_begin) chunks.push_back(cur);
-        cur = ResChunk{(int32_t)levels.size(), 0, item_end, 0, op_end, 0, (int32_t)g_rows.size(), 0};
-    };
-    auto desc_bytes = [&](int32_t item_end, int32_t op_end) {
-        return (int64_t)(item_end - cur.item_begin) * (int64_t)sizeof(DevItem) +
-               (int64_t)(op_end - cur.op_begin) * (int64_t)sizeof(ResOp);
+        for (int32_t k = cur.g_begin; k < cur.g_begin + cur.g_count; ++k) where[(size_t)g_rows[(size_t)k]] = -1;
+        cur = ResChunk{(int32_t)levels.size(), (int32_t)levels.size(), (int32_t)g_rows.size(), 0};
     };
     const int64_t nb = (int64_t)s.batch_first.size() - 1;
     for (int64_t b = 0; b < nb; ++b) {
@@ -229,28 +219,22 @@ void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResL
             int32_t fresh = 0;
             if (it.slot_a >= 0 && where[(size_t)it.slot_a] < 0) fresh += 1;
             if (it.slot_b >= 0 && it.slot_b != it.slot_a && where[(size_t)it.slot_b] < 0) fresh += 1;
-            const bool cache_full = (int32_t)cached.size() + fresh > capacity;
-            const bool desc_full = desc_bytes((int32_t)k + 1, (int32_t)(it.first_op + it.n_ops)) > kResidentDescBytes - 64;
-            if (cache_full || desc_full) {  // end the level and the chunk before this item
+            if (cur.g_count + fresh > capacity) {  // the cache is full: end the level here and start a new chunk
                 close_level((int32_t)k);
-                close_chunk((int32_t)k, (int32_t)it.first_op);
-                if (cache_full) {
-                    for (int32_t slot : cached) where[(size_t)slot] = -1;
-                    cached.clear();
-                }
+                close_chunk();
             }
             for (int32_t slot : {it.slot_a, it.slot_b}) {
                 if (slot < 0 || where[(size_t)slot] >= 0) continue;
-                where[(size_t)slot] = (int32_t)cached.size();
-                g_rows.push_back(ResGRow{slot, (int32_t)cached.size()});
-                cached.push_back(slot);
+                where[(size_t)slot] = cur.g_count;
+                g_rows.push_back(slot);
+                cur.g_count += 1;
             }
             if (it.slot_a >= 0) cache_a[(size_t)k] = where[(size_t)it.slot_a];
             if (it.slot_b >= 0) cache_b[(size_t)k] = where[(size_t)it.slot_b];
         }
         close_level((int32_t)s.batch_first[(size_t)b + 1]);
     }
-    close_chunk((int32_t)s.items.size(), (int32_t)s.ops.size());
+    close_chunk();
 }
 
 void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {
