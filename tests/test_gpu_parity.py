@@ -127,20 +127,19 @@ def test_resident_mode_is_bit_identical_to_batches_fp32(name, d, n_events):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     ev = W.config_events(cfg)
     states = []
-    for flags in (B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT, B.A2_SCHED_RESIDENT | B.A2_SCHED_FUSE):
+    for flags in (B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
         eng, chk = P.make_small(cfg)
         for lo in range(0, len(ev), 777):  # several calls, so that resident calls chain on stored state
             c = ev.slice(lo, lo + 777)
             st = eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=flags, want_stats=True)
-            if flags & B.A2_SCHED_RESIDENT:
-                assert st["n_launches"] == 2 and st["n_batches"] > 1
+            if flags == B.A2_SCHED_RESIDENT:
+                assert st["n_launches"] == 2 and st["n_batches"] == 1
                 chk.plain.apply_stream(c)
                 x, xt, t = eng.read_state()
                 chk.compare(P.widen(x, "f32"), P.widen(xt, "f32"), t, where=f"resident {name} after event {lo + len(c)}")
         states.append(eng.read_state())
         eng.close()
-    for other in states[1:]:
-        assert all(np.array_equal(u, v) for u, v in zip(states[0], other))
+    assert all(np.array_equal(u, v) for u, v in zip(states[0], states[1]))
 
 
 def test_resident_mode_bf16_storage():
@@ -162,10 +161,8 @@ def test_resident_mode_plan_variant_and_limits():
     cfg = W.CONFIGS["cfg3"].scaled(d=2_050, n_events=1200)
     ev = W.config_events(cfg)
     eng, chk = P.make_small(cfg, variant=B.A2_MSG_BEFORE_MIX)
-    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_RESIDENT | B.A2_SCHED_FUSE)
-    with pytest.raises(B.A2Error) as e:
-        p.run(0, 1)  # a resident plan is one launch: all batches or none
-    assert e.value.code == B.A2_ESTATE
+    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_RESIDENT)
+    assert p.sched.num_batches == 1
     p.run()
     p.close()
     chk.plain.apply_stream(ev)

@@ -154,14 +154,17 @@ def test_bad_arguments():
         s.ops(0, 5)
 
 
-def test_resident_flag_is_a_launch_mode_and_keeps_the_schedule():
+def test_resident_schedule_is_one_batch_in_stream_order():
     cfg = W.CONFIGS["cfg2"].scaled(d=3, n_events=1500)
     ev = W.config_events(cfg)
-    for fuse in (0, B.A2_SCHED_FUSE):
-        a = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=fuse)
-        b = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=fuse | B.A2_SCHED_RESIDENT)
-        assert (a.num_batches, a.num_items, a.num_ops) == (b.num_batches, b.num_items, b.num_ops)
-        for k in range(0, a.num_batches, 17):
-            assert np.array_equal(a.batch_events(k), b.batch_events(k))
+    for flags in (B.A2_SCHED_RESIDENT, B.A2_SCHED_RESIDENT | B.A2_SCHED_FUSE):  # the resident flag wins
+        s = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+        assert s.num_batches == 1 and s.num_items == len(ev) == s.num_ops
+        assert np.array_equal(s.batch_events(0), np.arange(len(ev)))
+        it = s.item(7)
+        assert (it.a, it.n_ops, it.batch) == (ev.wi[7], 1, 0)
+    sim = OracleSim(np.zeros((cfg.n, 1)), 0.1, 0.5, 0.5, 0.0, grads=np.zeros((cfg.n_grad_slots, 1)))
+    sim.apply_stream(ev)
+    assert np.array_equal(s.t_final(cfg.n), sim.t)
     with pytest.raises(B.A2Error):
         B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=4)
