@@ -84,10 +84,9 @@ struct Packed {
     // resident mode
     bool resident = false;
     int32_t cache_rows = 0;
-    size_t levels_off = 0, chunks_off = 0, g_rows_off = 0, res_ops_off = 0;
-    std::vector<a2::ResLevel> levels;
+    size_t chunks_off = 0, g_rows_off = 0, events_off = 0;
     std::vector<a2::ResChunk> chunks;
-    std::vector<int32_t> g_rows, cache_a, cache_b;
+    std::vector<int32_t> g_rows, cache_idx;
 };
 
 struct a2cid2_plan {
@@ -174,12 +173,11 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
         pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
         if (pk.cache_rows <= 0)
             return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT: the population does not fit shared memory (need 2 n + 16 <= 216)");
-        a2::build_resident_chunks(s, pk.cache_rows, pk.levels, pk.chunks, pk.g_rows, pk.cache_a, pk.cache_b);
-        pk.levels_off = align16(end);
-        pk.chunks_off = align16(pk.levels_off + pk.levels.size() * sizeof(a2::ResLevel));
+        a2::build_resident_chunks(s, pk.cache_rows, pk.chunks, pk.g_rows, pk.cache_idx);
+        pk.chunks_off = align16(end);
         pk.g_rows_off = align16(pk.chunks_off + pk.chunks.size() * sizeof(a2::ResChunk));
-        pk.res_ops_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(int32_t));
-        end = pk.res_ops_off + s.ops.size() * sizeof(a2::ResOp);  // this part is written on the device
+        pk.events_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(int32_t));
+        end = pk.events_off + s.items.size() * sizeof(a2::ResEv);  // this part is written on the device
     }
     pk.bytes = s.items.empty() ? 0 : end;
     return A2_OK;
@@ -189,7 +187,7 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
 // produced there).
 size_t upload_bytes(const a2cid2_sched& s, const Packed& pk) {
     if (s.items.empty()) return 0;
-    return pk.resident ? pk.res_ops_off : pk.bytes;
+    return pk.resident ? pk.events_off : pk.bytes;
 }
 
 void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
@@ -202,12 +200,10 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
                 di[k] = DevItem{it.a, it.b, it.slot_a, it.slot_b, (int32_t)(it.first_op - L.op0), it.n_ops};
             }
     } else {
-        for (size_t k = 0; k < s.items.size(); ++k) {  // gradient rows by cache index, operations by absolute index
+        for (size_t k = 0; k < s.items.size(); ++k) {  // one operation per item; slot_b carries the cache index
             const a2::SchedItem& it = s.items[k];
-            di[k] = DevItem{it.a, it.b, pk.cache_a[k], pk.cache_b[k], (int32_t)it.first_op, it.n_ops};
+            di[k] = DevItem{it.a, it.b, it.slot_a, pk.cache_idx[k], (int32_t)k, 1};
         }
-        if (!pk.levels.empty())
-            std::memcpy(static_cast<char*>(dst) + pk.levels_off, pk.levels.data(), pk.levels.size() * sizeof(a2::ResLevel));
         if (!pk.chunks.empty())
             std::memcpy(static_cast<char*>(dst) + pk.chunks_off, pk.chunks.data(), pk.chunks.size() * sizeof(a2::ResChunk));
         if (!pk.g_rows.empty())
@@ -226,18 +222,15 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     const DevItem* d_items = reinterpret_cast<const DevItem*>(base);
     const DevOp* d_ops = reinterpret_cast<const DevOp*>(base + pk.ops_off);
     if (pk.resident) {
-        if (b0 != 0 || b1 != (int64_t)s.batch_first.size() - 1)
-            return fail(h, A2_ESTATE, "a plan made with A2_SCHED_RESIDENT runs all its batches in one call");
         a2::ResidentLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.n = h->n; L.dtype = h->dtype; L.variant = h->variant; L.eta = h->eta;
         L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
         L.items = d_items; L.ops = d_ops;
-        L.res_ops = reinterpret_cast<a2::ResOp*>(base + pk.res_ops_off);
-        L.levels = reinterpret_cast<const a2::ResLevel*>(base + pk.levels_off);
+        L.events = reinterpret_cast<a2::ResEv*>(base + pk.events_off);
         L.chunks = reinterpret_cast<const a2::ResChunk*>(base + pk.chunks_off);
         L.g_rows = reinterpret_cast<const int32_t*>(base + pk.g_rows_off);
-        L.n_ops = (int32_t)s.ops.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
+        L.n_events = (int32_t)s.items.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
         const int rc = a2::launch_resident(L, h->dev, h->stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;

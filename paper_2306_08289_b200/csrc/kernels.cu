@@ -478,31 +478,34 @@ int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, in
 }
 
 // ---------------------------------------------------------------------------------------------
-// Resident mode: one launch for a whole schedule.
+// Resident mode: one launch for a whole event stream.
 //
 // Every operation of the method is element-wise over the parameter dimension, so a column never
-// needs another column and a CTA never needs another CTA. A CTA takes a tile of 256 columns, loads
-// x[:, tile] and x~[:, tile] of ALL n workers into shared memory, walks the schedule's levels (items
-// on disjoint workers) and writes the tile back: the state crosses HBM once per call. Inside a level,
-// (item, column) pairs are independent and are spread over the CTA's 1024 threads (4 items in flight
-// per column); between levels stands an ordinary __syncthreads(), reached by every thread the same
-// number of times (the level list is uniform across the CTA). The gradient rows come from a cache in
-// shared memory that is refilled per chunk of levels (the host cut the schedule so that a chunk's
-// distinct rows fit). Nothing spins, nothing waits on another CTA.
+// needs another column. A thread therefore owns one column of a 256-column tile for ALL n workers:
+// it loads x[:, c] and x~[:, c] into its own lane of shared memory (used as a register file that
+// can be indexed by worker), walks the events in stream order, and writes the column back. No thread
+// reads what another thread wrote: there is no barrier, no flag and no wait anywhere. The gradient
+// rows an event needs come from a small cache in shared memory that is refilled chunk by chunk of the
+// stream (the host cut the stream so that a chunk's distinct rows fit). The state crosses HBM once per
+// call, gradient rows once per use; the rest is shared-memory traffic and ALU work.
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-__global__ void __launch_bounds__(kThreads) k_resident_prepare(const DevOp* __restrict__ ops, int n_ops, double eta,
-                                                             ResOp* __restrict__ out) {
-    const int o = blockIdx.x * kThreads + threadIdx.x;
-    if (o >= n_ops) return;
-    const DevOp op = ops[o];
-    ResOp r;
-    r.kind = op.kind;
-    r.ca = op.kind != A2_OP_GRAD_B ? (float)mix_coeff(eta, op.t - op.t_prev_a) : 0.f;
-    r.cb = op.kind != A2_OP_GRAD_A ? (float)mix_coeff(eta, op.t - op.t_prev_b) : 0.f;
-    r.pad = 0;
-    out[o] = r;
+__global__ void __launch_bounds__(kThreads) k_resident_prepare(const DevItem* __restrict__ items,
+                                                             const DevOp* __restrict__ ops, int n_events, double eta,
+                                                             ResEv* __restrict__ out) {
+    const int e = blockIdx.x * kThreads + threadIdx.x;
+    if (e >= n_events) return;
+    const DevItem it = items[e];
+    const DevOp op = ops[e];
+    ResEv r;
+    r.a = (int16_t)it.a;
+    r.b = (int16_t)it.b;
+    r.g = (int16_t)it.slot_b;  // cache index of the gradient row (set by the host for gradient events)
+    r.kind = (int16_t)op.kind;
+    r.ca = (float)mix_coeff(eta, op.t - op.t_prev_a);
+    r.cb = op.kind == A2_OP_COMM ? (float)mix_coeff(eta, op.t - op.t_prev_b) : 0.f;
+    out[e] = r;
 }
 
 template <typename T> __device__ __forceinline__ float widen1(T v);
@@ -519,9 +522,7 @@ struct ResidentArgs {
     long long pitch;
     long long n_tiles;
     int n;
-    const DevItem* items;
-    const ResOp* ops;
-    const ResLevel* levels;
+    const ResEv* events;
     const ResChunk* chunks;
     const int* g_rows;
     int n_chunks;
@@ -530,68 +531,62 @@ struct ResidentArgs {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kResidentThreads, 1) k_resident(const ResidentArgs p) {
+__global__ void __launch_bounds__(kResidentCols) k_resident(const ResidentArgs p) {
     extern __shared__ float s_tile[];  // [n][256] x, [n][256] x~, [cache][256] gradient rows
-    constexpr int W = kResidentCols;
-    constexpr int GROUPS = kResidentThreads / W;
-    const int c = threadIdx.x % W;   // column of the tile
-    const int q = threadIdx.x / W;   // which of the level's items this thread starts with
-    float* const sX = s_tile + c;
-    float* const sXt = sX + (size_t)p.n * W;
-    float* const sG = sXt + (size_t)p.n * W;
+    float* const sX = s_tile + threadIdx.x;
+    float* const sXt = sX + (size_t)p.n * kResidentCols;
+    float* const sG = sXt + (size_t)p.n * kResidentCols;
     T* const X = static_cast<T*>(p.x);
     T* const Xt = static_cast<T*>(p.xt);
     const T* const G = static_cast<const T*>(p.g);
+    const int lane = threadIdx.x & 31;
     const float ngamma = -p.gamma;
     const bool before = p.msg_before_mix != 0;
 
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
-        const long long col = tile * W + c;
+        const long long col = tile * kResidentCols + threadIdx.x;
         const bool active = col < p.pitch;  // padding columns are carried along; nothing past the pitch is touched
-        __syncthreads();  // the previous tile's write-back has read the tile
-#pragma unroll 4
-        for (int i = q; i < p.n; i += GROUPS) {
-            sX[i * W] = active ? widen1<T>(__ldcs(X + (long long)i * p.pitch + col)) : 0.f;
-            sXt[i * W] = active ? widen1<T>(__ldcs(Xt + (long long)i * p.pitch + col)) : 0.f;
+#pragma unroll 8
+        for (int i = 0; i < p.n; ++i) {
+            sX[i * kResidentCols] = active ? widen1<T>(__ldcs(X + (long long)i * p.pitch + col)) : 0.f;
+            sXt[i * kResidentCols] = active ? widen1<T>(__ldcs(Xt + (long long)i * p.pitch + col)) : 0.f;
         }
-        for (int ck = 0; ck < p.n_chunks; ++ck) {
-            const ResChunk ch = p.chunks[ck];
-            __syncthreads();  // the previous chunk's levels are done with the gradient cache (and the tile is loaded)
+        for (int c = 0; c < p.n_chunks; ++c) {
+            const ResChunk ch = p.chunks[c];
 #pragma unroll 4
-            for (int k = q; k < ch.g_count; k += GROUPS)
-                sG[k * W] = active ? widen1<T>(__ldg(G + (long long)p.g_rows[ch.g_begin + k] * p.pitch + col)) : 0.f;
-            for (int lv = ch.level_begin; lv < ch.level_end; ++lv) {
-                const ResLevel L = p.levels[lv];
-                __syncthreads();  // every thread passes here once per level: the rows this level reads are written
-                for (int k = L.item_begin + q; k < L.item_end; k += GROUPS) {
-                    const DevItem it = p.items[k];
-                    const bool has_b = it.b >= 0;
-                    const int rb = has_b ? it.b : it.a;
-                    float xa = sX[it.a * W], xta = sXt[it.a * W];
-                    float xb = sX[rb * W], xtb = sXt[rb * W];
-                    const float ga = it.slot_a >= 0 ? sG[it.slot_a * W] : 0.f;
-                    const float gb = it.slot_b >= 0 ? sG[it.slot_b * W] : 0.f;
-                    for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
-                        const ResOp op = p.ops[o];
-                        if (op.kind == A2_OP_GRAD_A) grad_elem(xa, xta, op.ca, ngamma, ga);
-                        else if (op.kind == A2_OP_GRAD_B) grad_elem(xb, xtb, op.cb, ngamma, gb);
-                        else comm_elem<sizeof(T) == 4>(xa, xta, xb, xtb, op.ca, op.cb, p.alpha, p.alpha_tilde, before);
+            for (int k = 0; k < ch.g_count; ++k)
+                sG[k * kResidentCols] = active ? widen1<T>(__ldg(G + (long long)p.g_rows[ch.g_begin + k] * p.pitch + col)) : 0.f;
+            for (int e0 = ch.ev_begin; e0 < ch.ev_end; e0 += 32) {
+                // a warp fetches 32 descriptors with one coalesced load and hands them round by shuffle
+                int4 mine = make_int4(0, 0, 0, 0);
+                if (e0 + lane < ch.ev_end) mine = __ldg(reinterpret_cast<const int4*>(p.events) + e0 + lane);
+                const int cnt = min(32, ch.ev_end - e0);
+                for (int l = 0; l < cnt; ++l) {
+                    const int w0 = __shfl_sync(0xffffffffu, mine.x, l);
+                    const int w1 = __shfl_sync(0xffffffffu, mine.y, l);
+                    const float ca = __int_as_float(__shfl_sync(0xffffffffu, mine.z, l));
+                    const float cb = __int_as_float(__shfl_sync(0xffffffffu, mine.w, l));
+                    const int a = (int)(short)(w0 & 0xFFFF), b = (int)(short)(w0 >> 16);
+                    const int gi = (int)(short)(w1 & 0xFFFF), kind = (int)(short)(w1 >> 16);
+                    float xa = sX[a * kResidentCols], xta = sXt[a * kResidentCols];
+                    if (kind == A2_OP_COMM) {
+                        float xb = sX[b * kResidentCols], xtb = sXt[b * kResidentCols];
+                        comm_elem<sizeof(T) == 4>(xa, xta, xb, xtb, ca, cb, p.alpha, p.alpha_tilde, before);
+                        sX[b * kResidentCols] = xb;
+                        sXt[b * kResidentCols] = xtb;
+                    } else {
+                        grad_elem(xa, xta, ca, ngamma, sG[gi * kResidentCols]);
                     }
-                    sX[it.a * W] = xa;
-                    sXt[it.a * W] = xta;
-                    if (has_b) {
-                        sX[rb * W] = xb;
-                        sXt[rb * W] = xtb;
-                    }
+                    sX[a * kResidentCols] = xa;
+                    sXt[a * kResidentCols] = xta;
                 }
             }
         }
-        __syncthreads();  // all levels done before the tile is written back
         if (active) {
-#pragma unroll 4
-            for (int i = q; i < p.n; i += GROUPS) {
-                __stcs(X + (long long)i * p.pitch + col, narrow1<T>(sX[i * W]));
-                __stcs(Xt + (long long)i * p.pitch + col, narrow1<T>(sXt[i * W]));
+#pragma unroll 8
+            for (int i = 0; i < p.n; ++i) {
+                __stcs(X + (long long)i * p.pitch + col, narrow1<T>(sX[i * kResidentCols]));
+                __stcs(Xt + (long long)i * p.pitch + col, narrow1<T>(sXt[i * kResidentCols]));
             }
         }
     }
@@ -603,19 +598,18 @@ int launch_resident_t(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream
     cudaError_t e = cudaFuncSetAttribute(k_resident<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_resident<T>, kResidentThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_resident<T>, kResidentCols, smem);
     if (e != cudaSuccess) return (int)e;
     if (occ < 1) return (int)cudaErrorInvalidConfiguration;
     ResidentArgs a;
     a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
     a.n_tiles = (L.d + kResidentCols - 1) / kResidentCols;
-    a.n = L.n; a.items = L.items; a.ops = L.res_ops; a.levels = L.levels; a.chunks = L.chunks; a.g_rows = L.g_rows;
-    a.n_chunks = L.n_chunks;
+    a.n = L.n; a.events = L.events; a.chunks = L.chunks; a.g_rows = L.g_rows; a.n_chunks = L.n_chunks;
     a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     long long grid = (long long)dev.sm_count * occ;
     if (grid > a.n_tiles) grid = a.n_tiles;
-    k_resident<T><<<(unsigned)grid, kResidentThreads, smem, stream>>>(a);
+    k_resident<T><<<(unsigned)grid, kResidentCols, smem, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -631,10 +625,10 @@ int resident_cache_rows(int32_t n, int32_t n_grad_slots) {
 }
 
 int launch_resident(const ResidentLaunch& L, const DeviceInfo& dev, void* stream_) {
-    if (L.n_ops <= 0) return 0;
+    if (L.n_events <= 0) return 0;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int blocks = (L.n_ops + kThreads - 1) / kThreads;
-    k_resident_prepare<<<blocks, kThreads, 0, stream>>>(L.ops, L.n_ops, L.eta, L.res_ops);
+    const int blocks = (L.n_events + kThreads - 1) / kThreads;
+    k_resident_prepare<<<blocks, kThreads, 0, stream>>>(L.items, L.ops, L.n_events, L.eta, L.events);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     if (L.dtype == A2_BF16) return launch_resident_t<__nv_bfloat16>(L, dev, stream);
