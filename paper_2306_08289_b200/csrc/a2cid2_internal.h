@@ -45,26 +45,22 @@ struct a2cid2_sched {
 namespace a2 {
 
 // Resident mode (one launch, column tile of the whole population in shared memory).
-struct ResOp {  // one elementary operation, as the resident kernel reads it (16 bytes)
-    int32_t kind;  // A2_OP_*
-    float ca, cb;  // mixing coefficients of a and b for this operation
-    int32_t pad;
-};
-struct ResLevel {
-    int32_t item_begin, item_end;  // items that touch disjoint workers
+struct ResEv {  // one event, as the resident kernel reads it (16 bytes)
+    int16_t a, b;  // workers (b = -1: gradient event)
+    int16_t g;     // index of the gradient row in the chunk's cache, or -1
+    int16_t kind;  // A2_OP_GRAD_A or A2_OP_COMM
+    float ca, cb;  // mixing coefficients of a and b for this event
 };
 struct ResChunk {
-    int32_t level_begin, level_end;  // levels of the chunk
-    int32_t g_begin, g_count;        // its gradient rows: g_rows[g_begin .. g_begin + g_count)
+    int32_t ev_begin, ev_end;  // events of the chunk
+    int32_t g_begin, g_count;  // its gradient rows: g_rows[g_begin .. g_begin + g_count)
 };
-constexpr int kResidentCols = 256;      // columns per tile
-constexpr int kResidentThreads = 1024;  // = 4 items of a level in flight per column
-constexpr int kResidentMaxRows = 216;   // 2 n + cache rows, 1 KB of shared memory each
+constexpr int kResidentCols = 256;     // columns per tile = threads per CTA
+constexpr int kResidentMaxRows = 216;  // 2 n + cache rows, 1 KB of shared memory each
 constexpr int kResidentMinCache = 16;
 
-void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResLevel>& levels,
-                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
-                           std::vector<int32_t>& cache_a, std::vector<int32_t>& cache_b);
+void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResChunk>& chunks,
+                           std::vector<int32_t>& g_rows, std::vector<int32_t>& cache_idx);
 
 // Builds a schedule; returns A2_OK or an error code with the text in `err`.
 int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
@@ -123,7 +119,7 @@ int consensus_grid(const DeviceInfo& dev);
 int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, int32_t dtype, double eta,
                      const double* dt, double* partials, int n_partials, double* out, void* stream);
 
-// Resident mode. DevItem.slot_a / slot_b hold cache indices; DevItem.op_first is absolute.
+// Resident mode. prepare: items/ops (one op per item, stream order; DevItem.slot_b = cache index) -> ResEv.
 struct ResidentLaunch {
     void* x;
     void* xt;
@@ -132,13 +128,12 @@ struct ResidentLaunch {
     int32_t n, dtype, variant;
     double eta;
     float alpha, alpha_tilde, gamma;
-    const DevItem* items;    // device
-    const DevOp* ops;        // device
-    ResOp* res_ops;          // device, n_ops (written by the prepare kernel)
-    const ResLevel* levels;  // device
+    const DevItem* items;    // device, n_events
+    const DevOp* ops;        // device, n_events
+    ResEv* events;           // device, n_events (written by the prepare kernel)
     const ResChunk* chunks;  // device
     const int32_t* g_rows;   // device
-    int32_t n_ops, n_chunks, cache_rows;
+    int32_t n_events, n_chunks, cache_rows;
 };
 int resident_cache_rows(int32_t n, int32_t n_grad_slots);  // 0: the population does not fit
 int launch_resident(const ResidentLaunch& L, const DeviceInfo& dev, void* stream);

@@ -40,7 +40,8 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     if (flags & ~uint32_t(A2_SCHED_FUSE | A2_SCHED_RESIDENT)) { err = "unknown scheduling flag"; return A2_EINVAL; }
     if (max_ops_per_item <= 0) max_ops_per_item = kDefaultMaxOpsPerItem;
     if (max_ops_per_item > kMaxOpsPerLaunch) max_ops_per_item = kMaxOpsPerLaunch;
-    const bool fuse = (flags & A2_SCHED_FUSE) != 0 && max_ops_per_item >= 2;
+    const bool resident = (flags & A2_SCHED_RESIDENT) != 0;
+    const bool fuse = !resident && (flags & A2_SCHED_FUSE) != 0 && max_ops_per_item >= 2;
 
     a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
     if (!s) { err = "out of host memory"; return A2_ENOMEM; }
@@ -161,6 +162,8 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             }
         }
         if (fuse) for (int32_t w = 0; w < n; ++w) flush(w);
+        if (resident)  // one batch, every event in stream order (items were created in that order)
+            for (SchedItem& it : items) it.batch = 0;
 
         // ---- order items by batch (stable) and lay the ops out in item order ----------------
         int32_t n_batches = 0;
@@ -187,54 +190,33 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     return A2_OK;
 }
 
-// Resident mode. The kernel walks "levels" (item ranges whose items touch disjoint workers: the
-// schedule's batches, split further where needed) and keeps the gradient rows of a "chunk" of
-// consecutive levels in a cache of `capacity` rows. Items get the cache indices of their rows.
-void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResLevel>& levels,
-                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
-                           std::vector<int32_t>& cache_a, std::vector<int32_t>& cache_b) {
-    levels.clear();
+// Resident mode: cut the stream into chunks whose distinct gradient rows fit `capacity` cache rows.
+// Inside a chunk a gradient row keeps the cache index it was given at first use.
+void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResChunk>& chunks,
+                           std::vector<int32_t>& g_rows, std::vector<int32_t>& cache_idx) {
     chunks.clear();
     g_rows.clear();
-    cache_a.assign(s.items.size(), -1);
-    cache_b.assign(s.items.size(), -1);
+    cache_idx.assign(s.items.size(), -1);
     std::vector<int32_t> where((size_t)std::max(1, s.n_grad_slots), -1);  // slot -> cache index in the open chunk
     ResChunk cur{0, 0, 0, 0};
-    ResLevel lev{0, 0};
-    auto close_level = [&](int32_t item_end) {
-        lev.item_end = item_end;
-        if (lev.item_end > lev.item_begin) levels.push_back(lev);
-        lev = ResLevel{item_end, item_end};
-    };
-    auto close_chunk = [&]() {
-        cur.level_end = (int32_t)levels.size();
-        if (cur.level_end > cur.level_begin) chunks.push_back(cur);
+    auto close = [&](int32_t ev_end) {
+        cur.ev_end = ev_end;
+        if (cur.ev_end > cur.ev_begin) chunks.push_back(cur);
         for (int32_t k = cur.g_begin; k < cur.g_begin + cur.g_count; ++k) where[(size_t)g_rows[(size_t)k]] = -1;
-        cur = ResChunk{(int32_t)levels.size(), (int32_t)levels.size(), (int32_t)g_rows.size(), 0};
+        cur = ResChunk{ev_end, ev_end, (int32_t)g_rows.size(), 0};
     };
-    const int64_t nb = (int64_t)s.batch_first.size() - 1;
-    for (int64_t b = 0; b < nb; ++b) {
-        for (int64_t k = s.batch_first[(size_t)b]; k < s.batch_first[(size_t)b + 1]; ++k) {
-            const SchedItem& it = s.items[(size_t)k];
-            int32_t fresh = 0;
-            if (it.slot_a >= 0 && where[(size_t)it.slot_a] < 0) fresh += 1;
-            if (it.slot_b >= 0 && it.slot_b != it.slot_a && where[(size_t)it.slot_b] < 0) fresh += 1;
-            if (cur.g_count + fresh > capacity) {  // the cache is full: end the level here and start a new chunk
-                close_level((int32_t)k);
-                close_chunk();
-            }
-            for (int32_t slot : {it.slot_a, it.slot_b}) {
-                if (slot < 0 || where[(size_t)slot] >= 0) continue;
-                where[(size_t)slot] = cur.g_count;
-                g_rows.push_back(slot);
-                cur.g_count += 1;
-            }
-            if (it.slot_a >= 0) cache_a[(size_t)k] = where[(size_t)it.slot_a];
-            if (it.slot_b >= 0) cache_b[(size_t)k] = where[(size_t)it.slot_b];
+    for (size_t e = 0; e < s.items.size(); ++e) {
+        const int32_t slot = s.items[e].slot_a;
+        if (slot < 0) continue;
+        if (where[(size_t)slot] < 0) {
+            if (cur.g_count == capacity) close((int32_t)e);
+            where[(size_t)slot] = cur.g_count;
+            g_rows.push_back(slot);
+            cur.g_count += 1;
         }
-        close_level((int32_t)s.batch_first[(size_t)b + 1]);
+        cache_idx[e] = where[(size_t)slot];
     }
-    close_chunk();
+    close((int32_t)s.items.size());
 }
 
 void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {
