@@ -249,6 +249,75 @@ def config_events(cfg: WorkloadConfig, n_events: int | None = None, t0: float = 
                           cfg.seed, t0=t0, stream_id=stream_id, grad_pool=cfg.grad_pool)
 
 
+def fifo_pairing_events(n: int, edges: np.ndarray, comms_per_grad: float, n_events: int, seed: int,
+                        comm_duration: float = 0.05, jitter: float = 0.1, grad_pool: int = 1,
+                        stream_id: int = 0) -> EventStream:
+    """The event model of the paper's implementation (Sec. 4.1 "Practical implementation", App. E.2)
+    instead of ideal Poisson clocks. Every worker computes gradients back to back; one gradient
+    takes a unit of time times a log-normal jitter. After each gradient it draws a Poisson(
+    comms_per_grad) number of averagings still to do. A worker is *available* when it is not
+    averaging and has averagings left; a coordinator keeps the available workers in a
+    first-in-first-out queue and pairs a newly available worker with the longest-waiting available
+    neighbour. An averaging occupies both workers for `comm_duration` and counts for both.
+    Events are emitted in time order: a gradient event when a gradient completes, a communication
+    event at the moment of pairing. Gradient rows as in `poisson_events`."""
+    import heapq
+
+    edges = np.asarray(edges, dtype=np.int32).reshape(-1, 2)
+    nbr = [set() for _ in range(n)]
+    for i, j in edges:
+        nbr[int(i)].add(int(j))
+        nbr[int(j)].add(int(i))
+    rng = _rng(seed, TAG_EVENTS, 1000 + stream_id)
+    todo = [0] * n
+    busy = [False] * n
+    n_grad = [0] * n
+    queue: list[int] = []  # available workers, longest-waiting first
+    heap: list[tuple[float, int, int, int]] = []  # (time, tie-break, kind, worker); kind 0: gradient done, 1: averaging done
+    tick = 0
+
+    def push(t, kind, w):
+        nonlocal tick
+        heapq.heappush(heap, (t, tick, kind, w))
+        tick += 1
+
+    def duration():
+        return float(np.exp(jitter * rng.standard_normal() - 0.5 * jitter * jitter))
+
+    for w in range(n):
+        push(duration(), 0, w)
+    times, wi, wj, slot = [], [], [], []
+
+    def try_enqueue(w, t):
+        if todo[w] <= 0 or busy[w] or w in queue:
+            return
+        for pos, other in enumerate(queue):
+            if other in nbr[w]:
+                queue.pop(pos)
+                times.append(t); wi.append(other); wj.append(w); slot.append(-1)
+                for v in (w, other):
+                    todo[v] -= 1
+                    busy[v] = True
+                    push(t + comm_duration, 1, v)
+                return
+        queue.append(w)
+
+    while len(times) < n_events:
+        t, _, kind, w = heapq.heappop(heap)
+        if kind == 0:
+            times.append(t); wi.append(w); wj.append(-1); slot.append(w + n * (n_grad[w] % max(1, grad_pool)))
+            n_grad[w] += 1
+            todo[w] += int(rng.poisson(comms_per_grad))
+            push(t + duration(), 0, w)
+        else:
+            busy[w] = False
+        try_enqueue(w, t)
+    k = n_events
+    return EventStream(np.array(times[:k], dtype=np.float64), np.array(wi[:k], dtype=np.int32),
+                       np.array(wj[:k], dtype=np.int32), np.array(slot[:k], dtype=np.int32),
+                       {"n": n, "seed": seed, "model": "fifo"})
+
+
 # --------------------------------------------------------------------------------------
 # state and gradient rows
 # --------------------------------------------------------------------------------------

@@ -175,3 +175,25 @@ def test_resident_mode_plan_variant_and_limits():
     assert e.value.code == B.A2_EINVAL and "shared memory" in str(e.value)
     big.apply_events([1.0], [0], [1], [-1])  # the batched path takes any n
     big.close()
+
+
+def test_fifo_pairing_stream_with_ties():
+    """The paper's practical event model (availability queue, Sec. 4.1): a gradient completion and
+    the pairing it triggers carry the same time stamp, so zero elapsed times occur all the time."""
+    cfg = W.CONFIGS["cfg3"].scaled(d=4_099, n_events=3000)
+    ev = W.fifo_pairing_events(cfg.n, cfg.edges(), 2.0, cfg.n_events, seed=cfg.seed)
+    assert np.any(np.diff(ev.times) == 0)
+    outs = []
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
+        eng, chk = P.make_small(cfg)
+        if flags == B.A2_SCHED_RESIDENT:
+            eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+            chk.plain.apply_stream(ev)
+            x, xt, t = eng.read_state()
+            chk.compare(P.widen(x, "f32"), P.widen(xt, "f32"), t, where="fifo stream, resident")
+        else:
+            P.run_batches_and_check(eng, chk, ev, flags, every=3)
+        outs.append(eng.read_state())
+        eng.close()
+    for o in outs[1:]:
+        assert all(np.array_equal(u, v) for u, v in zip(outs[0], o))

@@ -168,3 +168,20 @@ def test_resident_schedule_is_one_batch_in_stream_order():
     assert np.array_equal(s.t_final(cfg.n), sim.t)
     with pytest.raises(B.A2Error):
         B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=4)
+
+
+def test_fifo_stream_with_ties_replays_exactly():
+    n, d = 16, 4
+    e = W.ring_edges(n)
+    ev = W.fifo_pairing_events(n, e, 2.0, 2500, seed=3)
+    rng = np.random.default_rng(0)
+    x0, G = rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    ref = OracleSim(x0, 0.3, 0.5, 1.1, 0.05, grads=G)
+    ref.apply_stream(ev)
+    for flags in (0, B.A2_SCHED_FUSE):
+        s = B.Schedule(n, n, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
+        sim = OracleSim(x0, 0.3, 0.5, 1.1, 0.05, grads=G)
+        for b in range(s.num_batches):
+            idx = np.sort(s.batch_events(b))  # stream order inside the batch (times tie)
+            sim.apply(ev.times[idx], ev.wi[idx], ev.wj[idx], ev.slot[idx])
+        assert np.array_equal(sim.X, ref.X) and np.array_equal(sim.Xt, ref.Xt) and np.array_equal(sim.t, ref.t)

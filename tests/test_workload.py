@@ -90,3 +90,36 @@ def test_sample_columns_cover_edges():
     cols = W.sample_columns(10_007, 4096, 50, seed=1)
     assert cols[0] == 0 and cols[-1] == 10_006 and 4095 in cols and 4096 in cols and 8192 in cols
     assert np.all(np.diff(cols) > 0)
+
+
+@pytest.mark.parametrize("graph", ["ring", "exponential", "complete"])
+def test_fifo_pairing_model_pairs_neighbours_uniformly(graph):
+    """App. E.2: with first-come-first-served pairing among available neighbours, the history of
+    communications is close to uniform over the edges (the assumption behind chi_1, chi_2), and
+    every worker does about `comms_per_grad` averagings per gradient."""
+    n, r = 32, 1.0
+    e = W.make_edges(graph, n)
+    ev = W.fifo_pairing_events(n, e, r, 60_000, seed=11)
+    assert np.all(np.diff(ev.times) >= 0)
+    comm = ev.wj >= 0
+    n_grad, n_comm = int((~comm).sum()), int(comm.sum())
+    assert abs(2 * n_comm / n_grad - r) < 0.05  # an averaging counts for both of its workers
+    lo, hi = np.minimum(ev.wi[comm], ev.wj[comm]), np.maximum(ev.wi[comm], ev.wj[comm])
+    key = lo.astype(np.int64) * n + hi
+    ekey = e[:, 0].astype(np.int64) * n + e[:, 1]
+    assert set(np.unique(key)) <= set(ekey)  # only neighbours are paired
+    hist = np.array([(key == k).sum() for k in ekey])
+    m = hist.mean()
+    assert np.all(np.abs(hist - m) < 0.15 * m + 5 * np.sqrt(m))
+    part = np.bincount(np.concatenate([lo, hi]), minlength=n)
+    grads = np.bincount(ev.wi[~comm], minlength=n)
+    assert np.all(np.abs(part / grads - r) < 0.15)
+    # a worker is never in two averagings at once: its communications are at least comm_duration apart
+    for w in (0, n // 2):
+        tw = ev.times[comm & ((ev.wi == w) | (ev.wj == w))]
+        assert np.all(np.diff(tw) >= 0.05 - 1e-12)
+    # gradient completions of a worker are about one unit apart
+    tg = ev.times[(~comm) & (ev.wi == 3)]
+    assert abs(np.diff(tg).mean() - 1.0) < 0.05
+    ev2 = W.fifo_pairing_events(n, e, r, 60_000, seed=11)
+    assert np.array_equal(ev.times, ev2.times) and np.array_equal(ev.wj, ev2.wj)
