@@ -197,3 +197,16 @@ def test_fifo_pairing_stream_with_ties():
         eng.close()
     for o in outs[1:]:
         assert all(np.array_equal(u, v) for u, v in zip(outs[0], o))
+
+
+def test_consensus_study_reproduces_the_papers_qualitative_claim():
+    """Sec. 4.2, Fig. 5(b): on the 64-worker ring, A2CiD2 at one averaging per gradient brings the
+    consensus distance down at least as much as doubling the communication rate does."""
+    from paper_2306_08289_b200 import consensus_study as CS
+
+    res = CS.run_study(n=64, d=4_096, T=200.0, pool=16)
+    final = {(r["comms_per_grad"], r["accelerated"]): np.mean([v for _, v in r["trace"][-3:]]) for r in res}
+    assert final[(2.0, False)] < final[(1.0, False)]          # more communication helps the baseline
+    assert final[(1.0, True)] < final[(1.0, False)] * 0.7     # the momentum helps at equal communication
+    assert final[(1.0, True)] < final[(2.0, False)] * 1.2     # ... about as much as doubling the rate
+    assert final[(2.0, True)] < final[(1.0, True)]
