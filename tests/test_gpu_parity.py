@@ -180,8 +180,11 @@ def test_resident_mode_plan_variant_and_limits():
 def test_fifo_pairing_stream_with_ties():
     """The paper's practical event model (availability queue, Sec. 4.1): a gradient completion and
     the pairing it triggers carry the same time stamp, so zero elapsed times occur all the time."""
-    cfg = W.CONFIGS["cfg3"].scaled(d=4_099, n_events=3000)
-    ev = W.fifo_pairing_events(cfg.n, cfg.edges(), 2.0, cfg.n_events, seed=cfg.seed)
+    from dataclasses import replace
+
+    # ring of 32 at two averagings per gradient; (eta, alpha~) prescribed for exactly these rates
+    cfg = replace(W.CONFIGS["cfg3"].scaled(d=4_099, n_events=3000), edge_rate=None, comms_per_grad=2.0)
+    ev = W.fifo_pairing_events(cfg.n, cfg.edges(), cfg.comms_per_grad, cfg.n_events, seed=cfg.seed)
     assert np.any(np.diff(ev.times) == 0)
     outs = []
     for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
