@@ -267,13 +267,13 @@ void a2cid2_sched_destroy(a2cid2_sched_t* s);
  * ------------------------------------------------------------------------------------------ */
 
 /* For the graph with n nodes and n_edges edges (ei[k], ej[k]) of rates lambda[k] > 0, form the
- * Laplacian of Def. 3.1 and return chi_1 = 1 / lambda_2(Lambda) (Eq. (2), algebraic
+ * Laplacian of the Laplacian definition of Sec. 3.1 and return chi_1 = 1 / lambda_2(Lambda) (the definition of chi_1 in Sec. 3.1, algebraic
  * connectivity) and chi_2 = 1/2 max over edges of the effective resistance
- * (e_i - e_j)^T Lambda^+ (e_i - e_j) (Eq. (3)). A2_EINVAL if the graph is not connected. */
+ * (e_i - e_j)^T Lambda^+ (e_i - e_j) (the definition of chi_2 in Sec. 3.1). A2_EINVAL if the graph is not connected. */
 int a2cid2_graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda,
                      double* chi1, double* chi2);
 
-/* Prop. 3.6: accelerated != 0: eta = 1/(2 sqrt(chi1 chi2)), alpha = 1/2,
+/* the convergence proposition of Sec. 3.4: accelerated != 0: eta = 1/(2 sqrt(chi1 chi2)), alpha = 1/2,
  * alpha~ = 1/2 sqrt(chi1/chi2); accelerated == 0: eta = 0, alpha = alpha~ = 1/2. */
 int a2cid2_prescribe(double chi1, double chi2, int32_t accelerated, double* eta, double* alpha, double* alpha_tilde);
 

@@ -6,5 +6,5 @@ import it; it shares no code with the CUDA library and never imports it.
 
   oracle.sim      OracleSim  -- sequential simulator backed by a2cid2_oracle.c (gcc)
   oracle.sim_np   NumpySim   -- the same steps in NumPy, for tiny cases
-  oracle.spectral Laplacian, chi_1, chi_2 and the parameter prescription of Prop. 3.6
+  oracle.spectral Laplacian, chi_1, chi_2 and the parameter prescription of the convergence proposition of Sec. 3.4
 """

@@ -1,10 +1,10 @@
 """Graph quantities and the parameter prescription -- TEST INFRASTRUCTURE (NumPy/LAPACK).
 
-  laplacian   Lambda = sum_{(i,j) in E} lambda^{ij} (e_i - e_j)(e_i - e_j)^T        (Def. 3.1)
+  laplacian   Lambda = sum_{(i,j) in E} lambda^{ij} (e_i - e_j)(e_i - e_j)^T        (the Laplacian definition of Sec. 3.1)
   chi_1       sup_{|x|=1, x perp 1} 1/(x^T Lambda x) = 1 / lambda_2(Lambda)          (Eq. 2)
   chi_2       1/2 sup_{(i,j) in E} (e_i - e_j)^T Lambda^+ (e_i - e_j)                (Eq. 3)
   prescribe   eta = 1/(2 sqrt(chi_1 chi_2)), alpha = 1/2, alpha~ = 1/2 sqrt(chi_1/chi_2);
-              without acceleration eta = 0, alpha = alpha~ = 1/2                     (Prop. 3.6)
+              without acceleration eta = 0, alpha = alpha~ = 1/2                     (the convergence proposition of Sec. 3.4)
 """
 from __future__ import annotations
 

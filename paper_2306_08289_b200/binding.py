@@ -143,7 +143,7 @@ def prescribe(chi1, chi2, accelerated=True):
 
 def config_params(cfg):
     """(eta, alpha, alpha_tilde) of a workload configuration: the values it fixes outright, else
-    the prescription of Prop. 3.6 evaluated by the library on the configuration's graph."""
+    the prescription of the convergence proposition of Sec. 3.4 evaluated by the library on the configuration's graph."""
     if cfg.fixed_params is not None:
         return tuple(float(v) for v in cfg.fixed_params)
     c1, c2 = graph_chi(cfg.n, cfg.edges(), cfg.rates())

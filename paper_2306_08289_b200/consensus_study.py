@@ -2,7 +2,7 @@
 
 The paper tracks the consensus distance between workers during ImageNet training on a ring of 64
 workers and finds that adding A2CiD2 at one averaging per gradient step lowers it as much as
-doubling the communication rate does (Sec. 4.2 "Consensus improvement", Fig. 5(b)). Neither the
+doubling the communication rate does (Sec. 4.2 "Consensus improvement", the consensus-distance panel of the ImageNet figure). Neither the
 data nor the model are here; this script replays the same comparison with the engine on gradients
 that are fresh zero-mean Gaussian draws (a pool of rows per worker), starting from consensus as the
 paper does (one All-Reduce before training). It is an experiment, not a parity target.
@@ -10,7 +10,7 @@ paper does (one All-Reduce before training). It is an experiment, not a parity t
     python -m paper_2306_08289_b200.consensus_study [--n 64] [--d 262144] [--T 300]
 
 prints, for the baseline (eta = 0, alpha = alpha~ = 1/2) at 1 and 2 averagings per gradient and for
-A2CiD2 (Prop. 3.6 parameters) at 1 and 2, the consensus distance sum_i |x_i - xbar|^2 / d at ten
+A2CiD2 (the convergence proposition of Sec. 3.4 parameters) at 1 and 2, the consensus distance sum_i |x_i - xbar|^2 / d at ten
 common evaluation times.
 """
 from __future__ import annotations

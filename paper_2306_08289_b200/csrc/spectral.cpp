@@ -1,4 +1,4 @@
-// Graph quantities of Sec. 3.1: Laplacian (Def. 3.1), chi_1 (Eq. (2)), chi_2 (Eq. (3)).
+// Graph quantities of Sec. 3.1: Laplacian (the Laplacian definition of Sec. 3.1), chi_1 (the definition of chi_1 in Sec. 3.1), chi_2 (the definition of chi_2 in Sec. 3.1).
 // Dense symmetric eigen-decomposition by cyclic Jacobi rotations (n is the number of workers,
 // at most a few thousand), then the pseudo-inverse through the non-zero eigenpairs.
 #include <algorithm>

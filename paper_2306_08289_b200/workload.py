@@ -8,7 +8,7 @@ What it models, from the paper:
   * the three topologies of the experiments (complete, ring/cycle, exponential), Sec. 4.1
     "Practical implementation" and App. E.1;
   * independent Poisson clocks, rate 1 per worker for gradient events and rate lambda^{ij}
-    per edge for pairwise communications (Assumption 3.1);
+    per edge for pairwise communications (the Poisson-process assumption of Sec. 3.4);
   * "r p2p communications per gradient computation for each worker" with peers picked
     uniformly among neighbours (Sec. 4.1 hyper-parameters, App. E.2): every worker takes
     part in r averagings per unit time, so lambda^{ij} = r / degree on a regular graph.
@@ -206,7 +206,7 @@ def _rng(seed: int, tag: int, row: int = 0) -> np.random.Generator:
 
 def poisson_events(n: int, edges: np.ndarray, rates: np.ndarray, n_events: int, seed: int,
                    grad_rate: float = 1.0, t0: float = 0.0, stream_id: int = 0, grad_pool: int = 1) -> EventStream:
-    """Superposition of independent Poisson clocks (Assumption 3.1): one clock of rate
+    """Superposition of independent Poisson clocks (the Poisson-process assumption of Sec. 3.4): one clock of rate
     `grad_rate` per worker and one of rate rates[e] per edge. The superposition is a Poisson
     process of rate R = n*grad_rate + sum(rates); each event belongs to a clock with
     probability rate/R. Worker i owns the gradient rows i, i + n, ..., i + (grad_pool-1) n and

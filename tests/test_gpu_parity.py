@@ -69,7 +69,7 @@ def test_message_before_mix_variant():
 
 
 def test_baseline_parameters_keep_momentum_equal_to_x():
-    """eta = 0, alpha = alpha~ = 1/2 (Prop. 3.6, non-accelerated): x~ stays a bit-exact copy of x."""
+    """eta = 0, alpha = alpha~ = 1/2 (the convergence proposition of Sec. 3.4, non-accelerated): x~ stays a bit-exact copy of x."""
     cfg = W.CONFIGS["cfg2"].scaled(d=3_000, n_events=2000)
     xs, _ = W.x0_matrix(cfg)
     gs, _ = W.grad_matrix(cfg)
@@ -203,7 +203,7 @@ def test_fifo_pairing_stream_with_ties():
 
 
 def test_consensus_study_reproduces_the_papers_qualitative_claim():
-    """Sec. 4.2, Fig. 5(b): on the 64-worker ring, A2CiD2 at one averaging per gradient brings the
+    """Sec. 4.2, the consensus-distance panel of the ImageNet figure: on the 64-worker ring, A2CiD2 at one averaging per gradient brings the
     consensus distance down at least as much as doubling the communication rate does."""
     from paper_2306_08289_b200 import consensus_study as CS
 

@@ -382,7 +382,7 @@ def test_checker_rejects_bad_events():
         s.apply(*_one([2.0], [1], [-1], [7]))  # slot out of range
 
 
-# ---- spectral quantities: Def. 3.1, Eq. (2), Eq. (3), Prop. 3.6 ---------------------------
+# ---- spectral quantities: the Laplacian definition of Sec. 3.1, the definition of chi_1 in Sec. 3.1, the definition of chi_2 in Sec. 3.1, the convergence proposition of Sec. 3.4 ---------------------------
 @pytest.mark.parametrize("n,lam", [(4, 1.0), (16, 0.5), (32, 2.0), (64, 0.5)])
 def test_ring_closed_forms(n, lam):
     e = W.ring_edges(n)
@@ -411,7 +411,7 @@ def test_laplacian_definition_and_trace():
     L = spectral.laplacian(8, e, lam)
     x = np.random.default_rng(0).standard_normal(8)
     assert abs(x @ L @ x - sum(l * (x[i] - x[j]) ** 2 for (i, j), l in zip(e, lam))) < 1e-12
-    assert abs(np.trace(L) / 2 - lam.sum()) < 1e-12  # Prop. 3.6: Tr(Lambda)/2 communications per unit time
+    assert abs(np.trace(L) / 2 - lam.sum()) < 1e-12  # the convergence proposition of Sec. 3.4: Tr(Lambda)/2 communications per unit time
     assert np.allclose(L @ np.ones(8), 0)
 
 
@@ -428,7 +428,7 @@ def test_printed_chi_values_n16():
         e = W.make_edges(g, 16)
         _, _, _, h1, h2 = spectral.prescribe(16, e, W.edge_rates_per_worker(16, e, 1.0))
         assert round(h1) == c1 and round(h2) == c2, (g, h1, h2)
-        assert h2 <= h1 * (1 + 1e-12)  # Eq. (3): chi_2 <= chi_1
+        assert h2 <= h1 * (1 + 1e-12)  # the definition of chi_2 in Sec. 3.1: chi_2 <= chi_1
 
 
 def test_prescription_formulas():

@@ -1,4 +1,4 @@
-"""The input generator against the paper's model: Assumption 3.1 (Poisson clocks), Prop. 3.6
+"""The input generator against the paper's model: the Poisson-process assumption of Sec. 3.4 (Poisson clocks), the convergence proposition of Sec. 3.4
 (expected counts), App. E.2 (uniform pairing among neighbours), App. E.1 (topologies)."""
 import numpy as np
 import pytest
