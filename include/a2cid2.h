@@ -5,7 +5,8 @@
  * parameter row x_i and a continuous-momentum row x~_i (stacked [n, d] device buffers) and a
  * last-event time t_i. Events arrive as a time-sorted stream and are applied as the paper
  * "A2CiD2: Accelerating Asynchronous Communication in Decentralized Deep Learning" defines
- * them (Sec. 3.2, Eq. (dynamic); Algorithm 1):
+ * them (Sec. 3.2 "Training dynamic": the SDE for dx^i_t, dx~^i_t, cited below as Eq. (dynamic) after its
+ * label in the paper's source; Algorithm 1):
  *
  *   mixing    before any update of worker w at time t, (x_w, x~_w) is advanced over t - t_w by
  *             the flow dx = eta (x~ - x) dt, dx~ = eta (x - x~) dt, in closed form:
@@ -267,13 +268,13 @@ void a2cid2_sched_destroy(a2cid2_sched_t* s);
  * ------------------------------------------------------------------------------------------ */
 
 /* For the graph with n nodes and n_edges edges (ei[k], ej[k]) of rates lambda[k] > 0, form the
- * Laplacian of the Laplacian definition of Sec. 3.1 and return chi_1 = 1 / lambda_2(Lambda) (the definition of chi_1 in Sec. 3.1, algebraic
+ * Laplacian as Sec. 3.1 defines it and return chi_1 = 1 / lambda_2(Lambda) (the definition of chi_1 in Sec. 3.1, algebraic
  * connectivity) and chi_2 = 1/2 max over edges of the effective resistance
  * (e_i - e_j)^T Lambda^+ (e_i - e_j) (the definition of chi_2 in Sec. 3.1). A2_EINVAL if the graph is not connected. */
 int a2cid2_graph_chi(int32_t n, int64_t n_edges, const int32_t* ei, const int32_t* ej, const double* lambda,
                      double* chi1, double* chi2);
 
-/* the convergence proposition of Sec. 3.4: accelerated != 0: eta = 1/(2 sqrt(chi1 chi2)), alpha = 1/2,
+/* Parameters of the convergence proposition of Sec. 3.4: accelerated != 0: eta = 1/(2 sqrt(chi1 chi2)), alpha = 1/2,
  * alpha~ = 1/2 sqrt(chi1/chi2); accelerated == 0: eta = 0, alpha = alpha~ = 1/2. */
 int a2cid2_prescribe(double chi1, double chi2, int32_t accelerated, double* eta, double* alpha, double* alpha_tilde);
 
