@@ -169,10 +169,8 @@ def cpu_baseline(cfg, ev, n_cols, threads):
     return len(ev) / dt * (n_cols / cfg.d), dt, cons
 
 
-def run_reference(args, cfg, ranks):
+def run_reference(args, cfg):
     """Reference arm: the CPU checker on the host cores (rank 0 only)."""
-    if ranks.rank != 0:
-        return
     threads = max(1, min(os.cpu_count() or 1, 32))
     n_cols = args.cpu_sample_cols or max(1, min(cfg.d, 256_000))
     eps = args.events_per_step
@@ -214,9 +212,9 @@ def main():
     if args.d is not None:
         cfg = cfg.scaled(d=args.d, name=f"{cfg.name}-d{args.d}")
     if args.impl == "reference":
-        ranks = Ranks(backend="gloo")
-        run_reference(args, cfg, ranks)
-        ranks.close()
+        # rank 0 alone times the CPU checker; the other ranks have nothing to do and no group is formed
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, cfg)
         return
 
     import torch

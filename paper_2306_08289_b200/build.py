@@ -36,6 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-Xcompiler", "-fPIC,-O2,-Wall", "-shared", "-cudart", "static",
            "-I", INCLUDE, "-I", CSRC, "-o", tmp]
+    cmd += os.environ.get("A2CID2_NVCC_FLAGS", "").split()  # extra flags for experiments, e.g. -DA2_EVENT_THREADS=512
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]

@@ -39,6 +39,10 @@ namespace a2 {
 namespace {
 
 constexpr int kThreads = 256;
+#ifndef A2_EVENT_THREADS
+#define A2_EVENT_THREADS 256
+#endif
+constexpr int kEventThreads = A2_EVENT_THREADS;  // threads per CTA of the event kernel
 
 // ---------------------------------------------------------------------------------------------
 // Vector access for the two storage types: BYTES = 32 (256-bit ld/st.global.v8, the widest
@@ -180,7 +184,7 @@ struct EventArgs {
 };
 
 template <typename T, int BYTES, int UNROLL>
-__global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
+__global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
@@ -188,8 +192,8 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
     __shared__ float s_cb[kMaxOpsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
 
-    for (int i = threadIdx.x; i < p.n_items; i += kThreads) s_items[i] = p.items[i];
-    for (int o = threadIdx.x; o < p.n_ops; o += kThreads) {
+    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
         const DevOp op = p.ops[o];
         s_kind[o] = (unsigned char)op.kind;
         s_ca[o] = (op.kind != A2_OP_GRAD_B) ? (float)mix_coeff(p.eta, op.t - op.t_prev_a) : 0.f;
@@ -208,7 +212,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
         const long long tile = unit / p.n_items;
         const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
-        const long long v0 = tile * (long long)(kThreads * UNROLL) + threadIdx.x;
+        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
 
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxta = Xt + (long long)it.a * p.pitch;
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
         bool live[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const long long v = v0 + (long long)u * kThreads;
+            const long long v = v0 + (long long)u * kEventThreads;
             live[u] = v < p.n_vec;
             const long long off = v * N;
 #pragma unroll
@@ -268,7 +272,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_events(const EventArgs p) {
 
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const long long off = (v0 + (long long)u * kThreads) * N;
+            const long long off = (v0 + (long long)u * kEventThreads) * N;
             if (live[u]) {
                 V::store(pxa + off, xa[u]);
                 V::store(pxta + off, xta[u]);
@@ -377,7 +381,7 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
     a.n_vec = (L.d + N - 1) / N;
     a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
-    const long long vec_per_tile = (long long)kThreads * U;
+    const long long vec_per_tile = (long long)kEventThreads * U;
     a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
@@ -386,7 +390,7 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     long long grid = (long long)dev.sm_count * per_sm;
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events<T, BYTES, U><<<(unsigned)grid, kThreads, 0, stream>>>(a);
+    k_apply_events<T, BYTES, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -402,7 +406,7 @@ template <typename T, int BYTES>
 cudaError_t event_occupancy(int* out) {
     int occ = 0;
     const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL>, kThreads, 0);
+        &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL>, kEventThreads, 0);
     *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
     return e;
 }
