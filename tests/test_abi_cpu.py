@@ -89,3 +89,43 @@ def test_create_validates_without_a_device():
     assert L.a2cid2_sync(h) == B.A2_OK
     L.a2cid2_destroy(h)
     L.a2cid2_destroy(None)
+
+
+def test_header_is_plain_c_and_a_c_program_links_against_the_library(tmp_path):
+    """The boundary is a C ABI: the header compiles as strict C99 and a C program that only uses
+    host-side entry points (no device needed) links against the shared library and runs."""
+    import subprocess
+
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-fsyntax-only", "-x", "c", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror",
+                    os.path.join(inc, "a2cid2.h")], check=True)
+    src = tmp_path / "use_abi.c"
+    src.write_text(r"""
+#include <stdio.h>
+#include "a2cid2.h"
+int main(void) {
+    int32_t ei[4] = {0, 1, 2, 0}, ej[4] = {1, 2, 3, 3};
+    double lam[4] = {1.0, 1.0, 1.0, 1.0}, c1, c2, eta, alpha, at;
+    if (a2cid2_graph_chi(4, 4, ei, ej, lam, &c1, &c2) != A2_OK) return 1;
+    if (a2cid2_prescribe(c1, c2, 1, &eta, &alpha, &at) != A2_OK) return 2;
+    double times[3] = {0.5, 1.0, 1.5};
+    int32_t wi[3] = {0, 2, 1}, wj[3] = {1, 3, 2}, slot[3] = {-1, -1, -1};
+    a2cid2_sched_t* s = 0;
+    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, A2_SCHED_FUSE, 0, &s) != A2_OK) return 3;
+    long long nb = (long long)a2cid2_sched_num_batches(s);
+    a2cid2_sched_destroy(s);
+    wi[0] = 7;  /* out of range: rejected with a message */
+    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, 0, 0, &s) != A2_ERANGE) return 4;
+    printf("%.6f %.6f %.6f %.6f %lld %s|%s\n", c1, c2, eta, at, nb, a2cid2_last_error(0), a2cid2_version());
+    return 0;
+}
+""")
+    exe = tmp_path / "use_abi"
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), "-L", libdir, "-la2cid2",
+                    f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()
+    c1, c2, eta, at = (float(v) for v in out[:4])
+    # ring of 4 with unit rates: chi_1 = 1/2, chi_2 = 3/8
+    assert abs(c1 - 0.5) < 1e-6 and abs(c2 - 0.375) < 1e-6 and abs(eta - 1 / (2 * math.sqrt(c1 * c2))) < 1e-5
+    assert int(out[4]) == 2 and "out of range" in " ".join(out[5:])
