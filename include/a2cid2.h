@@ -198,7 +198,8 @@ int a2cid2_sync(a2cid2_t* h);
 const char* a2cid2_last_error(const a2cid2_t* h);
 
 /* Release the handle and everything the library allocated for it (waits for the stream).
- * Plans created from it must be destroyed first. NULL is allowed. */
+ * Plans created from it should be destroyed first; one that is still alive stays valid only as an
+ * argument of a2cid2_plan_destroy. NULL is allowed. */
 void a2cid2_destroy(a2cid2_t* h);
 
 /* ------------------------------------------------------------------------------------------

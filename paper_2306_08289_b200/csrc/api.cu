@@ -70,7 +70,7 @@ struct a2cid2 {
     double* h_pinned = nullptr;    // n + 1 doubles: dt staging and the result
     Arena arena[2];
     int arena_next = 0;
-    int64_t live_plans = 0;
+    std::vector<a2cid2_plan*> plans;  // live plans made from this handle
     std::string err;
 };
 
@@ -487,8 +487,10 @@ int a2cid2_sync(a2cid2_t* h) {
 
 void a2cid2_destroy(a2cid2_t* h) {
     if (!h) return;
+    if (h->dev_ok) cudaStreamSynchronize(h->stream);
+    // plans that outlive the handle keep their memory until a2cid2_plan_destroy, but can no longer run
+    for (a2cid2_plan* p : h->plans) p->owner = nullptr;
     if (h->dev_ok) {
-        cudaStreamSynchronize(h->stream);
         for (Arena& A : h->arena) {
             if (A.host) cudaFreeHost(A.host);
             if (A.dev) cudaFree(A.dev);
@@ -560,7 +562,7 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
             return fail_cuda(h, e, "plan descriptor upload");
         }
     }
-    h->live_plans += 1;
+    h->plans.push_back(p);
     *out = p;
     return A2_OK;
 }
@@ -597,7 +599,9 @@ void a2cid2_plan_destroy(a2cid2_plan_t* p) {
     if (!p) return;
     if (p->owner) {
         if (p->owner->dev_ok) cudaStreamSynchronize(p->owner->stream);  // queued kernels may still read the descriptors
-        p->owner->live_plans -= 1;
+        std::vector<a2cid2_plan*>& v = p->owner->plans;
+        for (size_t k = 0; k < v.size(); ++k)
+            if (v[k] == p) { v.erase(v.begin() + (long)k); break; }
     }
     if (p->d_desc) cudaFree(p->d_desc);
     a2cid2_sched_destroy(p->sched);

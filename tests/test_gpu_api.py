@@ -246,3 +246,14 @@ def test_many_items_per_batch_are_split_into_launches():
     x, xt, t = eng.read_state()
     assert P.rel_err(x, sim.X) <= 1e-5 and P.rel_err(xt, sim.Xt) <= 1e-5 and np.array_equal(t, sim.t)
     eng.close()
+
+
+def test_plan_may_outlive_its_engine():
+    cfg = _small(n_events=100)
+    ev = W.config_events(cfg)
+    eng, _ = P.make_small(cfg)
+    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot)
+    q = eng.plan(ev.times, ev.wi, ev.wj, ev.slot)
+    q.close()
+    eng.close()  # p is still alive: it may only be destroyed now
+    p.close()
