@@ -381,6 +381,11 @@ def main():
             "value": v, "unit": "events/s", "cores": cores, "kind": "oracle", "seconds": dt,
             "sample": f"first {n_cols} of {cfg.d} columns, all {cfg.n} workers, {4 * eps} events + one consensus "
                       f"distance; events/s scaled by the column fraction"}
+        # the same checker strictly sequential on one thread, on a smaller slice
+        n1 = max(1, min(cfg.d, n_cols // 10))
+        v1, dt1, _ = cpu_baseline(cfg, W.config_events(cfg, n_events=eps), n1, 1)
+        line["cpu_baseline"]["one_thread"] = {"value": v1, "seconds": dt1,
+                                              "sample": f"first {n1} columns, {eps} events + one consensus distance"}
     eng.close()
     if ranks.rank == 0:
         print(json.dumps(line), flush=True)
