@@ -285,101 +285,6 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     }
 }
 
-// bf16 rows with 256-bit accesses: the 16 elements a thread holds per row stay packed (two per
-// register) and are widened, updated and re-packed one register at a time, so that the wide loads do
-// not cost the occupancy the bf16 path needs. The operations of an item are applied to each pair in
-// turn; values stay in fp32 from the first operation of the item to the last, as everywhere else.
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-__device__ __forceinline__ uint32_t bf16_pack(float lo, float hi) {
-    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&h);
-}
-
-__global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_wide(const EventArgs p) {
-    constexpr int WORDS = 8;       // 32 bytes per row per thread
-    constexpr int N = 2 * WORDS;   // elements
-    __shared__ DevItem s_items[kMaxItemsPerLaunch];
-    __shared__ float s_ca[kMaxOpsPerLaunch];
-    __shared__ float s_cb[kMaxOpsPerLaunch];
-    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
-
-    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
-    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
-        const DevOp op = p.ops[o];
-        s_kind[o] = (unsigned char)op.kind;
-        s_ca[o] = (op.kind != A2_OP_GRAD_B) ? (float)mix_coeff(p.eta, op.t - op.t_prev_a) : 0.f;
-        s_cb[o] = (op.kind != A2_OP_GRAD_A) ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
-    }
-    __syncthreads();
-
-    __nv_bfloat16* const X = static_cast<__nv_bfloat16*>(p.x);
-    __nv_bfloat16* const Xt = static_cast<__nv_bfloat16*>(p.xt);
-    const __nv_bfloat16* const G = static_cast<const __nv_bfloat16*>(p.g);
-    const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
-    const bool before = p.msg_before_mix != 0;
-    const long long n_units = (long long)p.n_items * p.n_tiles;
-
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int item_idx = (int)(unit % p.n_items);
-        const long long tile = unit / p.n_items;
-        const DevItem it = s_items[item_idx];
-        const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
-        const long long v = tile * (long long)kEventThreads + threadIdx.x;
-        if (v >= p.n_vec) continue;
-        const long long off = v * N;
-        __nv_bfloat16* const pxa = X + (long long)it.a * p.pitch + off;
-        __nv_bfloat16* const pxta = Xt + (long long)it.a * p.pitch + off;
-        __nv_bfloat16* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch + off;
-        __nv_bfloat16* const pxtb = Xt + (long long)(has_b ? it.b : it.a) * p.pitch + off;
-
-        uint32_t wa[WORDS], wta[WORDS], wb[WORDS], wtb[WORDS], wga[WORDS], wgb[WORDS];
-#pragma unroll
-        for (int k = 0; k < WORDS; ++k) { wb[k] = 0u; wtb[k] = 0u; wga[k] = 0u; wgb[k] = 0u; }
-        ld_u32x8(pxa, wa);
-        ld_u32x8(pxta, wta);
-        if (has_b) {
-            ld_u32x8(pxb, wb);
-            ld_u32x8(pxtb, wtb);
-        }
-        if (has_ga) ld_u32x8(G + (long long)it.slot_a * p.pitch + off, wga);
-        if (has_gb) ld_u32x8(G + (long long)it.slot_b * p.pitch + off, wgb);
-
-#pragma unroll
-        for (int k = 0; k < WORDS; ++k) {
-            float xa0 = bf16_lo(wa[k]), xa1 = bf16_hi(wa[k]), xta0 = bf16_lo(wta[k]), xta1 = bf16_hi(wta[k]);
-            float xb0 = bf16_lo(wb[k]), xb1 = bf16_hi(wb[k]), xtb0 = bf16_lo(wtb[k]), xtb1 = bf16_hi(wtb[k]);
-            const float ga0 = bf16_lo(wga[k]), ga1 = bf16_hi(wga[k]), gb0 = bf16_lo(wgb[k]), gb1 = bf16_hi(wgb[k]);
-            for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
-                const int kind = s_kind[o];
-                if (kind == A2_OP_GRAD_A) {
-                    const float c = s_ca[o];
-                    grad_elem(xa0, xta0, c, ngamma, ga0);
-                    grad_elem(xa1, xta1, c, ngamma, ga1);
-                } else if (kind == A2_OP_GRAD_B) {
-                    const float c = s_cb[o];
-                    grad_elem(xb0, xtb0, c, ngamma, gb0);
-                    grad_elem(xb1, xtb1, c, ngamma, gb1);
-                } else {
-                    const float ca = s_ca[o], cb = s_cb[o];
-                    comm_elem<false>(xa0, xta0, xb0, xtb0, ca, cb, alpha, alpha_t, before);
-                    comm_elem<false>(xa1, xta1, xb1, xtb1, ca, cb, alpha, alpha_t, before);
-                }
-            }
-            wa[k] = bf16_pack(xa0, xa1);
-            wta[k] = bf16_pack(xta0, xta1);
-            wb[k] = bf16_pack(xb0, xb1);
-            wtb[k] = bf16_pack(xtb0, xtb1);
-        }
-        st_u32x8(pxa, wa);
-        st_u32x8(pxta, wta);
-        if (has_b) {
-            st_u32x8(pxb, wb);
-            st_u32x8(pxtb, wtb);
-        }
-    }
-}
-
 // Vectors per thread and tile. 256-bit accesses: one vector per thread already keeps 4-6 rows x 32 B
 // in flight per thread; 128-bit fp32 uses two.
 template <typename T, int BYTES> struct EventCfg { static constexpr int UNROLL = 1; };
@@ -497,28 +402,6 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
 template <typename T> struct EventCtas { static constexpr int PER_SM = 2; };
 template <> struct EventCtas<__nv_bfloat16> { static constexpr int PER_SM = 4; };
 
-bool bf16_rows_32B_aligned(const void* a, const void* b, const void* c, int64_t pitch) {
-    static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
-    const uintptr_t bits = reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c);
-    return !force_narrow && (bits % 32 == 0) && ((pitch * 2) % 32 == 0);
-}
-
-int launch_events_bf16_wide(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
-    EventArgs a;
-    a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
-    a.n_vec = (L.d + 15) / 16;
-    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
-    a.n_tiles = (int)((a.n_vec + kEventThreads - 1) / kEventThreads);
-    a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
-    a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
-    const long long n_units = (long long)a.n_items * a.n_tiles;
-    long long grid = (long long)dev.sm_count * dev.event_ctas_per_sm[1][1];
-    if (grid > n_units) grid = n_units;
-    if (grid < 1) return 0;
-    k_apply_events_bf16_wide<<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
-    return (int)cudaGetLastError();
-}
-
 template <typename T, int BYTES>
 cudaError_t event_occupancy(int* out) {
     int occ = 0;
@@ -561,12 +444,7 @@ int query_device(DeviceInfo* info) {
     if ((e = event_occupancy<float, 16>(&info->event_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<float, 32>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<__nv_bfloat16, 16>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
-    {
-        int occ = 0;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_bf16_wide, kEventThreads, 0)) != cudaSuccess)
-            return (int)e;
-        info->event_ctas_per_sm[1][1] = occ > 0 ? occ : 1;
-    }
+    info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
     info->consensus_ctas_per_sm = 4;
     if (const char* v = std::getenv("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
         const int k = std::atoi(v);
@@ -581,10 +459,7 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.n_items <= 0) return 0;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
-    if (L.dtype == A2_BF16) {
-        if (bf16_rows_32B_aligned(L.x, L.xt, L.g, L.pitch)) return launch_events_bf16_wide(L, dev, stream);
-        return launch_events_t<__nv_bfloat16, 16>(L, dev, stream);
-    }
+    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16>(L, dev, stream);
     return wide ? launch_events_t<float, 32>(L, dev, stream) : launch_events_t<float, 16>(L, dev, stream);
 }
 
