@@ -118,8 +118,16 @@ template <int BYTES> struct Vec<__nv_bfloat16, BYTES> {
 };
 
 // Gradient event on one element: mixing over the elapsed time, then -gamma g on both buffers.
+// ONE_ROUNDING (fp32 storage) adds mixing term and jump as a single increment; with bf16 storage the
+// store's rounding dwarfs that refinement and the plain two-step form saves instructions.
+template <bool ONE_ROUNDING>
 __device__ __forceinline__ void grad_elem(float& x, float& xt, float c, float ngamma, float g) {
     const float dlt = __fsub_rn(x, xt);
+    if (!ONE_ROUNDING) {
+        x = __fmaf_rn(ngamma, g, __fmaf_rn(-c, dlt, x));
+        xt = __fmaf_rn(ngamma, g, __fmaf_rn(c, dlt, xt));
+        return;
+    }
     const float tg = __fmul_rn(ngamma, g);
     x = __fadd_rn(x, __fmaf_rn(-c, dlt, tg));
     xt = __fadd_rn(xt, __fmaf_rn(c, dlt, tg));
@@ -133,13 +141,17 @@ __device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, floa
                                           float alpha, float alpha_t, bool msg_before_mix) {
     const float ua = __fmul_rn(-ca, __fsub_rn(xa, xta));
     const float ub = __fmul_rn(-cb, __fsub_rn(xb, xtb));
-    if (!COMPENSATED) {
-        const float d0 = __fsub_rn(xa, xb);
-        const float m0 = msg_before_mix ? d0 : __fadd_rn(d0, __fsub_rn(ua, ub));
-        xa = __fadd_rn(xa, __fmaf_rn(-alpha, m0, ua));
-        xta = __fadd_rn(xta, __fmaf_rn(-alpha_t, m0, -ua));
-        xb = __fadd_rn(xb, __fmaf_rn(alpha, m0, ub));
-        xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m0, -ub));
+    if (!COMPENSATED) {  // plain two-step form: mix both workers, take the message, jump
+        const float m_pre = __fsub_rn(xa, xb);
+        xa = __fadd_rn(xa, ua);
+        xta = __fsub_rn(xta, ua);
+        xb = __fadd_rn(xb, ub);
+        xtb = __fsub_rn(xtb, ub);
+        const float m0 = msg_before_mix ? m_pre : __fsub_rn(xa, xb);
+        xa = __fmaf_rn(-alpha, m0, xa);
+        xta = __fmaf_rn(-alpha_t, m0, xta);
+        xb = __fmaf_rn(alpha, m0, xb);
+        xtb = __fmaf_rn(alpha_t, m0, xtb);
         return;
     }
     // raw + e_raw == x_a - x_b exactly (two-sum)
@@ -207,9 +219,13 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
     const long long n_units = (long long)p.n_items * p.n_tiles;
 
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int item_idx = (int)(unit % p.n_items);
-        const long long tile = unit / p.n_items;
+    // unit -> (item = unit % n_items, tile = unit / n_items), advanced incrementally: one division per launch
+    int item_idx = (int)(blockIdx.x % (unsigned)p.n_items);
+    long long tile = blockIdx.x / (unsigned)p.n_items;
+    const int step_item = (int)(gridDim.x % (unsigned)p.n_items);
+    const long long step_tile = gridDim.x / (unsigned)p.n_items;
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x, item_idx += step_item, tile += step_tile) {
+        if (item_idx >= p.n_items) { item_idx -= p.n_items; tile += 1; }
         const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
         const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
@@ -228,9 +244,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
             const long long v = v0 + (long long)u * kEventThreads;
             live[u] = v < p.n_vec;
             const long long off = v * N;
-#pragma unroll
-            for (int k = 0; k < N; ++k) { xb[u][k] = 0.f; xtb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
-            if (live[u]) {
+            if (live[u]) {  // rows an item does not have are never read by its operations, nor stored
                 V::load(pxa + off, xa[u]);
                 V::load(pxta + off, xta[u]);
                 if (has_b) {
@@ -239,9 +253,6 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 }
                 if (has_ga) V::load(pga + off, ga[u]);
                 if (has_gb) V::load(pgb + off, gb[u]);
-            } else {
-#pragma unroll
-                for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xta[u][k] = 0.f; }
             }
         }
 
@@ -252,13 +263,13 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-                    for (int k = 0; k < N; ++k) grad_elem(xa[u][k], xta[u][k], c, ngamma, ga[u][k]);
+                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], c, ngamma, ga[u][k]);
             } else if (kind == A2_OP_GRAD_B) {
                 const float c = s_cb[o];
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-                    for (int k = 0; k < N; ++k) grad_elem(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
+                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
             } else {
                 const float ca = s_ca[o], cb = s_cb[o];
 #pragma unroll
@@ -579,7 +590,7 @@ __global__ void __launch_bounds__(kResidentCols) k_resident(const ResidentArgs p
                         sX[b * kResidentCols] = xb;
                         sXt[b * kResidentCols] = xtb;
                     } else {
-                        grad_elem(xa, xta, ca, ngamma, sG[gi * kResidentCols]);
+                        grad_elem<sizeof(T) == 4>(xa, xta, ca, ngamma, sG[gi * kResidentCols]);
                     }
                     sX[a * kResidentCols] = xa;
                     sXt[a * kResidentCols] = xta;
