@@ -74,7 +74,7 @@ enum {
 };
 
 /* Kinds of elementary operation inside an item. */
-enum { A2_OP_GRAD_A = 0, A2_OP_GRAD_B = 1, A2_OP_COMM = 2 };
+enum { A2_OP_GRAD_A = 0, A2_OP_GRAD_B = 1, A2_OP_COMM = 2, A2_OP_MIX_A = 3 /* mixing only (a2cid2_flush) */ };
 
 /* Variants of the order of operations at a communication event. */
 enum {
@@ -152,6 +152,13 @@ int a2cid2_set_times(a2cid2_t* h, const double* host_t);
  * kernel per batch is queued on the bound stream. stats may be NULL. Asynchronous. */
 int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, const int32_t* wi,
                         const int32_t* wj, const int32_t* grad_slot, uint32_t flags, a2cid2_stats* stats);
+
+/* Bring every worker to the common time t_flush >= max_i t_i: the mixing flow is applied to each
+ * (x_i, x~_i) over t_flush - t_i and t_i = t_flush is recorded; no gradient, no averaging. This is the
+ * state Algorithm 1 returns at the end of training (x_T), and the one at which mean(x) = mean(x~)
+ * holds (Eq. (mean)). One kernel launch on the bound stream; asynchronous. A2_EORDER if t_flush
+ * precedes a worker's time. */
+int a2cid2_flush(a2cid2_t* h, double t_flush);
 
 /* Consensus distance sum_i |x_i - xbar|^2, xbar = (1/n) sum_i x_i (App. A). With t_eval = NaN
  * the stored rows are used as they are (each at its own t_i). With a finite

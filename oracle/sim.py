@@ -107,6 +107,14 @@ class OracleSim:
     def apply_stream(self, ev, threads=1):
         self.apply(ev.times, ev.wi, ev.wj, ev.slot, threads=threads)
 
+    def flush(self, t_flush):
+        """Every worker mixed forward to the common time t_flush, in place: the state Algorithm 1
+        returns at the end of training."""
+        if np.any(self.t > t_flush):
+            raise OracleError("flush time precedes a worker's last event")
+        self.X, self.Xt = self.flushed(t_flush)
+        self.t[:] = t_flush
+
     def round_rows(self, workers):
         """Model of bf16 *storage*: the rows of these workers are rounded to bfloat16, as happens
         whenever an implementation that keeps its state in bf16 writes them back. The arithmetic

@@ -20,7 +20,7 @@ A2_OK, A2_EINVAL, A2_EORDER, A2_ERANGE, A2_ENOMEM, A2_ECUDA, A2_ESTATE = 0, -1, 
 A2_F32, A2_BF16 = 0, 1
 A2_SCHED_FUSE = 1
 A2_SCHED_RESIDENT = 2
-A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM = 0, 1, 2
+A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A = 0, 1, 2, 3
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX = 0, 1
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
@@ -64,6 +64,7 @@ SIGNATURES = {
     "a2cid2_times": (C.c_int, [_vp, _dp]),
     "a2cid2_set_times": (C.c_int, [_vp, _dp]),
     "a2cid2_apply_events": (C.c_int, [_vp, C.c_int64, _dp, _ip, _ip, _ip, C.c_uint32, C.POINTER(Stats)]),
+    "a2cid2_flush": (C.c_int, [_vp, C.c_double]),
     "a2cid2_consensus_distance": (C.c_int, [_vp, C.c_double, _dp]),
     "a2cid2_consensus_distance_static": (C.c_int, [_vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, _vp, _vp]),
     "a2cid2_sync": (C.c_int, [_vp]),
@@ -360,6 +361,9 @@ class Engine:
         _check(lib().a2cid2_plan_create(self._h, None if ts is None else _ptr(ts, _dp), len(times), _ptr(times, _dp),
                                         _ptr(wi, _ip), _ptr(wj, _ip), _ptr(slot, _ip), flags, C.byref(p)), self._h)
         return Plan(self, p)
+
+    def flush(self, t_flush):
+        _check(lib().a2cid2_flush(self._h, float(t_flush)), self._h)
 
     def consensus_distance(self, t_eval=None):
         out = C.c_double()

@@ -271,7 +271,7 @@ void advance_times(const a2cid2_sched& s, int64_t b0, int64_t b1, std::vector<do
         for (int32_t o = 0; o < it.n_ops; ++o) {
             const a2::SchedOp& op = s.ops[(size_t)(it.first_op + o)];
             if (op.kind != A2_OP_GRAD_B) t[(size_t)it.a] = op.t;
-            if (op.kind != A2_OP_GRAD_A) t[(size_t)it.b] = op.t;
+            if (op.kind == A2_OP_GRAD_B || op.kind == A2_OP_COMM) t[(size_t)it.b] = op.t;
         }
     }
 }
@@ -399,17 +399,10 @@ int a2cid2_set_times(a2cid2_t* h, const double* host_t) {
     return A2_OK;
 }
 
-int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, const int32_t* wi, const int32_t* wj,
-                        const int32_t* grad_slot, uint32_t flags, a2cid2_stats* stats) {
-    int rc = need_bound(h);
-    if (rc != A2_OK) return rc;
-    const double t0 = now_ms();
-    a2cid2_sched* s = nullptr;
-    std::string err;
-    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, &s, err);
-    if (rc != A2_OK) return fail(h, rc, err);
+// Lay out, upload and queue a whole schedule through the handle's staging buffers; takes ownership of s.
+static int submit_schedule(a2cid2* h, a2cid2_sched* s, a2cid2_stats* stats, double t0) {
     Packed pk;
-    rc = plan_layout(h, *s, pk);
+    int rc = plan_layout(h, *s, pk);
     if (rc != A2_OK) { a2cid2_sched_destroy(s); return rc; }
     const int64_t nb = (int64_t)s->batch_first.size() - 1;
     if (stats) std::memset(stats, 0, sizeof *stats);
@@ -453,6 +446,41 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
     h->t = s->t_final;
     a2cid2_sched_destroy(s);
     return A2_OK;
+}
+
+int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, const int32_t* wi, const int32_t* wj,
+                        const int32_t* grad_slot, uint32_t flags, a2cid2_stats* stats) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    const double t0 = now_ms();
+    a2cid2_sched* s = nullptr;
+    std::string err;
+    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, &s, err);
+    if (rc != A2_OK) return fail(h, rc, err);
+    return submit_schedule(h, s, stats, t0);
+}
+
+int a2cid2_flush(a2cid2_t* h, double t_flush) {
+    int rc = need_bound(h);
+    if (rc != A2_OK) return rc;
+    if (!std::isfinite(t_flush)) return fail(h, A2_EINVAL, "t_flush must be finite");
+    for (int32_t w = 0; w < h->n; ++w)
+        if (t_flush < h->t[(size_t)w]) return fail(h, A2_EORDER, "t_flush precedes a worker's last event");
+    a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
+    if (!s) return fail(h, A2_ENOMEM, "out of host memory");
+    s->n = h->n;
+    s->n_grad_slots = h->n_slots;
+    s->t_start = h->t;
+    s->t_final = h->t;
+    for (int32_t w = 0; w < h->n; ++w) {  // one batch: a mixing-only item per worker that is behind
+        if (h->t[(size_t)w] == t_flush) continue;
+        s->items.push_back(a2::SchedItem{w, -1, -1, -1, (int64_t)s->ops.size(), 1, 0});
+        s->ops.push_back(a2::SchedOp{-1, A2_OP_MIX_A, t_flush, h->t[(size_t)w], 0.0});
+        s->t_final[(size_t)w] = t_flush;
+    }
+    s->batch_first.assign(1, 0);
+    if (!s->items.empty()) s->batch_first.push_back((int64_t)s->items.size());
+    return submit_schedule(h, s, nullptr, now_ms());
 }
 
 int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out) {

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
         const DevOp op = p.ops[o];
         s_kind[o] = (unsigned char)op.kind;
         s_ca[o] = (op.kind != A2_OP_GRAD_B) ? (float)mix_coeff(p.eta, op.t - op.t_prev_a) : 0.f;
-        s_cb[o] = (op.kind != A2_OP_GRAD_A) ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
+        s_cb[o] = (op.kind == A2_OP_GRAD_B || op.kind == A2_OP_COMM) ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
     }
     __syncthreads();
 
@@ -285,6 +285,12 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
                     for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
+            } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
+                const float c = s_ca[o];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], c, ngamma, 0.f);
             } else {
                 const float ca = s_ca[o], cb = s_cb[o];
 #pragma unroll

@@ -230,6 +230,7 @@ void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, in
         for (int32_t o = 0; o < it.n_ops; ++o) {
             const int32_t kind = s.ops[(size_t)(it.first_op + o)].kind;
             if (kind == A2_OP_COMM) { st.n_comm += 1; rows_single += 8; }
+            else if (kind == A2_OP_MIX_A) { rows_single += 4; }
             else { st.n_grad += 1; rows_single += 5; }
         }
     }

@@ -213,3 +213,38 @@ def test_consensus_study_reproduces_the_papers_qualitative_claim():
     assert final[(1.0, True)] < final[(1.0, False)] * 0.7     # the momentum helps at equal communication
     assert final[(1.0, True)] < final[(2.0, False)] * 1.2     # ... about as much as doubling the rate
     assert final[(2.0, True)] < final[(1.0, True)]
+
+
+@pytest.mark.parametrize("storage", ["f32", "bf16"])
+def test_flush_brings_every_worker_to_a_common_time(storage):
+    """a2cid2_flush applies the mixing flow alone; afterwards mean(x) = mean(x~) (Eq. (mean)), which
+    does not hold for the lazily stored state."""
+    name = "cfg3" if storage == "f32" else "cfg5"
+    cfg = W.CONFIGS[name].scaled(d=5_005, n_events=1500)
+    ev = W.config_events(cfg)
+    eng, chk = P.make_small(cfg)
+    eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    chk.plain.apply_stream(ev)
+    t_end = float(ev.times[-1]) + 0.75
+    with pytest.raises(B.A2Error) as e:
+        eng.flush(float(ev.times[-1]) - 1.0)
+    assert e.value.code == B.A2_EORDER
+    before = eng.read_state()
+    eng.flush(t_end)
+    chk.plain.flush(t_end)
+    x, xt, t = eng.read_state()
+    assert np.array_equal(t, np.full(cfg.n, t_end)) and not np.array_equal(before[0], x)
+    xw, xtw = P.widen(x, storage), P.widen(xt, storage)
+    if storage == "f32":
+        assert P.rel_err(xw, chk.plain.X) <= 1e-5 and P.rel_err(xtw, chk.plain.Xt) <= 1e-5
+        gap = np.abs(xw.mean(0) - xtw.mean(0)).max() / np.abs(xw.mean(0)).max()
+        gap_before = np.abs(before[0].mean(0) - before[1].mean(0)).max() / np.abs(xw.mean(0)).max()
+        assert gap < 1e-5 < gap_before
+    else:
+        assert P.row_norm_err(xw, chk.plain.X) <= 2e-2 and P.row_norm_err(xtw, chk.plain.Xt) <= 2e-2
+    # the consensus distance of the flushed state is what consensus_distance(t) reported without writing
+    c_now = eng.consensus_distance()
+    assert abs(c_now - chk.plain.consensus()) <= (1e-4 if storage == "f32" else 5e-2) * c_now
+    eng.flush(t_end)  # already there: nothing to do
+    assert all(np.array_equal(u, v) for u, v in zip((x, xt, t), eng.read_state()))
+    eng.close()
