@@ -85,69 +85,54 @@ def closed_loop_batches(sched, ev):
     return out
 
 
-def run_closed_loop(n, d, graph, comms_per_grad, accelerated, T, gamma, seed, samples=10, noise_std=0.0,
-                    device="cuda:0", backend="gpu"):
-    """Decentralised SGD on the quadratic with the engine (backend 'gpu') or with the CPU checker
-    ('oracle', for tests). As in Algorithm 1 the gradient is evaluated at the worker's stored
-    parameters when its gradient event fires, then the mixing and the step are applied. Gradients are
-    the user's model, not the library's: they are computed here (torch on the GPU, NumPy for the
-    checker) and handed over as rows of the gradient buffer, batch by batch."""
+def closed_loop_problem(n, d, graph, comms_per_grad, T, seed):
+    """The quadratic, the graph and the event stream of a closed-loop run (shared with the tests)."""
     edges = W.make_edges(graph, n)
     rates = W.edge_rates_per_worker(n, edges, comms_per_grad)
-    prob = Quadratic(n, d, seed)
     n_events = int((n + rates.sum()) * T)
-    ev = W.poisson_events(n, edges, rates, n_events, seed=seed)
+    return Quadratic(n, d, seed), edges, rates, W.poisson_events(n, edges, rates, n_events, seed=seed)
+
+
+def run_closed_loop(n, d, graph, comms_per_grad, accelerated, T, gamma, seed, samples=10, noise_std=0.0,
+                    device="cuda:0"):
+    """Decentralised SGD on the quadratic with the engine. As in Algorithm 1 the gradient is evaluated
+    at the worker's stored parameters when its gradient event fires, then the mixing and the step are
+    applied. Gradients are the user's model, not the library's: they are computed here with torch and
+    handed over as rows of the gradient buffer, batch by batch."""
+    prob, edges, rates, ev = closed_loop_problem(n, d, graph, comms_per_grad, T, seed)
+    n_events = len(ev)
     x0 = np.zeros((n, d), dtype=np.float32)
     trace = []
     step = max(1, n_events // samples)
-    if backend == "gpu":
-        import torch
+    import torch
 
-        chi1, chi2 = B.graph_chi(n, edges, rates)
-        eta, alpha, alpha_t = B.prescribe(chi1, chi2, accelerated)
-        eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n, device=device)
-        eng.write_state(x0)
-        a = torch.from_numpy(prob.a.astype(np.float32)).to(device)
-        bt = torch.from_numpy(prob.b.astype(np.float32)).to(device)
-        xs = torch.from_numpy(prob.x_star).to(device)
-        gen = torch.Generator(device=device).manual_seed(seed)
-        for k in range(0, n_events, step):
-            c = ev.slice(k, k + step)
-            plan = eng.plan(c.times, c.wi, c.wj, c.slot, flags=0)
-            for bi, (_, workers, slots) in enumerate(closed_loop_batches(plan.sched, c)):
-                if len(workers):
-                    w = torch.from_numpy(workers).to(device)
-                    g = a[w] * (eng.x[w, :d] - bt[w])
-                    if noise_std > 0:
-                        g = g + noise_std * torch.randn(g.shape, generator=gen, device=device)
-                    eng.g[torch.from_numpy(slots).to(device), :d] = g
-                plan.run(bi, 1)
-            plan.close()
-            t = float(c.times[-1])
-            eng.flush(t)
-            eng.sync()
-            xbar = eng.x[:, :d].double().mean(0)
-            trace.append((t, float(((xbar - xs) ** 2).mean()), eng.consensus_distance() / d))
-        x_final = eng.read_state()[0].astype(np.float64)
-        eng.close()
-    else:
-        from oracle import spectral  # test infrastructure: only tests pass backend="oracle"
-        from oracle.sim import OracleSim
-
-        eta, alpha, alpha_t = spectral.prescribe(n, edges, rates, accelerated=accelerated)[:3]
-        G = np.zeros((n, d))
-        sim = OracleSim(x0.astype(np.float64), eta, alpha, alpha_t, gamma, grads=G)
-        for k in range(0, n_events, step):
-            c = ev.slice(k, k + step)
-            for e in range(len(c)):  # strictly in time order, one event at a time
-                if c.wj[e] < 0:
-                    w = int(c.wi[e])
-                    sim.G[int(c.slot[e])] = prob.a[w] * (sim.X[w] - prob.b[w])
-                sim.apply(c.times[e:e + 1], c.wi[e:e + 1], c.wj[e:e + 1], c.slot[e:e + 1])
-            t = float(c.times[-1])
-            sim.flush(t)
-            trace.append((t, float(((sim.X.mean(0) - prob.x_star) ** 2).mean()), sim.consensus() / d))
-        x_final = sim.X.copy()
+    chi1, chi2 = B.graph_chi(n, edges, rates)
+    eta, alpha, alpha_t = B.prescribe(chi1, chi2, accelerated)
+    eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n, device=device)
+    eng.write_state(x0)
+    a = torch.from_numpy(prob.a.astype(np.float32)).to(device)
+    bt = torch.from_numpy(prob.b.astype(np.float32)).to(device)
+    xs = torch.from_numpy(prob.x_star).to(device)
+    gen = torch.Generator(device=device).manual_seed(seed)
+    for k in range(0, n_events, step):
+        c = ev.slice(k, k + step)
+        plan = eng.plan(c.times, c.wi, c.wj, c.slot, flags=0)
+        for bi, (_, workers, slots) in enumerate(closed_loop_batches(plan.sched, c)):
+            if len(workers):
+                w = torch.from_numpy(workers).to(device)
+                g = a[w] * (eng.x[w, :d] - bt[w])
+                if noise_std > 0:
+                    g = g + noise_std * torch.randn(g.shape, generator=gen, device=device)
+                eng.g[torch.from_numpy(slots).to(device), :d] = g
+            plan.run(bi, 1)
+        plan.close()
+        t = float(c.times[-1])
+        eng.flush(t)
+        eng.sync()
+        xbar = eng.x[:, :d].double().mean(0)
+        trace.append((t, float(((xbar - xs) ** 2).mean()), eng.consensus_distance() / d))
+    x_final = eng.read_state()[0].astype(np.float64)
+    eng.close()
     return {"comms_per_grad": comms_per_grad, "accelerated": bool(accelerated), "events": n_events, "trace": trace,
             "x_final": x_final}
 
