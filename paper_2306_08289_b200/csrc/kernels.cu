@@ -219,24 +219,34 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
     const long long n_units = (long long)p.n_items * p.n_tiles;
 
-    // unit -> (item = unit % n_items, tile = unit / n_items). The bf16 kernel issues twice the instructions
-    // per byte and is helped by every instruction saved: it advances (item, tile) incrementally and leaves
-    // absent rows uninitialised. The fp32 kernel measured about 1 % FASTER with the 64-bit division per unit
-    // and the zero fill left in (6.37 against 6.30 TB/s on 64 rows of 25.6e6 columns): it is bound by DRAM
-    // alone and the extra work between units spaces its bursts of loads; so it keeps them.
+    // unit -> (tile = unit / n_items, item = (unit % n_items + tile) % n_items). The skew by the tile index
+    // makes every CTA walk through ALL items of the batch: without it a CTA whose stride shares a factor with
+    // n_items would see only some of them, and items differ in cost (5 to 10 rows), which left the batches of
+    // the 64-worker ring with a 2.7 % load imbalance across CTAs (0.4 % with the skew).
+    // The bf16 kernel issues twice the instructions per byte and is helped by every instruction saved: it
+    // advances (item, tile) incrementally and leaves absent rows uninitialised. The fp32 kernel measured about
+    // 1 % FASTER with the 64-bit division per unit and the zero fill left in (6.37 against 6.30 TB/s on 64 rows
+    // of 25.6e6 columns): it is bound by DRAM alone and the extra work between units spaces its bursts of loads;
+    // so it keeps them.
     constexpr bool kRecompute = sizeof(T) == 4;
-    int item_idx = (int)(blockIdx.x % (unsigned)p.n_items);
-    long long tile = blockIdx.x / (unsigned)p.n_items;
-    const int step_item = (int)(gridDim.x % (unsigned)p.n_items);
-    const long long step_tile = gridDim.x / (unsigned)p.n_items;
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x, item_idx += step_item, tile += step_tile) {
+    const int n_it = p.n_items;
+    int rem = (int)(blockIdx.x % (unsigned)n_it);
+    long long tile = blockIdx.x / (unsigned)n_it;
+    int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+    const int step_rem = (int)(gridDim.x % (unsigned)n_it);
+    const long long step_tile = gridDim.x / (unsigned)n_it;
+    const int step_skew = (int)((unsigned long long)step_tile % (unsigned)n_it);
+    for (long long unit = blockIdx.x; unit < n_units;
+         unit += gridDim.x, rem += step_rem, tile += step_tile, skew += step_skew) {
         if (kRecompute) {
-            item_idx = (int)(unit % p.n_items);
-            tile = unit / p.n_items;
-        } else if (item_idx >= p.n_items) {
-            item_idx -= p.n_items;
-            tile += 1;
+            rem = (int)(unit % n_it);
+            tile = unit / n_it;
+            skew = (int)((unsigned)tile % (unsigned)n_it);
+        } else {
+            if (rem >= n_it) { rem -= n_it; tile += 1; skew += 1; }
+            if (skew >= n_it) skew -= n_it;
         }
+        const int item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
         const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
         const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
