@@ -46,7 +46,7 @@ NOMINAL_HBM_GBS = 8000.0
 # summary (profiles/k_apply_events_cfg4_d2m.md: three launches of a d = 2e6 case), as a ratio to
 # the bytes the launch's items must move: reads 1.000, writes 0.90 (the rest was still in L2 when
 # the small launches ended). None once the kernel has changed since the counters were taken.
-NCU_TRAFFIC_RATIO = 0.957
+NCU_TRAFFIC_RATIO = 0.955
 
 
 def parse_args():
