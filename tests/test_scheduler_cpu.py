@@ -185,3 +185,63 @@ def test_fifo_stream_with_ties_replays_exactly():
             idx = np.sort(s.batch_events(b))  # stream order inside the batch (times tie)
             sim.apply(ev.times[idx], ev.wi[idx], ev.wj[idx], ev.slot[idx])
         assert np.array_equal(sim.X, ref.X) and np.array_equal(sim.Xt, ref.Xt) and np.array_equal(sim.t, ref.t)
+
+
+def test_random_streams_property():
+    """Property test over random small streams (ties, bursts on one worker, several gradient rows per
+    worker, tight caps): the batches cover every event once, keep workers disjoint inside a batch, and
+    replay to the bit-exact state of the time-ordered run."""
+    from hypothesis import given, settings, strategies as st
+
+    @st.composite
+    def streams(draw):
+        n = draw(st.integers(2, 9))
+        n_slots = draw(st.integers(1, 2 * n))
+        m = draw(st.integers(0, 60))
+        gaps = draw(st.lists(st.sampled_from([0.0, 0.0, 0.25, 1.0, 3.5]), min_size=m, max_size=m))
+        times = np.cumsum(np.array(gaps, dtype=np.float64)) if m else np.zeros(0)
+        wi, wj, sl = [], [], []
+        for _ in range(m):
+            i = draw(st.integers(0, n - 1))
+            if draw(st.booleans()):
+                j = draw(st.integers(0, n - 2))
+                j = j + 1 if j >= i else j
+                wi.append(i); wj.append(j); sl.append(-1)
+            else:
+                wi.append(i); wj.append(-1); sl.append(draw(st.integers(0, n_slots - 1)))
+        flags = draw(st.sampled_from([0, B.A2_SCHED_FUSE]))
+        cap = draw(st.sampled_from([0, 2, 3, 5]))
+        return n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32), flags, cap
+
+    @settings(max_examples=150, deadline=None)
+    @given(streams())
+    def check(case):
+        n, n_slots, times, wi, wj, sl, flags, cap = case
+        rng = np.random.default_rng(len(times) * 31 + n)
+        x0, G = rng.standard_normal((n, 3)), rng.standard_normal((n_slots, 3))
+        ref = OracleSim(x0, 0.4, 0.5, 1.7, 0.1, grads=G)
+        ref.apply(times, wi, wj, sl)
+        s = B.Schedule(n, n_slots, times, wi, wj, sl, flags=flags, max_ops_per_item=cap)
+        sim = OracleSim(x0, 0.4, 0.5, 1.7, 0.1, grads=G)
+        seen = []
+        for b in range(s.num_batches):
+            first, cnt = s.batch_items(b)
+            used = set()
+            for k in range(first, first + cnt):
+                it = s.item(k)
+                ws = {it.a} | ({it.b} if it.b >= 0 else set())
+                assert not (ws & used) and (cap == 0 or it.n_ops <= max(cap, 1))
+                used |= ws
+                evs, _ = s.ops(it.first_op, it.n_ops)
+                e = evs[np.argsort(times[evs], kind="stable")]
+                # inside an item a worker's own events are already in stream order
+                for w in ws:
+                    mine = [x for x in evs if wi[x] == w or wj[x] == w]
+                    assert mine == sorted(mine)
+                sim.apply(times[e], wi[e], wj[e], sl[e])
+                seen.extend(evs.tolist())
+        assert sorted(seen) == list(range(len(times)))
+        assert np.array_equal(sim.X, ref.X) and np.array_equal(sim.Xt, ref.Xt) and np.array_equal(sim.t, ref.t)
+        assert np.array_equal(s.t_final(n), ref.t)
+
+    check()
