@@ -464,15 +464,29 @@ bool rows_32B_aligned(const void* a, const void* b, const void* c, int64_t pitch
     return (bits % 32 == 0) && (pitch_bytes % 32 == 0);
 }
 
+// Launches the partial-sum kernel with as many CTAs as are resident at once for this variant (at most
+// `capacity`, the size of the scratch array) and returns that number: a grid of one full wave, so that no
+// CTA waits for a slot while others already finish.
+template <typename T, int BYTES, bool FLUSH>
+int consensus_partial_variant(const T* X, const T* Xt, int64_t pitch, int32_t n, int64_t d, double eta, const double* dt,
+                              double* partials, int capacity, int sm_count, cudaStream_t stream) {
+    const size_t smem = FLUSH ? (size_t)n * sizeof(float) : 0;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_consensus_partial<T, BYTES, FLUSH>, kThreads, smem) != cudaSuccess || occ < 1)
+        occ = 1;
+    int grid = sm_count * occ;
+    if (grid > capacity) grid = capacity;
+    k_consensus_partial<T, BYTES, FLUSH><<<grid, kThreads, smem, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+    return grid;
+}
+
 template <typename T, int BYTES>
-void launch_consensus_partial_t(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, double eta,
-                                const double* dt, double* partials, int n_partials, cudaStream_t stream) {
+int launch_consensus_partial_t(const void* x, const void* xt, int64_t pitch, int32_t n, int64_t d, double eta,
+                               const double* dt, double* partials, int capacity, int sm_count, cudaStream_t stream) {
     const T* X = static_cast<const T*>(x);
     const T* Xt = static_cast<const T*>(xt);
-    if (dt)
-        k_consensus_partial<T, BYTES, true><<<n_partials, kThreads, (size_t)n * sizeof(float), stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
-    else
-        k_consensus_partial<T, BYTES, false><<<n_partials, kThreads, 0, stream>>>(X, Xt, pitch, n, d, eta, dt, partials);
+    if (dt) return consensus_partial_variant<T, BYTES, true>(X, Xt, pitch, n, d, eta, dt, partials, capacity, sm_count, stream);
+    return consensus_partial_variant<T, BYTES, false>(X, Xt, pitch, n, d, eta, dt, partials, capacity, sm_count, stream);
 }
 
 }  // namespace
@@ -487,7 +501,7 @@ int query_device(DeviceInfo* info) {
     if ((e = event_occupancy<float, 32>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<__nv_bfloat16, 16>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
     info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
-    info->consensus_ctas_per_sm = 4;
+    info->consensus_ctas_per_sm = 8;  // capacity of the partial-sum scratch, CTAs per SM
     if (const char* v = std::getenv("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
         const int k = std::atoi(v);
         if (k > 0)
@@ -511,15 +525,17 @@ int launch_consensus(const void* x, const void* xt, int64_t pitch, int32_t n, in
                      const double* dt, double* partials, int n_partials, double* out, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const bool wide = rows_32B_aligned(x, xt, nullptr, pitch, dtype);
+    const int sms = n_partials / 8 > 0 ? n_partials / 8 : 1;  // the scratch holds 8 partial sums per SM
+    int used;
     if (dtype == A2_BF16) {
-        launch_consensus_partial_t<__nv_bfloat16, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
+        used = launch_consensus_partial_t<__nv_bfloat16, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, sms, stream);
     } else {
-        if (wide) launch_consensus_partial_t<float, 32>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
-        else launch_consensus_partial_t<float, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, stream);
+        if (wide) used = launch_consensus_partial_t<float, 32>(x, xt, pitch, n, d, eta, dt, partials, n_partials, sms, stream);
+        else used = launch_consensus_partial_t<float, 16>(x, xt, pitch, n, d, eta, dt, partials, n_partials, sms, stream);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
-    k_consensus_final<<<1, kThreads, 0, stream>>>(partials, n_partials, out);
+    k_consensus_final<<<1, kThreads, 0, stream>>>(partials, used, out);
     return (int)cudaGetLastError();
 }
 
