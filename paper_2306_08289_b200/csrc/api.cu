@@ -71,6 +71,8 @@ struct a2cid2 {
     Arena arena[2];
     int arena_next = 0;
     std::vector<a2cid2_plan*> plans;  // live plans made from this handle
+    uint64_t bind_epoch = 0;          // bumped whenever buffers, stream or variant change (invalidates plan graphs)
+    cudaStream_t capture_stream = nullptr;  // private stream on which plan graphs are recorded
     std::string err;
 };
 
@@ -94,6 +96,8 @@ struct a2cid2_plan {
     a2cid2_sched* sched = nullptr;
     void* d_desc = nullptr;  // the descriptor blob on the device
     Packed pk;
+    cudaGraphExec_t graph = nullptr;  // all launches of the plan as one CUDA graph (built on first whole run)
+    uint64_t graph_epoch = 0;
     int64_t next_batch = 0;
     bool uses_gradients = false;
     std::vector<double> t_expect;  // workers' times the next batch expects
@@ -216,7 +220,8 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
 }
 
 // Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
-int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev, int64_t b0, int64_t b1) {
+int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev, int64_t b0, int64_t b1,
+                  cudaStream_t stream) {
     if (b1 <= b0) return A2_OK;
     char* base = static_cast<char*>(dev);
     const DevItem* d_items = reinterpret_cast<const DevItem*>(base);
@@ -231,7 +236,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.chunks = reinterpret_cast<const a2::ResChunk*>(base + pk.chunks_off);
         L.g_rows = reinterpret_cast<const int32_t*>(base + pk.g_rows_off);
         L.n_events = (int32_t)s.items.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
-        const int rc = a2::launch_resident(L, h->dev, h->stream);
+        const int rc = a2::launch_resident(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;
     }
@@ -246,9 +251,42 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.eta = h->eta;
         L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
         L.variant = h->variant; L.dtype = h->dtype;
-        const int rc = a2::launch_events(L, h->dev, h->stream);
+        const int rc = a2::launch_events(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
+    return A2_OK;
+}
+
+constexpr int64_t kGraphMinLaunches = 4;
+
+// Record all launches of a (batched) plan into a CUDA graph if that has not been done for the current
+// binding, then launch the graph on the handle's stream.
+int ensure_plan_graph(a2cid2* h, a2cid2_plan* p) {
+    if (p->graph && p->graph_epoch != h->bind_epoch) {
+        cudaGraphExecDestroy(p->graph);
+        p->graph = nullptr;
+    }
+    if (!p->graph) {
+        if (!h->capture_stream) A2_CUDA(h, cudaStreamCreateWithFlags(&h->capture_stream, cudaStreamNonBlocking));
+        const int64_t nb = (int64_t)p->sched->batch_first.size() - 1;
+        A2_CUDA(h, cudaStreamBeginCapture(h->capture_stream, cudaStreamCaptureModeThreadLocal));
+        const int rc = queue_batches(h, *p->sched, p->pk, p->d_desc, 0, nb, h->capture_stream);
+        cudaGraph_t g = nullptr;
+        const cudaError_t e = cudaStreamEndCapture(h->capture_stream, &g);
+        if (rc != A2_OK) { if (g) cudaGraphDestroy(g); return rc; }
+        if (e != cudaSuccess) return fail_cuda(h, e, "cudaStreamEndCapture");
+        const cudaError_t ei = cudaGraphInstantiate(&p->graph, g, 0);
+        cudaGraphDestroy(g);
+        if (ei != cudaSuccess) { p->graph = nullptr; return fail_cuda(h, ei, "cudaGraphInstantiate"); }
+        p->graph_epoch = h->bind_epoch;
+    }
+    return A2_OK;
+}
+
+int run_plan_graph(a2cid2* h, a2cid2_plan* p) {
+    const int rc = ensure_plan_graph(h, p);
+    if (rc != A2_OK) return rc;
+    A2_CUDA(h, cudaGraphLaunch(p->graph, h->stream));
     return A2_OK;
 }
 
@@ -318,6 +356,7 @@ int a2cid2_set_variant(a2cid2_t* h, int32_t variant) {
     if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
     if (variant != A2_MSG_AFTER_MIX && variant != A2_MSG_BEFORE_MIX) return fail(h, A2_EINVAL, "unknown variant");
     h->variant = variant;
+    h->bind_epoch += 1;
     return A2_OK;
 }
 
@@ -337,6 +376,7 @@ int a2cid2_bind(a2cid2_t* h, void* x, void* x_tilde, void* grads, int32_t n_grad
     h->n_slots = n_grad_slots; h->pitch = row_pitch_elems;
     h->stream = static_cast<cudaStream_t>(cuda_stream);
     h->bound = true;
+    h->bind_epoch += 1;
     return A2_OK;
 }
 
@@ -435,7 +475,7 @@ static int submit_schedule(a2cid2* h, a2cid2_sched* s, a2cid2_stats* stats, doub
         if (e != cudaSuccess) { a2cid2_sched_destroy(s); return fail_cuda(h, e, "descriptor upload"); }
         A.in_flight = true;
         const double t1 = now_ms();
-        rc = queue_batches(h, *s, pk, A.dev, 0, nb);
+        rc = queue_batches(h, *s, pk, A.dev, 0, nb, h->stream);
         if (rc != A2_OK) { a2cid2_sched_destroy(s); return rc; }
         if (stats) {
             fill_stats(h, *s, pk, 0, nb, stats);
@@ -524,6 +564,7 @@ void a2cid2_destroy(a2cid2_t* h) {
             if (A.dev) cudaFree(A.dev);
             if (A.copied) cudaEventDestroy(A.copied);
         }
+        if (h->capture_stream) cudaStreamDestroy(h->capture_stream);
         if (h->d_partials) cudaFree(h->d_partials);
         if (h->d_dt) cudaFree(h->d_dt);
         if (h->h_pinned) cudaFreeHost(h->h_pinned);
@@ -590,6 +631,15 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
             return fail_cuda(h, e, "plan descriptor upload");
         }
     }
+    if (!p->pk.resident && (int64_t)p->pk.launches.size() >= kGraphMinLaunches) {
+        rc = ensure_plan_graph(h, p);  // recorded now, so that running the plan is a single submission
+        if (rc != A2_OK) {
+            if (p->d_desc) cudaFree(p->d_desc);
+            a2cid2_sched_destroy(s);
+            delete p;
+            return rc;
+        }
+    }
     h->plans.push_back(p);
     *out = p;
     return A2_OK;
@@ -609,7 +659,15 @@ int a2cid2_plan_run(a2cid2_t* h, a2cid2_plan_t* p, int64_t first_batch, int64_t 
     if (p->uses_gradients && !h->g) return fail(h, A2_ESTATE, "plan has gradient events but no gradient buffer is bound");
     const int64_t b1 = first_batch + n_batches;
     if (n_batches > 0) {
-        rc = queue_batches(h, *p->sched, p->pk, p->d_desc, first_batch, b1);
+        // A plan of several launches run whole goes out as one CUDA graph: one submission instead of one per
+        // batch. The graph was recorded on a private stream when the plan was made and is recorded again only if
+        // the bound buffers, the stream or the variant have changed since.
+        const bool whole = first_batch == 0 && b1 == nb;
+        if (whole && !p->pk.resident && (int64_t)p->pk.launches.size() >= kGraphMinLaunches) {
+            rc = run_plan_graph(h, p);
+        } else {
+            rc = queue_batches(h, *p->sched, p->pk, p->d_desc, first_batch, b1, h->stream);
+        }
         if (rc != A2_OK) return rc;
         advance_times(*p->sched, first_batch, b1, h->t);
     }
@@ -631,6 +689,7 @@ void a2cid2_plan_destroy(a2cid2_plan_t* p) {
         for (size_t k = 0; k < v.size(); ++k)
             if (v[k] == p) { v.erase(v.begin() + (long)k); break; }
     }
+    if (p->graph) cudaGraphExecDestroy(p->graph);
     if (p->d_desc) cudaFree(p->d_desc);
     a2cid2_sched_destroy(p->sched);
     delete p;

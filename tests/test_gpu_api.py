@@ -257,3 +257,23 @@ def test_plan_may_outlive_its_engine():
     q.close()
     eng.close()  # p is still alive: it may only be destroyed now
     p.close()
+
+
+def test_plan_graph_follows_a_change_of_variant():
+    """A plan run whole goes out as one CUDA graph recorded when the plan was made; changing what the
+    kernels were recorded with (here the variant) must re-record it, not replay the stale one."""
+    cfg = _small(n_events=400)
+    ev = W.config_events(cfg)
+    want_eng, _ = P.make_small(cfg, variant=B.A2_MSG_BEFORE_MIX)
+    want_eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    want = want_eng.read_state()
+    want_eng.close()
+    eng, _ = P.make_small(cfg)
+    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)  # recorded with the default variant
+    assert p.sched.num_batches >= 4
+    eng.set_variant(B.A2_MSG_BEFORE_MIX)
+    p.run()
+    got = eng.read_state()
+    p.close()
+    eng.close()
+    assert all(np.array_equal(u, v) for u, v in zip(want, got))
