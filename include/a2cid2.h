@@ -215,7 +215,9 @@ void a2cid2_destroy(a2cid2_t* h);
 
 /* Validate and schedule an event stream as a2cid2_apply_events does and upload its
  * descriptors, but launch nothing. t_start[n] gives the workers' times the stream starts
- * from (NULL = the handle's current times); a2cid2_plan_run checks them against the handle. */
+ * from (NULL = the handle's current times); a2cid2_plan_run checks them against the handle. A plan of
+ * several launches also records them as one CUDA graph (on a private stream), so that running the
+ * whole plan is a single submission. */
 int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, const double* times,
                        const int32_t* wi, const int32_t* wj, const int32_t* grad_slot, uint32_t flags,
                        a2cid2_plan_t** out);
