@@ -61,18 +61,16 @@ enum {
     A2_SCHED_FUSE = 1u, /* fold the gradient events that directly precede a communication of the
                            same worker into that communication's item, so their rows are read
                            and written once (the arithmetic per element is unchanged)          */
-    A2_SCHED_RESIDENT = 2u /* launch mode: the schedule is the unfused batch schedule (A2_SCHED_FUSE
-                              is ignored), but ONE launch walks all of it while a 256-column tile of
-                              all n workers' x and x~ stays in shared memory, so the state crosses HBM
-                              once per call instead of once per batch. Columns never interact: a
-                              thread owns a column and never waits for another thread. Events of one
-                              batch touch disjoint workers, so a thread keeps up to four of them in
-                              flight. Only valid when the gradients of the whole stream are known up
-                              front (they are rows of the bound buffer), for populations that fit
-                              shared memory (2 n + 16 <= 216 rows of 256 floats; A2_EINVAL otherwise);
-                              a plan made with it must be run whole (all batches in one
-                              a2cid2_plan_run, A2_ESTATE otherwise). With bf16 storage the tile is
-                              kept in fp32 and rounded once, at the end of the call.           */
+    A2_SCHED_RESIDENT = 2u /* no batches: one launch walks the whole stream in time order while a
+                              column tile of all n workers' x and x~ stays in shared memory, so the
+                              state crosses HBM once per call instead of once per batch. Columns
+                              never interact, so no thread ever waits for another. Only valid when
+                              the gradients of the whole stream are known up front (they are rows
+                              of the bound buffer), and only for populations that fit shared
+                              memory (2 n + 16 <= 216 rows of 256 floats; A2_EINVAL otherwise).
+                              With bf16 storage the tile is kept in fp32 and rounded once, at the
+                              end of the call. The schedule then has a single batch holding every
+                              event in stream order. Overrides A2_SCHED_FUSE.                  */
 };
 
 /* Kinds of elementary operation inside an item. */

@@ -48,7 +48,7 @@ namespace a2 {
 struct ResEv {  // one event, as the resident kernel reads it (16 bytes)
     int16_t a, b;  // workers (b = -1: gradient event)
     int16_t g;     // index of the gradient row in the chunk's cache, or -1
-    int16_t kind;  // A2_OP_GRAD_A, A2_OP_COMM, or -1 for the padding of a short group
+    int16_t kind;  // A2_OP_GRAD_A or A2_OP_COMM
     float ca, cb;  // mixing coefficients of a and b for this event
 };
 struct ResChunk {
@@ -59,9 +59,8 @@ constexpr int kResidentCols = 256;     // columns per tile = threads per CTA
 constexpr int kResidentMaxRows = 216;  // 2 n + cache rows, 1 KB of shared memory each
 constexpr int kResidentMinCache = 16;
 
-void build_resident_chunks(const a2cid2_sched& s, int capacity, int group, std::vector<int32_t>& order,
-                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
-                           std::vector<int32_t>& cache_idx);
+void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResChunk>& chunks,
+                           std::vector<int32_t>& g_rows, std::vector<int32_t>& cache_idx);
 
 // Builds a schedule; returns A2_OK or an error code with the text in `err`.
 int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
@@ -134,8 +133,7 @@ struct ResidentLaunch {
     ResEv* events;           // device, n_events (written by the prepare kernel)
     const ResChunk* chunks;  // device
     const int32_t* g_rows;   // device
-    int32_t n_events, n_chunks, cache_rows;  // n_events counts the padded list
-    int32_t group;                           // events in flight together: 1, 2 or 4
+    int32_t n_events, n_chunks, cache_rows;
 };
 int resident_cache_rows(int32_t n, int32_t n_grad_slots);  // 0: the population does not fit
 int launch_resident(const ResidentLaunch& L, const DeviceInfo& dev, void* stream);

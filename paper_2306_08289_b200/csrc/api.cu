@@ -86,8 +86,6 @@ struct Packed {
     // resident mode
     bool resident = false;
     int32_t cache_rows = 0;
-    int32_t group = 1;           // events the resident kernel keeps in flight together
-    std::vector<int32_t> order;  // item index of every slot of the padded event list (-1: padding)
     size_t chunks_off = 0, g_rows_off = 0, events_off = 0;
     std::vector<a2::ResChunk> chunks;
     std::vector<int32_t> g_rows, cache_idx;
@@ -179,17 +177,11 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
         pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
         if (pk.cache_rows <= 0)
             return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT: the population does not fit shared memory (need 2 n + 16 <= 216)");
-        const int64_t nb = (int64_t)s.batch_first.size() - 1;
-        const double width = nb > 0 ? (double)s.items.size() / (double)nb : 1.0;  // events per batch
-        pk.group = width >= 6.0 ? 4 : (width >= 2.5 ? 2 : 1);
-        a2::build_resident_chunks(s, pk.cache_rows, pk.group, pk.order, pk.chunks, pk.g_rows, pk.cache_idx);
-        // the item and operation records are laid out in the padded order, one operation per slot
-        pk.ops_off = align16(pk.order.size() * sizeof(DevItem));
-        end = pk.ops_off + pk.order.size() * sizeof(DevOp);
+        a2::build_resident_chunks(s, pk.cache_rows, pk.chunks, pk.g_rows, pk.cache_idx);
         pk.chunks_off = align16(end);
         pk.g_rows_off = align16(pk.chunks_off + pk.chunks.size() * sizeof(a2::ResChunk));
         pk.events_off = align16(pk.g_rows_off + pk.g_rows.size() * sizeof(int32_t));
-        end = pk.events_off + pk.order.size() * sizeof(a2::ResEv);  // this part is written on the device
+        end = pk.events_off + s.items.size() * sizeof(a2::ResEv);  // this part is written on the device
     }
     pk.bytes = s.items.empty() ? 0 : end;
     return A2_OK;
@@ -212,28 +204,19 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
                 di[k] = DevItem{it.a, it.b, it.slot_a, it.slot_b, (int32_t)(it.first_op - L.op0), it.n_ops};
             }
     } else {
-        for (size_t e = 0; e < pk.order.size(); ++e) {  // one operation per slot; slot_b carries the cache index
-            const int32_t k = pk.order[e];
-            if (k < 0) {
-                di[e] = DevItem{0, -1, -1, -1, (int32_t)e, 1};
-                dop[e] = DevOp{-1, 0, 0.0, 0.0, 0.0};  // padding: the kernel skips it
-                continue;
-            }
-            const a2::SchedItem& it = s.items[(size_t)k];
-            const a2::SchedOp& op = s.ops[(size_t)it.first_op];
-            di[e] = DevItem{it.a, it.b, it.slot_a, pk.cache_idx[e], (int32_t)e, 1};
-            dop[e] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
+        for (size_t k = 0; k < s.items.size(); ++k) {  // one operation per item; slot_b carries the cache index
+            const a2::SchedItem& it = s.items[k];
+            di[k] = DevItem{it.a, it.b, it.slot_a, pk.cache_idx[k], (int32_t)k, 1};
         }
         if (!pk.chunks.empty())
             std::memcpy(static_cast<char*>(dst) + pk.chunks_off, pk.chunks.data(), pk.chunks.size() * sizeof(a2::ResChunk));
         if (!pk.g_rows.empty())
             std::memcpy(static_cast<char*>(dst) + pk.g_rows_off, pk.g_rows.data(), pk.g_rows.size() * sizeof(int32_t));
     }
-    if (!pk.resident)
-        for (size_t o = 0; o < s.ops.size(); ++o) {
-            const a2::SchedOp& op = s.ops[o];
-            dop[o] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
-        }
+    for (size_t o = 0; o < s.ops.size(); ++o) {
+        const a2::SchedOp& op = s.ops[o];
+        dop[o] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
+    }
 }
 
 // Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
@@ -244,8 +227,6 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     const DevItem* d_items = reinterpret_cast<const DevItem*>(base);
     const DevOp* d_ops = reinterpret_cast<const DevOp*>(base + pk.ops_off);
     if (pk.resident) {
-        if (b0 != 0 || b1 != (int64_t)s.batch_first.size() - 1)
-            return fail(h, A2_ESTATE, "a plan made with A2_SCHED_RESIDENT runs all its batches in one call");
         a2::ResidentLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.n = h->n; L.dtype = h->dtype; L.variant = h->variant; L.eta = h->eta;
@@ -254,8 +235,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.events = reinterpret_cast<a2::ResEv*>(base + pk.events_off);
         L.chunks = reinterpret_cast<const a2::ResChunk*>(base + pk.chunks_off);
         L.g_rows = reinterpret_cast<const int32_t*>(base + pk.g_rows_off);
-        L.n_events = (int32_t)pk.order.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
-        L.group = pk.group;
+        L.n_events = (int32_t)s.items.size(); L.n_chunks = (int32_t)pk.chunks.size(); L.cache_rows = pk.cache_rows;
         const int rc = a2::launch_resident(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;

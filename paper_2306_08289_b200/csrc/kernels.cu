@@ -564,8 +564,8 @@ __global__ void __launch_bounds__(kThreads) k_resident_prepare(const DevItem* __
     r.a = (int16_t)it.a;
     r.b = (int16_t)it.b;
     r.g = (int16_t)it.slot_b;  // cache index of the gradient row (set by the host for gradient events)
-    r.kind = (int16_t)op.kind;  // -1: padding of a short group
-    r.ca = op.kind >= 0 ? (float)mix_coeff(eta, op.t - op.t_prev_a) : 0.f;
+    r.kind = (int16_t)op.kind;
+    r.ca = (float)mix_coeff(eta, op.t - op.t_prev_a);
     r.cb = op.kind == A2_OP_COMM ? (float)mix_coeff(eta, op.t - op.t_prev_b) : 0.f;
     out[e] = r;
 }
@@ -592,9 +592,7 @@ struct ResidentArgs {
     int msg_before_mix;
 };
 
-// GROUP events of one batch (disjoint workers) are fetched, computed and stored together, so that a thread
-// has GROUP independent chains of shared-memory loads and arithmetic in flight instead of one.
-template <typename T, int GROUP>
+template <typename T>
 __global__ void __launch_bounds__(kResidentCols) k_resident(const ResidentArgs p) {
     extern __shared__ float s_tile[];  // [n][256] x, [n][256] x~, [cache][256] gradient rows
     float* const sX = s_tile + threadIdx.x;
@@ -621,53 +619,28 @@ __global__ void __launch_bounds__(kResidentCols) k_resident(const ResidentArgs p
             for (int k = 0; k < ch.g_count; ++k)
                 sG[k * kResidentCols] = active ? widen1<T>(__ldg(G + (long long)p.g_rows[ch.g_begin + k] * p.pitch + col)) : 0.f;
             for (int e0 = ch.ev_begin; e0 < ch.ev_end; e0 += 32) {
-                // a warp fetches 32 event records with one coalesced load and hands them round by shuffle
-                int4 mine = make_int4(0, -65536, 0, 0);  // kind = -1
+                // a warp fetches 32 descriptors with one coalesced load and hands them round by shuffle
+                int4 mine = make_int4(0, 0, 0, 0);
                 if (e0 + lane < ch.ev_end) mine = __ldg(reinterpret_cast<const int4*>(p.events) + e0 + lane);
-                const int cnt = min(32, ch.ev_end - e0);  // a multiple of GROUP
-                for (int l = 0; l < cnt; l += GROUP) {
-                    int a[GROUP], b[GROUP], kind[GROUP];
-                    float ca[GROUP], cb[GROUP], xa[GROUP], xta[GROUP], xb[GROUP], xtb[GROUP], gg[GROUP];
-#pragma unroll
-                    for (int q = 0; q < GROUP; ++q) {
-                        const int w0 = __shfl_sync(0xffffffffu, mine.x, l + q);
-                        const int w1 = __shfl_sync(0xffffffffu, mine.y, l + q);
-                        ca[q] = __int_as_float(__shfl_sync(0xffffffffu, mine.z, l + q));
-                        cb[q] = __int_as_float(__shfl_sync(0xffffffffu, mine.w, l + q));
-                        a[q] = (int)(short)(w0 & 0xFFFF);
-                        b[q] = (int)(short)(w0 >> 16);
-                        kind[q] = (int)(short)(w1 >> 16);
-                        const int gi = (int)(short)(w1 & 0xFFFF);
-                        xa[q] = 0.f; xta[q] = 0.f; xb[q] = 0.f; xtb[q] = 0.f; gg[q] = 0.f;
-                        if (kind[q] >= 0) {
-                            xa[q] = sX[a[q] * kResidentCols];
-                            xta[q] = sXt[a[q] * kResidentCols];
-                            if (kind[q] == A2_OP_COMM) {
-                                xb[q] = sX[b[q] * kResidentCols];
-                                xtb[q] = sXt[b[q] * kResidentCols];
-                            } else {
-                                gg[q] = sG[gi * kResidentCols];
-                            }
-                        }
+                const int cnt = min(32, ch.ev_end - e0);
+                for (int l = 0; l < cnt; ++l) {
+                    const int w0 = __shfl_sync(0xffffffffu, mine.x, l);
+                    const int w1 = __shfl_sync(0xffffffffu, mine.y, l);
+                    const float ca = __int_as_float(__shfl_sync(0xffffffffu, mine.z, l));
+                    const float cb = __int_as_float(__shfl_sync(0xffffffffu, mine.w, l));
+                    const int a = (int)(short)(w0 & 0xFFFF), b = (int)(short)(w0 >> 16);
+                    const int gi = (int)(short)(w1 & 0xFFFF), kind = (int)(short)(w1 >> 16);
+                    float xa = sX[a * kResidentCols], xta = sXt[a * kResidentCols];
+                    if (kind == A2_OP_COMM) {
+                        float xb = sX[b * kResidentCols], xtb = sXt[b * kResidentCols];
+                        comm_elem<sizeof(T) == 4>(xa, xta, xb, xtb, ca, cb, p.alpha, p.alpha_tilde, before);
+                        sX[b * kResidentCols] = xb;
+                        sXt[b * kResidentCols] = xtb;
+                    } else {
+                        grad_elem<sizeof(T) == 4>(xa, xta, ca, ngamma, sG[gi * kResidentCols]);
                     }
-#pragma unroll
-                    for (int q = 0; q < GROUP; ++q) {
-                        if (kind[q] == A2_OP_COMM)
-                            comm_elem<sizeof(T) == 4>(xa[q], xta[q], xb[q], xtb[q], ca[q], cb[q], p.alpha, p.alpha_tilde, before);
-                        else if (kind[q] >= 0)
-                            grad_elem<sizeof(T) == 4>(xa[q], xta[q], ca[q], ngamma, gg[q]);
-                    }
-#pragma unroll
-                    for (int q = 0; q < GROUP; ++q) {
-                        if (kind[q] >= 0) {
-                            sX[a[q] * kResidentCols] = xa[q];
-                            sXt[a[q] * kResidentCols] = xta[q];
-                            if (kind[q] == A2_OP_COMM) {
-                                sX[b[q] * kResidentCols] = xb[q];
-                                sXt[b[q] * kResidentCols] = xtb[q];
-                            }
-                        }
-                    }
+                    sX[a * kResidentCols] = xa;
+                    sXt[a * kResidentCols] = xta;
                 }
             }
         }
@@ -681,13 +654,13 @@ __global__ void __launch_bounds__(kResidentCols) k_resident(const ResidentArgs p
     }
 }
 
-template <typename T, int GROUP>
+template <typename T>
 int launch_resident_t(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     const size_t smem = (size_t)(2 * L.n + L.cache_rows) * kResidentCols * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(k_resident<T, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_resident<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_resident<T, GROUP>, kResidentCols, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_resident<T>, kResidentCols, smem);
     if (e != cudaSuccess) return (int)e;
     if (occ < 1) return (int)cudaErrorInvalidConfiguration;
     ResidentArgs a;
@@ -698,15 +671,8 @@ int launch_resident_t(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     long long grid = (long long)dev.sm_count * occ;
     if (grid > a.n_tiles) grid = a.n_tiles;
-    k_resident<T, GROUP><<<(unsigned)grid, kResidentCols, smem, stream>>>(a);
+    k_resident<T><<<(unsigned)grid, kResidentCols, smem, stream>>>(a);
     return (int)cudaGetLastError();
-}
-
-template <typename T>
-int launch_resident_g(const ResidentLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
-    if (L.group == 4) return launch_resident_t<T, 4>(L, dev, stream);
-    if (L.group == 2) return launch_resident_t<T, 2>(L, dev, stream);
-    return launch_resident_t<T, 1>(L, dev, stream);
 }
 
 }  // namespace
@@ -727,8 +693,8 @@ int launch_resident(const ResidentLaunch& L, const DeviceInfo& dev, void* stream
     k_resident_prepare<<<blocks, kThreads, 0, stream>>>(L.items, L.ops, L.n_events, L.eta, L.events);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
-    if (L.dtype == A2_BF16) return launch_resident_g<__nv_bfloat16>(L, dev, stream);
-    return launch_resident_g<float>(L, dev, stream);
+    if (L.dtype == A2_BF16) return launch_resident_t<__nv_bfloat16>(L, dev, stream);
+    return launch_resident_t<float>(L, dev, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -162,6 +162,8 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             }
         }
         if (fuse) for (int32_t w = 0; w < n; ++w) flush(w);
+        if (resident)  // one batch, every event in stream order (items were created in that order)
+            for (SchedItem& it : items) it.batch = 0;
 
         // ---- order items by batch (stable) and lay the ops out in item order ----------------
         int32_t n_batches = 0;
@@ -188,30 +190,13 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     return A2_OK;
 }
 
-// Resident mode. The kernel walks the events of the (unfused) batch schedule batch by batch, `group`
-// events at a time; the events of a group come from one batch, so they touch disjoint workers and can be in
-// flight together. `order` lists item indices group by group, short groups padded with -1. The stream is
-// also cut into chunks whose distinct gradient rows fit `capacity` cache rows (a chunk is a whole number of
-// groups); inside a chunk a row keeps the cache index it got at first use.
-void build_resident_chunks(const a2cid2_sched& s, int capacity, int group, std::vector<int32_t>& order,
-                           std::vector<ResChunk>& chunks, std::vector<int32_t>& g_rows,
-                           std::vector<int32_t>& cache_idx) {
-    order.clear();
+// Resident mode: cut the stream into chunks whose distinct gradient rows fit `capacity` cache rows.
+// Inside a chunk a gradient row keeps the cache index it was given at first use.
+void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResChunk>& chunks,
+                           std::vector<int32_t>& g_rows, std::vector<int32_t>& cache_idx) {
     chunks.clear();
     g_rows.clear();
-    const int64_t nb = (int64_t)s.batch_first.size() - 1;
-    for (int64_t b = 0; b < nb; ++b) {
-        int64_t in_group = 0;
-        for (int64_t k = s.batch_first[(size_t)b]; k < s.batch_first[(size_t)b + 1]; ++k) {
-            order.push_back((int32_t)k);
-            in_group = (in_group + 1) % group;
-        }
-        while (in_group != 0) {  // pad the batch's last group
-            order.push_back(-1);
-            in_group = (in_group + 1) % group;
-        }
-    }
-    cache_idx.assign(order.size(), -1);
+    cache_idx.assign(s.items.size(), -1);
     std::vector<int32_t> where((size_t)std::max(1, s.n_grad_slots), -1);  // slot -> cache index in the open chunk
     ResChunk cur{0, 0, 0, 0};
     auto close = [&](int32_t ev_end) {
@@ -220,28 +205,18 @@ void build_resident_chunks(const a2cid2_sched& s, int capacity, int group, std::
         for (int32_t k = cur.g_begin; k < cur.g_begin + cur.g_count; ++k) where[(size_t)g_rows[(size_t)k]] = -1;
         cur = ResChunk{ev_end, ev_end, (int32_t)g_rows.size(), 0};
     };
-    for (size_t g0 = 0; g0 < order.size(); g0 += (size_t)group) {
-        int32_t fresh = 0;  // rows this group would add to the cache (a group's workers, hence rows, are distinct
-                            // unless two workers share a row; counting such a row twice only closes a chunk early)
-        for (int q = 0; q < group; ++q) {
-            const int32_t k = order[g0 + (size_t)q];
-            if (k >= 0 && s.items[(size_t)k].slot_a >= 0 && where[(size_t)s.items[(size_t)k].slot_a] < 0) fresh += 1;
+    for (size_t e = 0; e < s.items.size(); ++e) {
+        const int32_t slot = s.items[e].slot_a;
+        if (slot < 0) continue;
+        if (where[(size_t)slot] < 0) {
+            if (cur.g_count == capacity) close((int32_t)e);
+            where[(size_t)slot] = cur.g_count;
+            g_rows.push_back(slot);
+            cur.g_count += 1;
         }
-        if (cur.g_count + fresh > capacity) close((int32_t)g0);
-        for (int q = 0; q < group; ++q) {
-            const int32_t k = order[g0 + (size_t)q];
-            if (k < 0) continue;
-            const int32_t slot = s.items[(size_t)k].slot_a;
-            if (slot < 0) continue;
-            if (where[(size_t)slot] < 0) {
-                where[(size_t)slot] = cur.g_count;
-                g_rows.push_back(slot);
-                cur.g_count += 1;
-            }
-            cache_idx[g0 + (size_t)q] = where[(size_t)slot];
-        }
+        cache_idx[e] = where[(size_t)slot];
     }
-    close((int32_t)order.size());
+    close((int32_t)s.items.size());
 }
 
 void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {

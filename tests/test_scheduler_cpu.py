@@ -154,15 +154,18 @@ def test_bad_arguments():
         s.ops(0, 5)
 
 
-def test_resident_flag_keeps_the_unfused_batch_schedule():
+def test_resident_schedule_is_one_batch_in_stream_order():
     cfg = W.CONFIGS["cfg2"].scaled(d=3, n_events=1500)
     ev = W.config_events(cfg)
-    plain = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=0)
-    for flags in (B.A2_SCHED_RESIDENT, B.A2_SCHED_RESIDENT | B.A2_SCHED_FUSE):  # fusion is ignored
+    for flags in (B.A2_SCHED_RESIDENT, B.A2_SCHED_RESIDENT | B.A2_SCHED_FUSE):  # the resident flag wins
         s = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
-        assert (s.num_batches, s.num_items, s.num_ops) == (plain.num_batches, len(ev), len(ev))
-        for b in range(0, s.num_batches, 13):
-            assert np.array_equal(s.batch_events(b), plain.batch_events(b))
+        assert s.num_batches == 1 and s.num_items == len(ev) == s.num_ops
+        assert np.array_equal(s.batch_events(0), np.arange(len(ev)))
+        it = s.item(7)
+        assert (it.a, it.n_ops, it.batch) == (ev.wi[7], 1, 0)
+    sim = OracleSim(np.zeros((cfg.n, 1)), 0.1, 0.5, 0.5, 0.0, grads=np.zeros((cfg.n_grad_slots, 1)))
+    sim.apply_stream(ev)
+    assert np.array_equal(s.t_final(cfg.n), sim.t)
     with pytest.raises(B.A2Error):
         B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=4)
 
