@@ -25,6 +25,12 @@
  * taken at the event time, after both workers have been mixed forward to that time, as
  * Eq. (dynamic) states (variant 0). Algorithm 1 as printed forms the message before the
  * mixing line; that ordering is available as variant 1.
+ *
+ * Variant 2 is the asynchronous baseline the paper compares with, Eq. (baselinedynamic) of
+ * Sec. 3.2 (restated at the head of the proofs' appendix as what Eq. (dynamic) becomes when
+ * the method is not applied): there is no momentum buffer and no drift; a gradient event is
+ * x^i -= gamma g, a communication x^i -= alpha (x^i - x^j), x^j += alpha (x^i - x^j). X~ is
+ * never read or written; eta and alpha~ are ignored.
  */
 #include <math.h>
 #include <stddef.h>
@@ -45,20 +51,33 @@ static void a2o_mix(double* x, double* xt, int64_t d, double eta, double dt) {
     }
 }
 
+/* Eq. (baselinedynamic): the two jumps on x alone. */
+static void a2o_plain_grad(double* x, const double* g, int64_t d, double gamma) {
+    for (int64_t k = 0; k < d; ++k) x[k] = x[k] - gamma * g[k];
+}
+
+static void a2o_plain_comm(double* x, double* y, int64_t d, double alpha) {
+    for (int64_t k = 0; k < d; ++k) {
+        const double m = x[k] - y[k];
+        x[k] = x[k] - alpha * m;
+        y[k] = y[k] + alpha * m;
+    }
+}
+
 /*
  * Apply n_events events in the given order to X, Xt (row-major, row stride ld doubles,
  * d columns used) and the per-worker last-event times tl[n].
  *   wj[e] >= 0 : communication between wi[e] and wj[e]   (slot[e] must be -1)
  *   wj[e] == -1: gradient event on wi[e] with gradient row G[slot[e]] (row stride ldg)
  * variant 0: message after mixing (Eq. (dynamic)); variant 1: message before mixing
- * (Algorithm 1 as printed).
+ * (Algorithm 1 as printed); variant 2: Eq. (baselinedynamic), x only (Xt is left as it is).
  * Returns 0, or a negative code at the first invalid event (state is then partly updated).
  */
 int a2o_run(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double alpha_t, double gamma,
             double* X, double* Xt, double* tl, const double* G, int32_t n_slots, int64_t ldg,
             int64_t n_events, const double* times, const int32_t* wi, const int32_t* wj,
             const int32_t* slot, int32_t variant) {
-    if (n < 2 || d < 0 || ld < d || n_events < 0) return A2O_EINVAL;
+    if (n < 2 || d < 0 || ld < d || n_events < 0 || variant < 0 || variant > 2) return A2O_EINVAL;
     for (int64_t e = 0; e < n_events; ++e) {
         const double t = times[e];
         const int32_t i = wi[e], j = wj[e], s = slot[e];
@@ -71,6 +90,11 @@ int a2o_run(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double a
             if (j != -1 || s < 0 || s >= n_slots) return A2O_ERANGE;
             if (t < tl[i]) return A2O_EORDER;
             const double* g = G + (size_t)s * ldg;
+            if (variant == 2) {
+                a2o_plain_grad(xi, g, d, gamma);
+                tl[i] = t;
+                continue;
+            }
             a2o_mix(xi, xti, d, eta, t - tl[i]);
             for (int64_t k = 0; k < d; ++k) {
                 xi[k] = xi[k] - gamma * g[k];
@@ -83,6 +107,12 @@ int a2o_run(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double a
             if (t < tl[i] || t < tl[j]) return A2O_EORDER;
             double* xj = X + (size_t)j * ld;
             double* xtj = Xt + (size_t)j * ld;
+            if (variant == 2) {
+                a2o_plain_comm(xi, xj, d, alpha);
+                tl[i] = t;
+                tl[j] = t;
+                continue;
+            }
             if (variant == 0) {
                 a2o_mix(xi, xti, d, eta, t - tl[i]);
                 a2o_mix(xj, xtj, d, eta, t - tl[j]);

@@ -32,11 +32,21 @@ class NumpySim:
         self.t[w] = t
 
     def grad_event(self, t, i, s):
+        if self.variant == 2:  # Eq. (baselinedynamic): x alone, no flow
+            self.X[i] -= self.gamma * self.G[s]
+            self.t[i] = t
+            return
         self.mix(i, t)
         self.X[i] -= self.gamma * self.G[s]
         self.Xt[i] -= self.gamma * self.G[s]
 
     def comm_event(self, t, i, j):
+        if self.variant == 2:
+            m = self.X[i] - self.X[j]
+            self.X[i] -= self.alpha * m
+            self.X[j] += self.alpha * m
+            self.t[i] = self.t[j] = t
+            return
         if self.variant == 1:
             m = self.X[i] - self.X[j]
             self.mix(i, t)

@@ -30,6 +30,12 @@ MUTANTS = {
     "wrong_gradient_row": ("const double* g = G + (size_t)s * ldg;", "const double* g = G + (size_t)i * ldg;"),
     "consensus_not_centred": ("mean /= (double)n;\n        for (int32_t i = 0; i < n; ++i) {\n            const double dev = X[(size_t)i * ld + k] - mean;",
                               "mean /= (double)(n + 1);\n        for (int32_t i = 0; i < n; ++i) {\n            const double dev = X[(size_t)i * ld + k] - mean;"),
+    "plain_grad_sign": ("x[k] = x[k] - gamma * g[k];", "x[k] = x[k] + gamma * g[k];"),
+    "plain_comm_j_sign": ("y[k] = y[k] + alpha * m;", "y[k] = y[k] - alpha * m;"),
+    "plain_comm_message_reversed": ("const double m = x[k] - y[k];", "const double m = y[k] - x[k];"),
+    "plain_comm_forgets_time_j": ("a2o_plain_comm(xi, xj, d, alpha);\n                tl[i] = t;\n                tl[j] = t;",
+                                  "a2o_plain_comm(xi, xj, d, alpha);\n                tl[i] = t;"),
+    "plain_grad_touches_tilde": ("a2o_plain_grad(xi, g, d, gamma);", "a2o_plain_grad(xi, g, d, gamma); a2o_plain_grad(xti, g, d, gamma);"),
     "consensus_at_ignores_flow": ("mean += x - c * (x - xt);", "mean += x;"),
 }
 
@@ -46,6 +52,8 @@ DETECTORS = [
     lambda: pins.test_brute_force_matrix_exponential(pins.OracleSim, 3, 3, "complete"),
     lambda: pins.test_consensus_at_common_time_matches_flushed_state_and_definition(),
     lambda: pins.test_hand_example(pins.OracleSim),
+    lambda: pins.test_plain_dynamic_is_a_product_of_gossip_matrices(pins.OracleSim, 0.3),
+    lambda: pins.test_plain_dynamic_is_the_full_one_without_drift(),
 ]
 
 

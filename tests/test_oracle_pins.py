@@ -146,6 +146,69 @@ def test_baseline_equals_textbook_gossip_sgd(Sim):
     np.testing.assert_allclose(s.Xt, s.X, rtol=0, atol=1e-13)
 
 
+# ---- Eq. (baselinedynamic): the dynamic without the momentum buffer (variant 2) -----------
+@pytest.mark.parametrize("alpha", [0.5, 0.3])
+@pytest.mark.parametrize("Sim", SIMS)
+def test_plain_dynamic_is_a_product_of_gossip_matrices(Sim, alpha):
+    """Eq. (baselinedynamic) in matrix form (App. A notation): a communication on edge (i, j) multiplies
+    the stacked parameters by W = I - alpha (e_i - e_j)(e_i - e_j)^T, a gradient event subtracts
+    gamma e_i g^T. Written here with dense matrices; x~ must stay untouched, eta and alpha~ ignored."""
+    cfg = W.CONFIGS["cfg1"].scaled(d=7, n_events=300)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    xt0 = np.random.default_rng(3).standard_normal(x0.shape)
+    s = Sim(x0, 0.37, alpha, 1.9, cfg.gamma, grads=G, xt0=xt0, variant=2)
+    # the stream, then one last communication whose second worker is touched by nothing after it
+    times = np.append(ev.times, ev.times[-1] + 1.0)
+    wi, wj, slot = np.append(ev.wi, 2).astype(np.int32), np.append(ev.wj, 1).astype(np.int32), np.append(ev.slot, -1).astype(np.int32)
+    s.apply(times, wi, wj, slot)
+    n = cfg.n
+    ref = x0.copy()
+    eye = np.eye(n)
+    for i, j, sl in zip(wi, wj, slot):
+        if j < 0:
+            ref = ref - cfg.gamma * np.outer(eye[i], G[sl])
+        else:
+            u = eye[i] - eye[j]
+            ref = (eye - alpha * np.outer(u, u)) @ ref
+    np.testing.assert_allclose(s.X, ref, rtol=1e-12, atol=1e-13)
+    assert np.array_equal(s.Xt, xt0)
+    t_expect = np.zeros(n)
+    for t, i, j in zip(times, wi, wj):
+        t_expect[i] = t
+        if j >= 0:
+            t_expect[j] = t
+    assert np.array_equal(s.t, t_expect)
+
+
+def test_plain_dynamic_is_the_full_one_without_drift():
+    """The appendix of proofs restates Eq. (dynamic) and says it reduces to Eq. (baselinedynamic) when the
+    method is not applied: with eta = 0 the drift vanishes and x no longer sees x~, whatever alpha~ is.
+    With c = 0 exactly the x rows of the two runs go through the same operations, so they agree to the
+    bit; mean conservation and the contraction identity of a comm event hold for the plain run too."""
+    cfg = W.CONFIGS["cfg2"].scaled(d=9, n_events=600)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    full = OracleSim(x0, 0.0, 0.5, 2.3, cfg.gamma, grads=G, variant=0)
+    plain = OracleSim(x0, 0.8, 0.5, -7.0, cfg.gamma, grads=G, variant=2)
+    full.apply_stream(ev)
+    plain.apply_stream(ev)
+    assert np.array_equal(full.X, plain.X)
+    assert np.array_equal(plain.Xt, x0)
+    # sum over workers moves only by the gradient jumps (the remark on the mean in App. C)
+    gsum = sum(G[sl] for sl in ev.slot if sl >= 0)
+    np.testing.assert_allclose(plain.X.sum(0), x0.sum(0) - cfg.gamma * gsum, rtol=1e-12, atol=1e-12)
+    # one more comm event: consensus distance drops by 2 alpha (1 - alpha) |x_i - x_j|^2
+    alpha = 0.3
+    p2 = OracleSim(plain.X, 0.0, alpha, 0.0, 0.0, variant=2)
+    before = p2.consensus()
+    gap = float(((p2.X[1] - p2.X[4]) ** 2).sum())
+    p2.apply(*_one([0.0], [1], [4], [-1]))
+    np.testing.assert_allclose(before - p2.consensus(), 2 * alpha * (1 - alpha) * gap, rtol=1e-10)
+
+
 # ---- mean tracker: Eq. (mean) and the remark after (major:delta_f) in App. C -------------
 def test_mean_tracker_identity():
     cfg = W.CONFIGS["cfg1"].scaled(d=9, n_events=600)
@@ -349,7 +412,7 @@ def test_c_and_numpy_versions_agree_both_orderings():
     _, x0 = W.x0_matrix(cfg)
     _, G = W.grad_matrix(cfg)
     ev = W.config_events(cfg)
-    for variant in (0, 1):
+    for variant in (0, 1, 2):
         a = OracleSim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=variant)
         b = NumpySim(x0, 0.5, 0.5, 1.3, cfg.gamma, grads=G, variant=variant)
         a.apply_stream(ev)
