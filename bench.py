@@ -62,6 +62,7 @@ def parse_args():
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-resident-mode", action="store_true")
+    ap.add_argument("--skip-baseline-dynamic", action="store_true")
     return ap.parse_args()
 
 
@@ -240,8 +241,9 @@ def main():
     eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
                    device=str(device))
     fill_engine(eng, cfg, threads)
-    # three stretches of the stream: plans resident on the device, end to end, shared-memory-resident mode
-    ev_all = W.config_events(cfg, n_events=3 * n_steps * eps)
+    # four stretches of the stream: plans resident on the device, end to end, shared-memory-resident mode,
+    # and the asynchronous baseline without the momentum buffer
+    ev_all = W.config_events(cfg, n_events=4 * n_steps * eps)
 
     # ---- pass 1: descriptors resident on the device ---------------------------------------------
     plans, t_start = [], np.zeros(cfg.n)
@@ -339,6 +341,47 @@ def main():
         except B.A2Error as exc:
             resident = {"unavailable": str(exc)}
 
+    # ---- pass 4: the asynchronous baseline (no momentum buffer, half the rows), reported beside the main figure ---
+    plain = None
+    if not args.skip_baseline_dynamic:
+        eng.set_variant(B.A2_NO_MOMENTUM)
+        p_plans, t_start = [], eng.times()
+        for s in range(n_steps):
+            c = ev_all.slice((3 * n_steps + s) * eps, (3 * n_steps + s + 1) * eps)
+            p = eng.plan(c.times, c.wi, c.wj, c.slot, flags=flags, t_start=t_start)
+            t_start = p.sched.t_final(cfg.n)
+            p_plans.append(p)
+        marks = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
+        q_end = torch.cuda.Event(enable_timing=True)
+        p_bytes = p_launches = 0
+        for s in range(n_steps):
+            if s == W_:
+                torch.cuda.synchronize(device)
+                ranks.barrier()
+            marks[s][0].record(stream)
+            st = p_plans[s].run(want_stats=True)
+            marks[s][1].record(stream)
+            cons.append(eng.consensus_distance())
+            if s >= W_:
+                p_bytes += st["bytes_moved"]
+                p_launches += st["n_launches"]
+        q_end.record(stream)
+        torch.cuda.synchronize(device)
+        ranks.barrier()
+        p_ms = marks[W_][0].elapsed_time(q_end)
+        p_k1_ms = sum(marks[s][0].elapsed_time(marks[s][1]) for s in timed)
+        for p in p_plans:
+            p.close()
+        eng.set_variant(B.A2_MSG_AFTER_MIX)
+        p_value, p_slow = aggregate_throughput(ranks, K * eps, p_ms / 1e3)
+        plain = {"value": p_value, "unit": "events/s", "ms_per_step": 1e3 * p_slow / K,
+                 "kernel": "k_apply_events_plain", "achieved_gbs": p_bytes / (p_k1_ms / 1e3) / 1e9,
+                 "launches": p_launches,
+                 "note": "A2_NO_MOMENTUM: the paper's asynchronous baseline on the same stream recipe; x only, so "
+                         "an event moves half the bytes"}
+        if not all(np.isfinite(cons)):
+            raise SystemExit("non-finite consensus distance: the run is invalid")
+
     # ---- roofline of the event kernel ------------------------------------------------------------
     peak, peak_src = measured_peak()
     achieved = k1_bytes / (k1_ms / 1e3) / 1e9
@@ -370,7 +413,10 @@ def main():
         "consensus_kernel": {"ms": k2_ms / K, "gbs": consensus_gbs, "frac": consensus_gbs / peak},
         "batches_per_step": sum(stats[s]["n_batches"] for s in timed) / K,
         "resident_mode": resident,
+        "baseline_dynamic": plain,
     }
+    if plain is not None:
+        plain["frac"] = plain["achieved_gbs"] / peak
 
     if ranks.rank == 0 and ranks.world == 1 and not args.skip_cpu_baseline:
         cores = max(1, min(os.cpu_count() or 1, 32))

@@ -76,10 +76,18 @@ enum {
 /* Kinds of elementary operation inside an item. */
 enum { A2_OP_GRAD_A = 0, A2_OP_GRAD_B = 1, A2_OP_COMM = 2, A2_OP_MIX_A = 3 /* mixing only (a2cid2_flush) */ };
 
-/* Variants of the order of operations at a communication event. */
+/* Variants of the dynamic. */
 enum {
-    A2_MSG_AFTER_MIX = 0, /* message x_i - x_j taken at the event time, as Eq. (dynamic) states */
-    A2_MSG_BEFORE_MIX = 1 /* message taken from the un-mixed buffers, as Algorithm 1 is printed */
+    A2_MSG_AFTER_MIX = 0,  /* message x_i - x_j taken at the event time, as Eq. (dynamic) states */
+    A2_MSG_BEFORE_MIX = 1, /* message taken from the un-mixed buffers, as Algorithm 1 is printed */
+    A2_NO_MOMENTUM = 2     /* the asynchronous baseline, Eq. (baselinedynamic) of Sec. 3.2: what
+                              Eq. (dynamic) becomes without the method. There is no drift and no
+                              momentum buffer: gradient x_i -= gamma g; communication
+                              x_i -= alpha (x_i - x_j), x_j += alpha (x_i - x_j). x~ is never read or
+                              written (it may be left unbound), eta and alpha~ are ignored, and an
+                              event moves half the bytes. a2cid2_flush then only records the time,
+                              and the consensus distance at a common time is that of the stored
+                              rows. A2_SCHED_RESIDENT is not available (A2_EINVAL).               */
 };
 
 /* One item of a batch: all the work done on one worker (b = -1) or one pair of workers. */
@@ -99,7 +107,8 @@ typedef struct a2cid2_stats {
     int64_t n_launches; /* event-kernel launches (a batch is split if it exceeds a launch's caps) */
     int64_t n_items;
     int64_t bytes_moved;       /* rows read + rows written by the items, times d, times element size */
-    int64_t bytes_one_by_one;  /* the same stream applied one event per item: comm 8 rows, gradient 5 */
+    int64_t bytes_one_by_one;  /* the same stream applied one event per item: comm 8 rows, gradient 5
+                                  (4 and 3 under A2_NO_MOMENTUM)                                   */
     int64_t descriptor_bytes;  /* host-to-device bytes of the descriptors                        */
     double host_ms;            /* validation + scheduling + descriptor packing time on the host   */
 } a2cid2_stats;
@@ -115,26 +124,29 @@ typedef struct a2cid2_stats {
 int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_tilde, double gamma,
                   int32_t storage_dtype, a2cid2_t** out);
 
-/* Select A2_MSG_AFTER_MIX (default) or A2_MSG_BEFORE_MIX for later events. */
+/* Select A2_MSG_AFTER_MIX (default), A2_MSG_BEFORE_MIX or A2_NO_MOMENTUM for later events.
+ * A2_ESTATE when leaving A2_NO_MOMENTUM while no x~ buffer is bound. */
 int a2cid2_set_variant(a2cid2_t* h, int32_t variant);
 
 /* Lend the device buffers: x and x_tilde are [n, row_pitch_elems], grads is
  * [n_grad_slots, row_pitch_elems] (may be NULL with n_grad_slots = 0 if no gradient event is
  * ever applied), all of the storage type, row-major, 16-byte aligned. row_pitch_elems >= d and
  * a multiple of 8; the columns between d and the pitch are padding that the library may
- * overwrite. cuda_stream is a cudaStream_t (NULL = default stream). The caller keeps ownership
+ * overwrite. x_tilde may be NULL only while the variant is A2_NO_MOMENTUM. cuda_stream is a cudaStream_t (NULL = default stream). The caller keeps ownership
  * and must keep the buffers alive until a2cid2_sync/destroy. May be called again to re-bind. */
 int a2cid2_bind(a2cid2_t* h, void* x, void* x_tilde, void* grads, int32_t n_grad_slots,
                 int64_t row_pitch_elems, void* cuda_stream);
 
 /* Copy a dense host [n, d] array of the storage type into x; x~ from host_x_tilde, or a copy
- * of x when NULL (Algorithm 1: x~ <- x); times from host_t[n], or zeros when NULL. Waits. */
+ * of x when NULL (Algorithm 1: x~ <- x); times from host_t[n], or zeros when NULL. Waits.
+ * Without a bound x~ buffer only x is written (host_x_tilde must then be NULL). */
 int a2cid2_write_state(a2cid2_t* h, const void* host_x, const void* host_x_tilde, const double* host_t);
 
 /* Copy dense host rows [n_slots, d] into gradient rows first_slot.. . Waits. */
 int a2cid2_write_grads(a2cid2_t* h, int32_t first_slot, int32_t n_slots, const void* host_g);
 
-/* Copy x, x~ (dense [n, d], storage type) and t[n] to the host; any pointer may be NULL. Waits. */
+/* Copy x, x~ (dense [n, d], storage type) and t[n] to the host; any pointer may be NULL. Waits.
+ * A2_ESTATE if host_x_tilde is given while no x~ buffer is bound. */
 int a2cid2_read_state(a2cid2_t* h, void* host_x, void* host_x_tilde, double* host_t);
 
 /* Copy the workers' last-event times t[n] (kept on the host) without touching the device. */
@@ -267,7 +279,8 @@ int a2cid2_sched_ops(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, i
 int a2cid2_sched_t_final(const a2cid2_sched_t* s, double* t_out);
 
 /* Fill the descriptor-derived counters (events, batches, items, launches, bytes for d columns
- * of elem_bytes each) for batches [first_batch, first_batch + n_batches); -1 = all remaining. */
+ * of elem_bytes each, counted for the dynamic with the momentum buffer) for batches
+ * [first_batch, first_batch + n_batches); -1 = all remaining. */
 int a2cid2_sched_stats(const a2cid2_sched_t* s, int64_t first_batch, int64_t n_batches, int64_t d,
                        int32_t elem_bytes, a2cid2_stats* out);
 

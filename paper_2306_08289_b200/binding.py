@@ -21,7 +21,7 @@ A2_F32, A2_BF16 = 0, 1
 A2_SCHED_FUSE = 1
 A2_SCHED_RESIDENT = 2
 A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A = 0, 1, 2, 3
-A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX = 0, 1
+A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX, A2_NO_MOMENTUM = 0, 1, 2
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
                A2_ECUDA: "A2_ECUDA", A2_ESTATE: "A2_ESTATE"}
@@ -267,7 +267,7 @@ class Engine:
     stream only). x, x~ and the gradient buffer are torch tensors of shape [rows, pitch]."""
 
     def __init__(self, n, d, eta, alpha, alpha_tilde, gamma, storage="f32", n_grad_slots=None, device="cuda:0",
-                 stream=None, rows_16B_only=False):
+                 stream=None, rows_16B_only=False, momentum=True):
         import torch
 
         self.torch = torch
@@ -281,6 +281,9 @@ class Engine:
         h = _vp()
         _check(lib().a2cid2_create(self.n, self.d, eta, alpha, alpha_tilde, gamma, self.dtype_code, C.byref(h)))
         self._h = h
+        self.momentum = bool(momentum)  # False: the dynamic without x~ (A2_NO_MOMENTUM), no x~ buffer at all
+        if not self.momentum:
+            _check(lib().a2cid2_set_variant(self._h, A2_NO_MOMENTUM), self._h)
         self.device = torch.device(device)
         # rows start on 32-byte boundaries so that the kernels can use 256-bit accesses
         # (rows_16B_only: start them 16 bytes off instead, which is all the ABI requires)
@@ -294,10 +297,10 @@ class Engine:
                 return flat[shift:].view(r, self.pitch)
 
             self.x = rows(self.n)
-            self.xt = rows(self.n)
+            self.xt = rows(self.n) if self.momentum else None
             self.g = rows(max(self.n_slots, 1))
             self.stream = torch.cuda.current_stream(self.device) if stream is None else stream
-            _check(lib().a2cid2_bind(self._h, self.x.data_ptr(), self.xt.data_ptr(),
+            _check(lib().a2cid2_bind(self._h, self.x.data_ptr(), self.xt.data_ptr() if self.momentum else None,
                                      self.g.data_ptr() if self.n_slots > 0 else None, self.n_slots, self.pitch,
                                      self.stream.cuda_stream), self._h)
 
@@ -320,9 +323,10 @@ class Engine:
 
     def read_state(self):
         x = np.empty((self.n, self.d), dtype=self.np_dtype)
-        xt = np.empty((self.n, self.d), dtype=self.np_dtype)
+        xt = np.empty((self.n, self.d), dtype=self.np_dtype) if self.xt is not None else None
         t = np.empty(self.n, dtype=np.float64)
-        _check(lib().a2cid2_read_state(self._h, x.ctypes.data, xt.ctypes.data, _ptr(t, _dp)), self._h)
+        _check(lib().a2cid2_read_state(self._h, x.ctypes.data, None if xt is None else xt.ctypes.data, _ptr(t, _dp)),
+               self._h)
         return x, xt, t
 
     def times(self):

@@ -67,7 +67,9 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
                    const int32_t* wi, const int32_t* wj, const int32_t* slot, uint32_t flags,
                    int32_t max_ops_per_item, a2cid2_sched** out, std::string& err);
 
-void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out);
+// momentum = false counts the rows of the dynamic without x~ (Eq. (baselinedynamic)).
+void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, bool momentum,
+                    a2cid2_stats* out);
 
 // ---- device descriptors (layout shared by host packing and the event kernel) ---------------
 struct DevItem {
@@ -107,6 +109,7 @@ struct EventLaunch {
 struct DeviceInfo {
     int sm_count = 0;
     int event_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // [storage type][128-bit / 256-bit accesses]
+    int plain_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the kernel of the dynamic without x~
     int consensus_ctas_per_sm = 0;
 };
 

@@ -171,6 +171,8 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
     pk.resident = (s.flags & A2_SCHED_RESIDENT) != 0;
     pk.ops_off = align16(s.items.size() * sizeof(DevItem));
     size_t end = pk.ops_off + s.ops.size() * sizeof(DevOp);
+    if (pk.resident && h->variant == A2_NO_MOMENTUM)
+        return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT is not available for the A2_NO_MOMENTUM variant");
     if (!pk.resident) {
         make_launches(s, pk.launches, pk.batch_launch_first);
     } else {
@@ -227,6 +229,8 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     const DevItem* d_items = reinterpret_cast<const DevItem*>(base);
     const DevOp* d_ops = reinterpret_cast<const DevOp*>(base + pk.ops_off);
     if (pk.resident) {
+        if (h->variant == A2_NO_MOMENTUM)
+            return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT is not available for the A2_NO_MOMENTUM variant");
         a2::ResidentLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.n = h->n; L.dtype = h->dtype; L.variant = h->variant; L.eta = h->eta;
@@ -293,7 +297,7 @@ int run_plan_graph(a2cid2* h, a2cid2_plan* p) {
 // Descriptor-derived counters of batches [b0, b1).
 void fill_stats(const a2cid2* h, const a2cid2_sched& s, const Packed& pk, int64_t b0, int64_t b1, a2cid2_stats* st) {
     const int32_t eb = (int32_t)elem_bytes(h->dtype);
-    a2::schedule_stats(s, b0, b1, h->d, eb, st);
+    a2::schedule_stats(s, b0, b1, h->d, eb, h->variant != A2_NO_MOMENTUM, st);
     if (pk.resident) {  // the state crosses HBM once each way, every cached gradient row once per chunk
         st->n_launches = b1 > b0 ? 2 : 0;
         st->bytes_moved = b1 > b0 ? ((int64_t)4 * h->n + (int64_t)pk.g_rows.size()) * h->d * eb : 0;
@@ -354,7 +358,10 @@ int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_t
 
 int a2cid2_set_variant(a2cid2_t* h, int32_t variant) {
     if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
-    if (variant != A2_MSG_AFTER_MIX && variant != A2_MSG_BEFORE_MIX) return fail(h, A2_EINVAL, "unknown variant");
+    if (variant != A2_MSG_AFTER_MIX && variant != A2_MSG_BEFORE_MIX && variant != A2_NO_MOMENTUM)
+        return fail(h, A2_EINVAL, "unknown variant");
+    if (variant != A2_NO_MOMENTUM && h->bound && !h->xt)
+        return fail(h, A2_ESTATE, "this variant needs an x_tilde buffer and none is bound");
     h->variant = variant;
     h->bind_epoch += 1;
     return A2_OK;
@@ -363,7 +370,9 @@ int a2cid2_set_variant(a2cid2_t* h, int32_t variant) {
 int a2cid2_bind(a2cid2_t* h, void* x, void* x_tilde, void* grads, int32_t n_grad_slots, int64_t row_pitch_elems,
                 void* cuda_stream) {
     if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
-    if (!x || !x_tilde) return fail(h, A2_EINVAL, "x or x_tilde is NULL");
+    if (!x) return fail(h, A2_EINVAL, "x is NULL");
+    if (!x_tilde && h->variant != A2_NO_MOMENTUM)
+        return fail(h, A2_EINVAL, "x_tilde is NULL (only the A2_NO_MOMENTUM variant runs without it)");
     if (n_grad_slots < 0 || (n_grad_slots > 0 && !grads)) return fail(h, A2_EINVAL, "bad gradient buffer");
     if (row_pitch_elems < h->d || row_pitch_elems % 8 != 0)
         return fail(h, A2_EINVAL, "row pitch must be >= d and a multiple of 8 elements");
@@ -384,14 +393,16 @@ int a2cid2_write_state(a2cid2_t* h, const void* host_x, const void* host_x_tilde
     int rc = need_bound(h);
     if (rc != A2_OK) return rc;
     if (!host_x) return fail(h, A2_EINVAL, "host_x is NULL");
+    if (host_x_tilde && !h->xt) return fail(h, A2_EINVAL, "host_x_tilde given but no x_tilde buffer is bound");
     if (host_t)
         for (int32_t w = 0; w < h->n; ++w)
             if (!std::isfinite(host_t[w])) return fail(h, A2_EINVAL, "non-finite worker time");
     const size_t eb = elem_bytes(h->dtype);
     const size_t row = (size_t)h->d * eb, pitch = (size_t)h->pitch * eb;
     A2_CUDA(h, cudaMemcpy2DAsync(h->x, pitch, host_x, row, row, (size_t)h->n, cudaMemcpyHostToDevice, h->stream));
-    A2_CUDA(h, cudaMemcpy2DAsync(h->xt, pitch, host_x_tilde ? host_x_tilde : host_x, row, row, (size_t)h->n,
-                                 cudaMemcpyHostToDevice, h->stream));
+    if (h->xt)
+        A2_CUDA(h, cudaMemcpy2DAsync(h->xt, pitch, host_x_tilde ? host_x_tilde : host_x, row, row, (size_t)h->n,
+                                     cudaMemcpyHostToDevice, h->stream));
     A2_CUDA(h, cudaStreamSynchronize(h->stream));
     for (int32_t w = 0; w < h->n; ++w) h->t[(size_t)w] = host_t ? host_t[w] : 0.0;
     return A2_OK;
@@ -414,6 +425,7 @@ int a2cid2_write_grads(a2cid2_t* h, int32_t first_slot, int32_t n_slots, const v
 int a2cid2_read_state(a2cid2_t* h, void* host_x, void* host_x_tilde, double* host_t) {
     int rc = need_bound(h);
     if (rc != A2_OK) return rc;
+    if (host_x_tilde && !h->xt) return fail(h, A2_ESTATE, "no x_tilde buffer is bound");
     const size_t eb = elem_bytes(h->dtype);
     const size_t row = (size_t)h->d * eb, pitch = (size_t)h->pitch * eb;
     if (host_x)
@@ -506,6 +518,10 @@ int a2cid2_flush(a2cid2_t* h, double t_flush) {
     if (!std::isfinite(t_flush)) return fail(h, A2_EINVAL, "t_flush must be finite");
     for (int32_t w = 0; w < h->n; ++w)
         if (t_flush < h->t[(size_t)w]) return fail(h, A2_EORDER, "t_flush precedes a worker's last event");
+    if (h->variant == A2_NO_MOMENTUM) {  // no flow between events: only the clock moves
+        h->t.assign((size_t)h->n, t_flush);
+        return A2_OK;
+    }
     a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
     if (!s) return fail(h, A2_ENOMEM, "out of host memory");
     s->n = h->n;
@@ -527,12 +543,15 @@ int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out) {
     int rc = need_bound(h);
     if (rc != A2_OK) return rc;
     if (!out) return fail(h, A2_EINVAL, "out is NULL");
-    const bool flush = !std::isnan(t_eval);
+    bool flush = !std::isnan(t_eval);
     const int np = a2::consensus_grid(h->dev);
     if (flush) {
         if (!std::isfinite(t_eval)) return fail(h, A2_EINVAL, "t_eval must be finite or NaN");
         for (int32_t w = 0; w < h->n; ++w)
             if (t_eval < h->t[(size_t)w]) return fail(h, A2_EORDER, "t_eval precedes a worker's last event");
+        if (h->variant == A2_NO_MOMENTUM) flush = false;  // the rows do not move between events
+    }
+    if (flush) {
         // the staging buffer is free: every earlier call waited for the stream before returning
         for (int32_t w = 0; w < h->n; ++w) h->h_pinned[w] = t_eval - h->t[(size_t)w];
         A2_CUDA(h, cudaMemcpyAsync(h->d_dt, h->h_pinned, sizeof(double) * (size_t)h->n, cudaMemcpyHostToDevice, h->stream));
@@ -750,7 +769,7 @@ int a2cid2_sched_stats(const a2cid2_sched_t* s, int64_t first_batch, int64_t n_b
     if (n_batches < 0) n_batches = nb - first_batch;
     if (first_batch < 0 || n_batches < 0 || first_batch + n_batches > nb || d < 0 || elem_bytes_ <= 0)
         return fail(nullptr, A2_ERANGE, "batch range out of bounds");
-    a2::schedule_stats(*s, first_batch, first_batch + n_batches, d, elem_bytes_, out);
+    a2::schedule_stats(*s, first_batch, first_batch + n_batches, d, elem_bytes_, true, out);
     std::vector<LaunchRange> launches;
     std::vector<int64_t> bf;
     make_launches(*s, launches, bf);

@@ -327,6 +327,191 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Event kernel of the dynamic without the momentum buffer (Eq. (baselinedynamic), Sec. 3.2):
+//   gradient  x -= gamma g                       comm  m = x_a - x_b;  x_a -= alpha m;  x_b += alpha m
+// Same descriptors, same unit mapping, half the rows: x_a, x_b and the gradient rows. There is no
+// flow between events, so times play no part on the device and a mixing-only operation does nothing.
+// ---------------------------------------------------------------------------------------------
+#ifndef A2_PLAIN_UNROLL
+#define A2_PLAIN_UNROLL 2  // 256-bit vectors per thread and tile
+#endif
+#ifndef A2_PLAIN_UNROLL_128
+#define A2_PLAIN_UNROLL_128 4  // the same bytes per thread with 128-bit vectors
+#endif
+template <int BYTES> struct PlainCfg { static constexpr int UNROLL = BYTES == 32 ? A2_PLAIN_UNROLL : A2_PLAIN_UNROLL_128; };
+
+template <typename T, int BYTES, int UNROLL>
+__global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const EventArgs p) {
+    using V = Vec<T, BYTES>;
+    constexpr int N = V::N;
+    __shared__ DevItem s_items[kMaxItemsPerLaunch];
+    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) s_kind[o] = (unsigned char)p.ops[o].kind;
+    __syncthreads();
+
+    T* const X = static_cast<T*>(p.x);
+    const T* const G = static_cast<const T*>(p.g);
+    const float alpha = p.alpha, ngamma = -p.gamma;
+    const long long n_units = (long long)p.n_items * p.n_tiles;
+    const int n_it = p.n_items;
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int rem = (int)(unit % n_it);
+        const long long tile = unit / n_it;
+        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+        const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
+        T* const pxa = X + (long long)it.a * p.pitch;
+        T* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
+        const T* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
+        const T* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+
+        float xa[UNROLL][N], xb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N];
+        bool live[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long v = v0 + (long long)u * kEventThreads;
+            live[u] = v < p.n_vec;
+            const long long off = v * N;
+#pragma unroll
+            for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
+            if (live[u]) {
+                V::load(pxa + off, xa[u]);
+                if (has_b) V::load(pxb + off, xb[u]);
+                if (has_ga) V::load(pga + off, ga[u]);
+                if (has_gb) V::load(pgb + off, gb[u]);
+            }
+        }
+        bool dirty = false;
+        for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
+            const int kind = s_kind[o];
+            if (kind == A2_OP_MIX_A) continue;
+            dirty = true;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                for (int k = 0; k < N; ++k) {
+                    if (kind == A2_OP_GRAD_A) {
+                        xa[u][k] = __fmaf_rn(ngamma, ga[u][k], xa[u][k]);
+                    } else if (kind == A2_OP_GRAD_B) {
+                        xb[u][k] = __fmaf_rn(ngamma, gb[u][k], xb[u][k]);
+                    } else {
+                        const float m = __fsub_rn(xa[u][k], xb[u][k]);
+                        xa[u][k] = __fmaf_rn(-alpha, m, xa[u][k]);
+                        xb[u][k] = __fmaf_rn(alpha, m, xb[u][k]);
+                    }
+                }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long off = (v0 + (long long)u * kEventThreads) * N;
+            if (live[u] && dirty) {
+                V::store(pxa + off, xa[u]);
+                if (has_b) V::store(pxb + off, xb[u]);
+            }
+        }
+    }
+}
+
+// The same for bf16 rows. Half the bytes per column means twice the columns in flight for the same
+// DRAM traffic, and widening every row to fp32 on arrival would spend the register file on that. So the
+// rows stay packed (two columns per 32-bit register) while the loads are in flight, and each pair of
+// columns is widened, taken through the item's operations and rounded back on its own.
+#ifndef A2_PLAIN_BF16_UNROLL
+#define A2_PLAIN_BF16_UNROLL 1  // 256-bit vectors per thread and tile (the 128-bit kernel takes twice as many)
+#endif
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t bf16_pack(float lo, float hi) {  // round to nearest even
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+template <int WORDS, int UNROLL>
+__global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const EventArgs p) {
+    __shared__ DevItem s_items[kMaxItemsPerLaunch];
+    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) s_kind[o] = (unsigned char)p.ops[o].kind;
+    __syncthreads();
+
+    __nv_bfloat16* const X = static_cast<__nv_bfloat16*>(p.x);
+    const __nv_bfloat16* const G = static_cast<const __nv_bfloat16*>(p.g);
+    const float alpha = p.alpha, ngamma = -p.gamma;
+    const long long n_units = (long long)p.n_items * p.n_tiles;
+    const int n_it = p.n_items;
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int rem = (int)(unit % n_it);
+        const long long tile = unit / n_it;
+        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+        const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
+        __nv_bfloat16* const pxa = X + (long long)it.a * p.pitch;
+        __nv_bfloat16* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
+        const __nv_bfloat16* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
+        const __nv_bfloat16* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+
+        uint32_t xa[UNROLL][WORDS], xb[UNROLL][WORDS], ga[UNROLL][WORDS], gb[UNROLL][WORDS];
+        bool live[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long v = v0 + (long long)u * kEventThreads;
+            live[u] = v < p.n_vec;
+            const long long off = v * (2 * WORDS);
+#pragma unroll
+            for (int k = 0; k < WORDS; ++k) { xa[u][k] = 0u; xb[u][k] = 0u; ga[u][k] = 0u; gb[u][k] = 0u; }
+            if (live[u]) {
+                Words<WORDS>::ld(pxa + off, xa[u]);
+                if (has_b) Words<WORDS>::ld(pxb + off, xb[u]);
+                if (has_ga) Words<WORDS>::ld(pga + off, ga[u]);
+                if (has_gb) Words<WORDS>::ld(pgb + off, gb[u]);
+            }
+        }
+        const int o_begin = it.op_first, o_end = it.op_first + it.op_count;
+        bool dirty = false;
+        for (int o = o_begin; o < o_end; ++o) dirty |= s_kind[o] != A2_OP_MIX_A;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+            for (int k = 0; k < WORDS; ++k) {
+                float a0 = bf16_lo(xa[u][k]), a1 = bf16_hi(xa[u][k]);
+                float b0 = bf16_lo(xb[u][k]), b1 = bf16_hi(xb[u][k]);
+                const float ga0 = bf16_lo(ga[u][k]), ga1 = bf16_hi(ga[u][k]);
+                const float gb0 = bf16_lo(gb[u][k]), gb1 = bf16_hi(gb[u][k]);
+                for (int o = o_begin; o < o_end; ++o) {
+                    const int kind = s_kind[o];
+                    if (kind == A2_OP_GRAD_A) {
+                        a0 = __fmaf_rn(ngamma, ga0, a0);
+                        a1 = __fmaf_rn(ngamma, ga1, a1);
+                    } else if (kind == A2_OP_GRAD_B) {
+                        b0 = __fmaf_rn(ngamma, gb0, b0);
+                        b1 = __fmaf_rn(ngamma, gb1, b1);
+                    } else if (kind == A2_OP_COMM) {
+                        const float m0 = __fsub_rn(a0, b0), m1 = __fsub_rn(a1, b1);
+                        a0 = __fmaf_rn(-alpha, m0, a0);
+                        a1 = __fmaf_rn(-alpha, m1, a1);
+                        b0 = __fmaf_rn(alpha, m0, b0);
+                        b1 = __fmaf_rn(alpha, m1, b1);
+                    }
+                }
+                xa[u][k] = bf16_pack(a0, a1);
+                xb[u][k] = bf16_pack(b0, b1);
+            }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long off = (v0 + (long long)u * kEventThreads) * (2 * WORDS);
+            if (live[u] && dirty) {
+                Words<WORDS>::st(pxa + off, xa[u]);
+                if (has_b) Words<WORDS>::st(pxb + off, xb[u]);
+            }
+        }
+    }
+}
+
 // Vectors per thread and tile. 256-bit accesses: one vector per thread already keeps 4-6 rows x 32 B
 // in flight per thread; 128-bit fp32 uses two.
 template <typename T, int BYTES> struct EventCfg { static constexpr int UNROLL = 1; };
@@ -436,6 +621,46 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     return (int)cudaGetLastError();
 }
 
+template <typename T, int BYTES>
+int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
+    constexpr int U = PlainCfg<BYTES>::UNROLL;
+    constexpr int N = Vec<T, BYTES>::N;
+    EventArgs a;
+    a.x = L.x; a.xt = nullptr; a.g = L.g; a.pitch = L.pitch;
+    a.n_vec = (L.d + N - 1) / N;
+    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
+    const long long vec_per_tile = (long long)kEventThreads * U;
+    a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
+    a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
+    a.msg_before_mix = 0;
+    const long long n_units = (long long)a.n_items * a.n_tiles;
+    const int per_sm = dev.plain_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
+    long long grid = (long long)dev.sm_count * per_sm;
+    if (grid > n_units) grid = n_units;
+    if (grid < 1) return 0;
+    k_apply_events_plain<T, BYTES, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    return (int)cudaGetLastError();
+}
+
+template <int WORDS>
+int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
+    constexpr int U = A2_PLAIN_BF16_UNROLL * (8 / WORDS);
+    EventArgs a;
+    a.x = L.x; a.xt = nullptr; a.g = L.g; a.pitch = L.pitch;
+    a.n_vec = (L.d + 2 * WORDS - 1) / (2 * WORDS);
+    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
+    const long long vec_per_tile = (long long)kEventThreads * U;
+    a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
+    a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
+    a.msg_before_mix = 0;
+    const long long n_units = (long long)a.n_items * a.n_tiles;
+    long long grid = (long long)dev.sm_count * dev.plain_ctas_per_sm[1][WORDS == 8 ? 1 : 0];
+    if (grid > n_units) grid = n_units;
+    if (grid < 1) return 0;
+    k_apply_events_plain_bf16<WORDS, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    return (int)cudaGetLastError();
+}
+
 // Resident CTAs per SM the persistent grid is sized for, measured on B200 with 64 rows of 25.6e6
 // columns. fp32 rows, fused ring batches, 256-bit accesses: 1 CTA/SM 5.13 TB/s, 2: 6.33, 3: 6.01,
 // 4: 5.97 -- beyond two CTAs the extra concurrent row streams cost more DRAM locality than the extra
@@ -449,6 +674,15 @@ cudaError_t event_occupancy(int* out) {
     int occ = 0;
     const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
         &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL>, kEventThreads, 0);
+    *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
+    return e;
+}
+
+template <typename T, int BYTES>
+cudaError_t plain_occupancy(int* out) {
+    int occ = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &occ, k_apply_events_plain<T, BYTES, PlainCfg<BYTES>::UNROLL>, kEventThreads, 0);
     *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
     return e;
 }
@@ -501,6 +735,25 @@ int query_device(DeviceInfo* info) {
     if ((e = event_occupancy<float, 32>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<__nv_bfloat16, 16>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
     info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
+    if ((e = plain_occupancy<float, 16>(&info->plain_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = plain_occupancy<float, 32>(&info->plain_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    {
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<4, 2 * A2_PLAIN_BF16_UNROLL>,
+                                                          kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->plain_ctas_per_sm[1][0] = occ > 4 ? 4 : (occ > 0 ? occ : 1);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<8, A2_PLAIN_BF16_UNROLL>,
+                                                          kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->plain_ctas_per_sm[1][1] = occ > 4 ? 4 : (occ > 0 ? occ : 1);
+    }
+    if (const char* v = std::getenv("A2CID2_PLAIN_CTAS_PER_SM")) {  // tuning override, as for the event kernel
+        const int k = std::atoi(v);
+        if (k > 0)
+            for (auto& row : info->plain_ctas_per_sm)
+                for (int& c : row) c = k;
+    }
     info->consensus_ctas_per_sm = 8;  // capacity of the partial-sum scratch, CTAs per SM
     if (const char* v = std::getenv("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
         const int k = std::atoi(v);
@@ -514,6 +767,16 @@ int query_device(DeviceInfo* info) {
 int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.n_items <= 0) return 0;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (L.variant == A2_NO_MOMENTUM) {
+        const bool wide_x = rows_32B_aligned(L.x, nullptr, L.g, L.pitch, L.dtype);
+        if (L.dtype == A2_BF16) {
+            static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+            const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.g);
+            const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;
+            return wide_bf16 ? launch_plain_bf16<8>(L, dev, stream) : launch_plain_bf16<4>(L, dev, stream);
+        }
+        return wide_x ? launch_plain_t<float, 32>(L, dev, stream) : launch_plain_t<float, 16>(L, dev, stream);
+    }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
     if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16>(L, dev, stream);
     return wide ? launch_events_t<float, 32>(L, dev, stream) : launch_events_t<float, 16>(L, dev, stream);

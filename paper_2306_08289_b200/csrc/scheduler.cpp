@@ -219,19 +219,24 @@ void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResC
     close((int32_t)s.items.size());
 }
 
-void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, a2cid2_stats* out) {
+void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, bool momentum,
+                    a2cid2_stats* out) {
     a2cid2_stats st{};
     const int64_t i0 = s.batch_first[(size_t)b0], i1 = s.batch_first[(size_t)b1];
     int64_t rows_moved = 0, rows_single = 0;
     for (int64_t k = i0; k < i1; ++k) {
         const SchedItem& it = s.items[(size_t)k];
-        const int64_t state_rows = it.b >= 0 ? 4 : 2;
-        rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0);
+        const int64_t per_worker = momentum ? 2 : 1;  // x and x~, or x alone
+        const int64_t state_rows = (it.b >= 0 ? 2 : 1) * per_worker;
+        bool touches_state = momentum;  // without x~ a mixing-only item moves nothing
+        for (int32_t o = 0; o < it.n_ops && !touches_state; ++o)
+            touches_state = s.ops[(size_t)(it.first_op + o)].kind != A2_OP_MIX_A;
+        if (touches_state) rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0);
         for (int32_t o = 0; o < it.n_ops; ++o) {
             const int32_t kind = s.ops[(size_t)(it.first_op + o)].kind;
-            if (kind == A2_OP_COMM) { st.n_comm += 1; rows_single += 8; }
-            else if (kind == A2_OP_MIX_A) { rows_single += 4; }
-            else { st.n_grad += 1; rows_single += 5; }
+            if (kind == A2_OP_COMM) { st.n_comm += 1; rows_single += momentum ? 8 : 4; }
+            else if (kind == A2_OP_MIX_A) { rows_single += momentum ? 4 : 0; }
+            else { st.n_grad += 1; rows_single += momentum ? 5 : 3; }
         }
     }
     st.n_events = st.n_comm + st.n_grad;

@@ -17,7 +17,10 @@ bf16 storage -- bar 2e-2, applied norm-wise against the plain fp64 run:
       the engine writes them back, i.e. after every item): bound 5e-2 (a few bf16 ulps: the two
       runs differ where fp32 and fp64 arithmetic round a store to different neighbours, and
       those one-ulp differences are integrated like any other perturbation);
-    * with the plain fp64 run: bound 0.3.
+    * with the plain fp64 run: bound 0.3 (rows of >= 256 columns, like the norm: on a row of one or two
+      columns the floor of the metric is the element itself, and what the storage format loses over a few
+      hundred events is then measured against a value that has shrunk towards zero -- an ideal
+      bf16-storage run of 2 workers x 1 column is already 0.38 away from the fp64 run).
 """
 from __future__ import annotations
 
@@ -61,6 +64,15 @@ def oracle_params(cfg):
     return tuple(float(v) for v in spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3])
 
 
+class _XOnly:
+    """View of a simulator in which x stands in for x~ too, for engines that hold x alone."""
+
+    def __init__(self, sim):
+        self.X = sim.X
+        self.Xt = sim.X
+        self.t = sim.t
+
+
 class Checker:
     """The fp64 run, plus (bf16 storage only) a second fp64 run whose rows are rounded to bf16
     wherever the engine stores them."""
@@ -84,10 +96,15 @@ class Checker:
                 self.stored.round_rows([it.a] + ([it.b] if it.b >= 0 else []))
 
     def compare(self, x, xt, t, where="", cols=None):
-        """x, xt: widened device state (optionally only the columns `cols` of the checker)."""
+        """x, xt: widened device state (optionally only the columns `cols` of the checker). xt = None
+        (an engine without a momentum buffer): x alone is compared."""
         pl, st = self.plain, self.stored
         sel = (lambda a: a) if cols is None else (lambda a: a[:, cols])
         assert np.array_equal(t, pl.t), f"times differ {where}"
+        if xt is None:
+            xt = x
+            pl = _XOnly(pl)
+            st = None if st is None else _XOnly(st)
         out = {"elem_plain": max(rel_err(x, sel(pl.X)), rel_err(xt, sel(pl.Xt)))}
         if st is None:
             assert out["elem_plain"] <= TOL["f32"], f"parity {where}: {out}"
@@ -96,19 +113,23 @@ class Checker:
             out["norm_plain"] = max(row_norm_err(x, sel(pl.X)), row_norm_err(xt, sel(pl.Xt)))
             if x.shape[1] >= BF16_NORM_MIN_COLS:
                 assert out["norm_plain"] <= TOL["bf16"], f"parity {where}: {out}"
+                assert out["elem_plain"] <= BF16_ELEM_PLAIN_BOUND, f"parity {where}: {out}"
             assert out["elem_stored"] <= BF16_ELEM_STORED_BOUND, f"parity {where}: {out}"
-            assert out["elem_plain"] <= BF16_ELEM_PLAIN_BOUND, f"parity {where}: {out}"
         return out
 
 
-def make_small(cfg, variant=0):
-    """Engine + checker for a configuration whose arrays fit the host: same stored inputs on both."""
+def make_small(cfg, variant=0, momentum=True):
+    """Engine + checker for a configuration whose arrays fit the host: same stored inputs on both.
+    momentum=False: an engine with no x~ buffer (the variant is then A2_NO_MOMENTUM)."""
     xs, xw = W.x0_matrix(cfg)
     gs, gw = W.grad_matrix(cfg)
-    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots)
+    if not momentum:
+        variant = B.A2_NO_MOMENTUM
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
+                   momentum=momentum)
     eng.write_state(xs)
     eng.write_grads(gs)
-    if variant:
+    if variant and momentum:
         eng.set_variant(variant)
     chk = Checker(xw, oracle_params(cfg), cfg.gamma, gw, cfg.storage, variant=variant)
     return eng, chk
@@ -131,6 +152,7 @@ def run_batches_and_check(eng, chk, ev, flags, every=1):
         chk.apply_batch(ev, plan.sched, b)
         if b % every == 0 or b == nb - 1:
             x, xt, t = eng.read_state()
-            _merge(worst, chk.compare(widen(x, chk.storage), widen(xt, chk.storage), t, where=f"after batch {b}/{nb}"))
+            _merge(worst, chk.compare(widen(x, chk.storage), None if xt is None else widen(xt, chk.storage), t,
+                                      where=f"after batch {b}/{nb}"))
     plan.close()
     return worst, nb

@@ -87,6 +87,13 @@ def test_create_validates_without_a_device():
     back = np.zeros(4)
     assert L.a2cid2_times(h, back.ctypes.data_as(C.POINTER(C.c_double))) == B.A2_OK and np.array_equal(back, tt)
     assert L.a2cid2_sync(h) == B.A2_OK
+    for v in (B.A2_MSG_BEFORE_MIX, B.A2_NO_MOMENTUM, B.A2_MSG_AFTER_MIX):
+        assert L.a2cid2_set_variant(h, v) == B.A2_OK
+    assert L.a2cid2_set_variant(h, 3) == B.A2_EINVAL and L.a2cid2_set_variant(h, -1) == B.A2_EINVAL
+    # binding without an x~ buffer is refused unless the variant has no momentum (checked before any device call)
+    dummy = C.c_void_p(4096)
+    assert L.a2cid2_bind(h, dummy, None, None, 0, 16, None) == B.A2_EINVAL
+    assert b"x_tilde" in L.a2cid2_last_error(h)
     L.a2cid2_destroy(h)
     L.a2cid2_destroy(None)
 
