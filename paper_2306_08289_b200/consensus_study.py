@@ -37,7 +37,8 @@ def run_setting(n, d, graph, comms_per_grad, accelerated, T, gamma, g_std, pool,
     ev = W.poisson_events(n, edges, rates, n_events, seed=seed, grad_pool=pool)
     rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 7])))
     x0 = np.tile((rng.standard_normal(d) * 0.02).astype(np.float32), (n, 1))  # consensus at the start
-    eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n * pool, device=device)
+    # the baseline has eta = 0 and alpha~ = alpha: x~ would stay a copy of x, so it runs without the buffer
+    eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n * pool, device=device, momentum=bool(accelerated))
     eng.write_state(x0)
     for row in range(n * pool):
         eng.fill_row("g", row, (rng.standard_normal(d) * g_std).astype(np.float32))
@@ -108,7 +109,7 @@ def run_closed_loop(n, d, graph, comms_per_grad, accelerated, T, gamma, seed, sa
 
     chi1, chi2 = B.graph_chi(n, edges, rates)
     eta, alpha, alpha_t = B.prescribe(chi1, chi2, accelerated)
-    eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n, device=device)
+    eng = B.Engine(n, d, eta, alpha, alpha_t, gamma, n_grad_slots=n, device=device, momentum=bool(accelerated))
     eng.write_state(x0)
     a = torch.from_numpy(prob.a.astype(np.float32)).to(device)
     bt = torch.from_numpy(prob.b.astype(np.float32)).to(device)
