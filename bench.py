@@ -61,6 +61,7 @@ def parse_args():
     ap.add_argument("--no-fuse", action="store_true", help="one event per item (no gradient fusion)")
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chain", action="store_true", help="gradient fusion only (A2_SCHED_FUSE), no item chaining")
     ap.add_argument("--skip-resident-mode", action="store_true")
     ap.add_argument("--skip-baseline-dynamic", action="store_true")
     return ap.parse_args()
@@ -234,7 +235,7 @@ def main():
     ranks.barrier()
 
     W_, K, eps = args.warmup, args.steps, args.events_per_step
-    flags = 0 if args.no_fuse else B.A2_SCHED_FUSE
+    flags = 0 if args.no_fuse else (B.A2_SCHED_FUSE if args.no_chain else B.A2_SCHED_CHAIN)
     n_steps = W_ + K
     threads = max(1, min(os.cpu_count() or 1, 32) // max(1, ranks.world))
 
@@ -403,7 +404,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: {cfg.note}", "n": cfg.n, "d": cfg.d, "graph": cfg.graph,
                    "storage": cfg.storage, "events_per_step": eps, "consensus_every_events": eps,
-                   "gradient_fusion": not args.no_fuse, "parallelism": "replicas only" if ranks.world > 1 else "1 gpu",
+                   "gradient_fusion": not args.no_fuse, "item_chaining": not (args.no_fuse or args.no_chain), "parallelism": "replicas only" if ranks.world > 1 else "1 gpu",
                    "l2": "state 2*n*d*elem bytes per replica exceeds L2; no flush needed" if
                    2 * cfg.n * cfg.d * eng.elem_bytes > 3 * 126e6 else "state fits L2: figures are L2-assisted"},
         "clocks": clocks, "roofline": roofline,

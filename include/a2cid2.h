@@ -61,7 +61,7 @@ enum {
     A2_SCHED_FUSE = 1u, /* fold the gradient events that directly precede a communication of the
                            same worker into that communication's item, so their rows are read
                            and written once (the arithmetic per element is unchanged)          */
-    A2_SCHED_RESIDENT = 2u /* no batches: one launch walks the whole stream in time order while a
+    A2_SCHED_RESIDENT = 2u, /* no batches: one launch walks the whole stream in time order while a
                               column tile of all n workers' x and x~ stays in shared memory, so the
                               state crosses HBM once per call instead of once per batch. Columns
                               never interact, so no thread ever waits for another. Only valid when
@@ -70,11 +70,27 @@ enum {
                               memory (2 n + 16 <= 216 rows of 256 floats; A2_EINVAL otherwise).
                               With bf16 storage the tile is kept in fp32 and rounded once, at the
                               end of the call. The schedule then has a single batch holding every
-                              event in stream order. Overrides A2_SCHED_FUSE.                  */
+                              event in stream order. Overrides the other flags.                */
+    A2_SCHED_CHAIN = 4u /* A2_SCHED_FUSE, and further: (1) an event whose workers' latest events are
+                           all in one item is appended to that item, whose rows then serve one
+                           more event without crossing HBM again; (2) a communication between a
+                           worker that is free earlier and one whose latest events sit in an item
+                           of two workers joins that item as its third worker, so the shared
+                           worker's rows are not written and read again in between. Every
+                           worker's own order is kept and the arithmetic per event is unchanged;
+                           batches get fewer and items longer (up to three workers)            */
 };
 
 /* Kinds of elementary operation inside an item. */
-enum { A2_OP_GRAD_A = 0, A2_OP_GRAD_B = 1, A2_OP_COMM = 2, A2_OP_MIX_A = 3 /* mixing only (a2cid2_flush) */ };
+enum {
+    A2_OP_GRAD_A = 0, /* gradient event on the item's worker a                                   */
+    A2_OP_GRAD_B = 1,
+    A2_OP_COMM = 2,   /* communication between workers a and b                                   */
+    A2_OP_MIX_A = 3,  /* mixing only (a2cid2_flush)                                              */
+    A2_OP_GRAD_C = 4,
+    A2_OP_COMM_AC = 5,
+    A2_OP_COMM_BC = 6
+};
 
 /* Variants of the dynamic. */
 enum {
@@ -90,13 +106,14 @@ enum {
                               rows. A2_SCHED_RESIDENT is not available (A2_EINVAL).               */
 };
 
-/* One item of a batch: all the work done on one worker (b = -1) or one pair of workers. */
+/* One item of a batch: all the work done on one worker (b = c = -1), a pair, or three workers. */
 typedef struct a2cid2_item_info {
     int32_t a, b;           /* worker rows; b = -1 for a gradient-only item                    */
     int32_t slot_a, slot_b; /* gradient rows read for worker a / b, or -1                       */
     int64_t first_op;       /* index of the item's first elementary operation                   */
     int32_t n_ops;          /* operations applied, in order, while the rows sit in registers    */
     int32_t batch;          /* batch (dependency level) the item belongs to                     */
+    int32_t c, slot_c;      /* third worker and its gradient row (A2_SCHED_CHAIN), or -1         */
 } a2cid2_item_info;
 
 /* Counters of one a2cid2_apply_events / a2cid2_plan_run call (all device figures are what the
@@ -255,12 +272,15 @@ void a2cid2_plan_destroy(a2cid2_plan_t* p);
  * the state of the time-ordered run. With A2_SCHED_FUSE, gradient events of a worker are held
  * back and applied, in order, inside the next communication item of that worker (or in a
  * gradient-only item at the end of the stream, or when max_ops_per_item is reached or the
- * gradient slot changes). t_last[n] are the workers' times at the start (NULL = zeros).
- * max_ops_per_item <= 0 selects the default. Validation and error codes as in
+ * gradient slot changes). With A2_SCHED_CHAIN items also take later events of workers they already
+ * hold, and a third worker (see the flag). t_last[n] are the workers' times at the start
+ * (NULL = zeros). max_ops_per_item <= 0 selects the default; max_workers_per_item is 2 or 3
+ * (<= 0: 3) and only matters with A2_SCHED_CHAIN. Validation and error codes as in
  * a2cid2_apply_events. */
 int a2cid2_sched_create(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events,
                         const double* times, const int32_t* wi, const int32_t* wj, const int32_t* grad_slot,
-                        uint32_t flags, int32_t max_ops_per_item, a2cid2_sched_t** out);
+                        uint32_t flags, int32_t max_ops_per_item, int32_t max_workers_per_item,
+                        a2cid2_sched_t** out);
 
 int64_t a2cid2_sched_num_batches(const a2cid2_sched_t* s);
 int64_t a2cid2_sched_num_items(const a2cid2_sched_t* s);

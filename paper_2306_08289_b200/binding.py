@@ -20,7 +20,8 @@ A2_OK, A2_EINVAL, A2_EORDER, A2_ERANGE, A2_ENOMEM, A2_ECUDA, A2_ESTATE = 0, -1, 
 A2_F32, A2_BF16 = 0, 1
 A2_SCHED_FUSE = 1
 A2_SCHED_RESIDENT = 2
-A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A = 0, 1, 2, 3
+A2_SCHED_CHAIN = 4
+A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A, A2_OP_GRAD_C, A2_OP_COMM_AC, A2_OP_COMM_BC = 0, 1, 2, 3, 4, 5, 6
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX, A2_NO_MOMENTUM = 0, 1, 2
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
@@ -29,7 +30,11 @@ ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ER
 
 class ItemInfo(C.Structure):
     _fields_ = [("a", C.c_int32), ("b", C.c_int32), ("slot_a", C.c_int32), ("slot_b", C.c_int32),
-                ("first_op", C.c_int64), ("n_ops", C.c_int32), ("batch", C.c_int32)]
+                ("first_op", C.c_int64), ("n_ops", C.c_int32), ("batch", C.c_int32),
+                ("c", C.c_int32), ("slot_c", C.c_int32)]
+
+    def workers(self):
+        return [w for w in (self.a, self.b, self.c) if w >= 0]
 
 
 class Stats(C.Structure):
@@ -74,7 +79,8 @@ SIGNATURES = {
     "a2cid2_plan_sched": (_vp, [_vp]),
     "a2cid2_plan_run": (C.c_int, [_vp, _vp, C.c_int64, C.c_int64, C.POINTER(Stats)]),
     "a2cid2_plan_destroy": (None, [_vp]),
-    "a2cid2_sched_create": (C.c_int, [C.c_int32, C.c_int32, _dp, C.c_int64, _dp, _ip, _ip, _ip, C.c_uint32, C.c_int32, C.POINTER(_vp)]),
+    "a2cid2_sched_create": (C.c_int, [C.c_int32, C.c_int32, _dp, C.c_int64, _dp, _ip, _ip, _ip, C.c_uint32, C.c_int32, C.c_int32,
+                                      C.POINTER(_vp)]),
     "a2cid2_sched_num_batches": (C.c_int64, [_vp]),
     "a2cid2_sched_num_items": (C.c_int64, [_vp]),
     "a2cid2_sched_num_ops": (C.c_int64, [_vp]),
@@ -162,7 +168,8 @@ def consensus_distance_static(x_ptr, n, d, row_pitch_elems, storage_dtype, cuda_
 class Schedule:
     """a2cid2_sched_* : batches of worker-disjoint items for an event stream (host only)."""
 
-    def __init__(self, n, n_grad_slots, times, wi, wj, slot, flags=0, t_last=None, max_ops_per_item=0, _borrowed=None):
+    def __init__(self, n, n_grad_slots, times, wi, wj, slot, flags=0, t_last=None, max_ops_per_item=0,
+                 max_workers_per_item=0, _borrowed=None):
         self._owned = _borrowed is None
         if _borrowed is not None:
             self._h = _borrowed
@@ -172,7 +179,7 @@ class Schedule:
         h = _vp()
         _check(lib().a2cid2_sched_create(n, n_grad_slots, None if tl is None else _ptr(tl, _dp), len(times),
                                          _ptr(times, _dp), _ptr(wi, _ip), _ptr(wj, _ip), _ptr(slot, _ip),
-                                         flags, max_ops_per_item, C.byref(h)))
+                                         flags, max_ops_per_item, max_workers_per_item, C.byref(h)))
         self._h = h
         self.n = n
 

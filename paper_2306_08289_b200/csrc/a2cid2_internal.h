@@ -18,12 +18,15 @@ struct SchedOp {
     int64_t event;    // index into the caller's event arrays
     int32_t kind;     // A2_OP_*
     double t;         // event time
-    double t_prev_a;  // time worker a was last updated before this op (GRAD_A, COMM)
-    double t_prev_b;  // same for worker b (GRAD_B, COMM)
+    double t_prev_a;  // time the operation's first (or only) worker was last updated before it
+    double t_prev_b;  // same for the second worker of a communication
 };
 
+constexpr int kMaxItemWorkers = 3;
+
 struct SchedItem {
-    int32_t a, b, slot_a, slot_b;
+    int32_t a, b, c;  // workers; b, c = -1 when absent
+    int32_t slot_a, slot_b, slot_c;
     int64_t first_op;
     int32_t n_ops;
     int32_t batch;
@@ -65,7 +68,7 @@ void build_resident_chunks(const a2cid2_sched& s, int capacity, std::vector<ResC
 // Builds a schedule; returns A2_OK or an error code with the text in `err`.
 int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events, const double* times,
                    const int32_t* wi, const int32_t* wj, const int32_t* slot, uint32_t flags,
-                   int32_t max_ops_per_item, a2cid2_sched** out, std::string& err);
+                   int32_t max_ops_per_item, int32_t max_workers_per_item, a2cid2_sched** out, std::string& err);
 
 // momentum = false counts the rows of the dynamic without x~ (Eq. (baselinedynamic)).
 void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, int32_t elem_bytes, bool momentum,
@@ -73,7 +76,7 @@ void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, in
 
 // ---- device descriptors (layout shared by host packing and the event kernel) ---------------
 struct DevItem {
-    int32_t a, b, slot_a, slot_b;
+    int32_t a, b, c, slot_a, slot_b, slot_c;
     int32_t op_first;  // relative to the launch's first op
     int32_t op_count;
 };
@@ -82,8 +85,8 @@ struct DevOp {
     int32_t kind;
     int32_t pad;
     double t;         // event time
-    double t_prev_a;  // worker a's last-event time before this op
-    double t_prev_b;  // worker b's
+    double t_prev_a;  // last-event time, before this op, of its first (or only) worker
+    double t_prev_b;  // of the second worker of a communication
 };
 
 constexpr int kMaxItemsPerLaunch = 128;
@@ -104,11 +107,13 @@ struct EventLaunch {
     float alpha, alpha_tilde, gamma;
     int32_t variant;
     int32_t dtype;
+    bool three_workers;  // some item holds a third worker: the three-worker instance of the kernel is needed
 };
 
 struct DeviceInfo {
     int sm_count = 0;
     int event_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // [storage type][128-bit / 256-bit accesses]
+    int event3_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the three-worker instances
     int plain_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the kernel of the dynamic without x~
     int consensus_ctas_per_sm = 0;
 };

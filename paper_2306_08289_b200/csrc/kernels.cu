@@ -195,7 +195,8 @@ struct EventArgs {
     int msg_before_mix;
 };
 
-template <typename T, int BYTES, int UNROLL>
+// KW = 2 or 3: workers an item may hold (three-worker items come from A2_SCHED_CHAIN schedules).
+template <typename T, int BYTES, int UNROLL, int KW>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
@@ -208,8 +209,9 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
         const DevOp op = p.ops[o];
         s_kind[o] = (unsigned char)op.kind;
-        s_ca[o] = (op.kind != A2_OP_GRAD_B) ? (float)mix_coeff(p.eta, op.t - op.t_prev_a) : 0.f;
-        s_cb[o] = (op.kind == A2_OP_GRAD_B || op.kind == A2_OP_COMM) ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
+        const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC;
+        s_ca[o] = (float)mix_coeff(p.eta, op.t - op.t_prev_a);  // the operation's first (or only) worker
+        s_cb[o] = comm ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
     }
     __syncthreads();
 
@@ -249,16 +251,22 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
         const int item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
         const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
         const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
 
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxta = Xt + (long long)it.a * p.pitch;
         T* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
         T* const pxtb = Xt + (long long)(has_b ? it.b : it.a) * p.pitch;
+        T* const pxc = X + (long long)(has_c ? it.c : it.a) * p.pitch;
+        T* const pxtc = Xt + (long long)(has_c ? it.c : it.a) * p.pitch;
         const T* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
         const T* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+        const T* const pgc = G + (long long)(has_gc ? it.slot_c : 0) * p.pitch;
 
+        constexpr int UC = KW == 3 ? UNROLL : 1, NC = KW == 3 ? N : 1;  // no registers for a worker the instance never has
         float xa[UNROLL][N], xta[UNROLL][N], xb[UNROLL][N], xtb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N];
+        float xc[UC][NC], xtc[UC][NC], gc[UC][NC];
         bool live[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -268,6 +276,10 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
             if (kRecompute) {
 #pragma unroll
                 for (int k = 0; k < N; ++k) { xb[u][k] = 0.f; xtb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; xa[u][k] = 0.f; xta[u][k] = 0.f; }
+                if constexpr (KW == 3) {
+#pragma unroll
+                    for (int k = 0; k < NC; ++k) { xc[u][k] = 0.f; xtc[u][k] = 0.f; gc[u][k] = 0.f; }
+                }
             }
             if (live[u]) {  // rows an item does not have are never read by its operations, nor stored
                 V::load(pxa + off, xa[u]);
@@ -278,6 +290,13 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 }
                 if (has_ga) V::load(pga + off, ga[u]);
                 if (has_gb) V::load(pgb + off, gb[u]);
+                if constexpr (KW == 3) {
+                    if (has_c) {
+                        V::load(pxc + off, xc[u]);
+                        V::load(pxtc + off, xtc[u]);
+                    }
+                    if (has_gc) V::load(pgc + off, gc[u]);
+                }
             }
         }
 
@@ -290,11 +309,33 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
 #pragma unroll
                     for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], c, ngamma, ga[u][k]);
             } else if (kind == A2_OP_GRAD_B) {
-                const float c = s_cb[o];
+                const float c = s_ca[o];
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
                     for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
+            } else if (KW == 3 && kind == A2_OP_GRAD_C) {
+                const float c = s_ca[o];
+#pragma unroll
+                for (int u = 0; u < UC; ++u)
+#pragma unroll
+                    for (int k = 0; k < NC; ++k) grad_elem<sizeof(T) == 4>(xc[u][k], xtc[u][k], c, ngamma, gc[u][k]);
+            } else if (KW == 3 && kind == A2_OP_COMM_AC) {
+                const float ca = s_ca[o], cb = s_cb[o];
+#pragma unroll
+                for (int u = 0; u < UC; ++u)
+#pragma unroll
+                    for (int k = 0; k < NC; ++k)
+                        comm_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], xc[u][k], xtc[u][k], ca, cb, alpha, alpha_t,
+                                                  p.msg_before_mix != 0);
+            } else if (KW == 3 && kind == A2_OP_COMM_BC) {
+                const float ca = s_ca[o], cb = s_cb[o];
+#pragma unroll
+                for (int u = 0; u < UC; ++u)
+#pragma unroll
+                    for (int k = 0; k < NC; ++k)
+                        comm_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], xc[u][k], xtc[u][k], ca, cb, alpha, alpha_t,
+                                                  p.msg_before_mix != 0);
             } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
                 const float c = s_ca[o];
 #pragma unroll
@@ -321,6 +362,12 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 if (has_b) {
                     V::store(pxb + off, xb[u]);
                     V::store(pxtb + off, xtb[u]);
+                }
+                if constexpr (KW == 3) {
+                    if (has_c) {
+                        V::store(pxc + off, xc[u]);
+                        V::store(pxtc + off, xtc[u]);
+                    }
                 }
             }
         }
@@ -600,7 +647,7 @@ __global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __re
     }
 }
 
-template <typename T, int BYTES>
+template <typename T, int BYTES, int KW>
 int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr int U = EventCfg<T, BYTES>::UNROLL;
     constexpr int N = Vec<T, BYTES>::N;
@@ -613,11 +660,11 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    const int per_sm = dev.event_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
+    const int per_sm = (KW == 3 ? dev.event3_ctas_per_sm : dev.event_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
     long long grid = (long long)dev.sm_count * per_sm;
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events<T, BYTES, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    k_apply_events<T, BYTES, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -669,11 +716,11 @@ int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t 
 template <typename T> struct EventCtas { static constexpr int PER_SM = 2; };
 template <> struct EventCtas<__nv_bfloat16> { static constexpr int PER_SM = 4; };
 
-template <typename T, int BYTES>
+template <typename T, int BYTES, int KW>
 cudaError_t event_occupancy(int* out) {
     int occ = 0;
     const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL>, kEventThreads, 0);
+        &occ, k_apply_events<T, BYTES, EventCfg<T, BYTES>::UNROLL, KW>, kEventThreads, 0);
     *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
     return e;
 }
@@ -731,10 +778,14 @@ int query_device(DeviceInfo* info) {
     if (e != cudaSuccess) return (int)e;
     e = cudaDeviceGetAttribute(&info->sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return (int)e;
-    if ((e = event_occupancy<float, 16>(&info->event_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
-    if ((e = event_occupancy<float, 32>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
-    if ((e = event_occupancy<__nv_bfloat16, 16>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<float, 16, 2>(&info->event_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<float, 32, 2>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<__nv_bfloat16, 16, 2>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
     info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
+    if ((e = event_occupancy<float, 16, 3>(&info->event3_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<float, 32, 3>(&info->event3_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    if ((e = event_occupancy<__nv_bfloat16, 16, 3>(&info->event3_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
+    info->event3_ctas_per_sm[1][1] = info->event3_ctas_per_sm[1][0];
     if ((e = plain_occupancy<float, 16>(&info->plain_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
     if ((e = plain_occupancy<float, 32>(&info->plain_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     {
@@ -761,6 +812,12 @@ int query_device(DeviceInfo* info) {
             for (auto& row : info->event_ctas_per_sm)
                 for (int& c : row) c = k;
     }
+    if (const char* v = std::getenv("A2CID2_EVENT3_CTAS_PER_SM")) {  // the same for the three-worker instances
+        const int k = std::atoi(v);
+        if (k > 0)
+            for (auto& row : info->event3_ctas_per_sm)
+                for (int& c : row) c = k;
+    }
     return 0;
 }
 
@@ -778,8 +835,12 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
         return wide_x ? launch_plain_t<float, 32>(L, dev, stream) : launch_plain_t<float, 16>(L, dev, stream);
     }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
-    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16>(L, dev, stream);
-    return wide ? launch_events_t<float, 32>(L, dev, stream) : launch_events_t<float, 16>(L, dev, stream);
+    if (L.three_workers) {
+        if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16, 3>(L, dev, stream);
+        return wide ? launch_events_t<float, 32, 3>(L, dev, stream) : launch_events_t<float, 16, 3>(L, dev, stream);
+    }
+    if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16, 2>(L, dev, stream);
+    return wide ? launch_events_t<float, 32, 2>(L, dev, stream) : launch_events_t<float, 16, 2>(L, dev, stream);
 }
 
 int consensus_grid(const DeviceInfo& dev) { return dev.sm_count * dev.consensus_ctas_per_sm; }

@@ -93,7 +93,7 @@ class Checker:
                 e, _ = sched.ops(it.first_op, it.n_ops)
                 e = e[np.argsort(ev.times[e], kind="stable")]
                 self.stored.apply(ev.times[e], ev.wi[e], ev.wj[e], ev.slot[e])
-                self.stored.round_rows([it.a] + ([it.b] if it.b >= 0 else []))
+                self.stored.round_rows(it.workers())
 
     def compare(self, x, xt, t, where="", cols=None):
         """x, xt: widened device state (optionally only the columns `cols` of the checker). xt = None

@@ -118,11 +118,11 @@ int main(void) {
     double times[3] = {0.5, 1.0, 1.5};
     int32_t wi[3] = {0, 2, 1}, wj[3] = {1, 3, 2}, slot[3] = {-1, -1, -1};
     a2cid2_sched_t* s = 0;
-    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, A2_SCHED_FUSE, 0, &s) != A2_OK) return 3;
+    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, A2_SCHED_CHAIN, 0, 0, &s) != A2_OK) return 3;
     long long nb = (long long)a2cid2_sched_num_batches(s);
     a2cid2_sched_destroy(s);
     wi[0] = 7;  /* out of range: rejected with a message */
-    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, 0, 0, &s) != A2_ERANGE) return 4;
+    if (a2cid2_sched_create(4, 0, 0, 3, times, wi, wj, slot, 0, 0, 0, &s) != A2_ERANGE) return 4;
     printf("%.6f %.6f %.6f %.6f %lld %s|%s\n", c1, c2, eta, at, nb, a2cid2_last_error(0), a2cid2_version());
     return 0;
 }

@@ -10,7 +10,7 @@ from tests import parity as P
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 def test_cfg1_full_every_batch(flags):
     cfg = W.CONFIGS["cfg1"]
     eng, chk = P.make_small(cfg)
@@ -27,7 +27,7 @@ def test_cfg1_full_every_batch(flags):
     ("cfg4", 4_097, 4000),    # one column past two tiles
     ("cfg5", 16_389, 4000),   # bf16: two tiles + 5 columns
 ])
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 def test_scaled_configs_every_batch(name, d, n_events, flags):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     eng, chk = P.make_small(cfg)
@@ -41,30 +41,31 @@ def test_scaled_configs_every_batch(name, d, n_events, flags):
 def test_degenerate_sizes(n, d, storage):
     cfg = W.WorkloadConfig(name=f"tiny{n}x{d}", n=n, graph="ring", d=d, storage=storage, n_events=300,
                            x0_std=1.0, g_std=0.5, gamma=0.05, edge_rate=1.0, fixed_params=(0.7, 0.5, 1.5), seed=77)
-    for flags in (0, B.A2_SCHED_FUSE):
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN):
         eng, chk = P.make_small(cfg)
         P.run_batches_and_check(eng, chk, W.config_events(cfg), flags, every=7)
         eng.close()
 
 
-def test_fused_and_unfused_schedules_are_bit_identical():
-    """Fusion only changes which rows share a trip through registers, not the arithmetic."""
+def test_fused_chained_and_unfused_schedules_are_bit_identical():
+    """Fusion and chaining only change which rows share a trip through registers, not the arithmetic
+    (a communication stored with its two workers swapped gives the same bits: the update is antisymmetric)."""
     cfg = W.CONFIGS["cfg4"].scaled(d=10_003, n_events=3000)
     ev = W.config_events(cfg)
     out = []
-    for flags in (0, B.A2_SCHED_FUSE):
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN):
         eng, _ = P.make_small(cfg)
         eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
         out.append(eng.read_state())
         eng.close()
-    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
-    assert np.array_equal(out[0][2], out[1][2])
+    for o in out[1:]:
+        assert all(np.array_equal(u, v) for u, v in zip(out[0], o))
 
 
 def test_message_before_mix_variant():
     cfg = W.CONFIGS["cfg3"].scaled(d=5_001, n_events=1500)
     eng, chk = P.make_small(cfg, variant=B.A2_MSG_BEFORE_MIX)
-    P.run_batches_and_check(eng, chk, W.config_events(cfg), B.A2_SCHED_FUSE, every=5)
+    P.run_batches_and_check(eng, chk, W.config_events(cfg), B.A2_SCHED_CHAIN, every=5)
     eng.close()
 
 
@@ -127,7 +128,7 @@ def test_resident_mode_is_bit_identical_to_batches_fp32(name, d, n_events):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     ev = W.config_events(cfg)
     states = []
-    for flags in (B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
+    for flags in (B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_RESIDENT):
         eng, chk = P.make_small(cfg)
         for lo in range(0, len(ev), 777):  # several calls, so that resident calls chain on stored state
             c = ev.slice(lo, lo + 777)
@@ -187,7 +188,7 @@ def test_fifo_pairing_stream_with_ties():
     ev = W.fifo_pairing_events(cfg.n, cfg.edges(), cfg.comms_per_grad, cfg.n_events, seed=cfg.seed)
     assert np.any(np.diff(ev.times) == 0)
     outs = []
-    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_RESIDENT):
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_RESIDENT):
         eng, chk = P.make_small(cfg)
         if flags == B.A2_SCHED_RESIDENT:
             eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)

@@ -28,7 +28,7 @@ def _replay(cfg, ev, sched, params, x0, G):
 
 
 @pytest.mark.parametrize("name,d,n_events", [("cfg1", 7, 2000), ("cfg2", 5, 3000), ("cfg4", 3, 4000), ("cfg5", 3, 4000)])
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     cfg = cfg if cfg.storage == "f32" else W.WorkloadConfig(**{**cfg.__dict__, "storage": "f32"})
@@ -52,20 +52,22 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
         for k in range(first, first + cnt):
             it = s.item(k)
             assert it.batch == b and it.n_ops >= 1
-            ws = {it.a} | ({it.b} if it.b >= 0 else set())
-            assert not (ws & used)
+            ws = set(it.workers())
+            assert len(ws) == len(it.workers()) and not (ws & used)
+            assert (it.c < 0 or it.b >= 0) and (flags == B.A2_SCHED_CHAIN or it.c < 0)
             used |= ws
             evs, kinds = s.ops(it.first_op, it.n_ops)
+            pairs = {B.A2_OP_COMM: (it.a, it.b), B.A2_OP_COMM_AC: (it.a, it.c), B.A2_OP_COMM_BC: (it.b, it.c)}
+            grads = {B.A2_OP_GRAD_A: (it.a, it.slot_a), B.A2_OP_GRAD_B: (it.b, it.slot_b), B.A2_OP_GRAD_C: (it.c, it.slot_c)}
             for e, kd in zip(evs, kinds):
-                if kd == B.A2_OP_COMM:
-                    assert (ev.wi[e], ev.wj[e]) == (it.a, it.b)
-                    touched = (it.a, it.b)
-                elif kd == B.A2_OP_GRAD_A:
-                    assert ev.wi[e] == it.a and ev.wj[e] == -1 and ev.slot[e] == it.slot_a
-                    touched = (it.a,)
+                if kd in pairs:
+                    # the pair may be stored the other way round: the update is symmetric in its two workers
+                    assert {ev.wi[e], ev.wj[e]} == set(pairs[kd]) and min(pairs[kd]) >= 0
+                    touched = pairs[kd]
                 else:
-                    assert ev.wi[e] == it.b and ev.wj[e] == -1 and ev.slot[e] == it.slot_b
-                    touched = (it.b,)
+                    w, sl = grads[kd]
+                    assert ev.wi[e] == w and ev.wj[e] == -1 and ev.slot[e] == sl
+                    touched = (w,)
                 for w in touched:
                     assert last_pos.get(w, -1) < e  # this worker's events come in stream order
                     last_pos[w] = e
@@ -78,6 +80,12 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
     assert st["bytes_one_by_one"] == (8 * st["n_comm"] + 5 * st["n_grad"]) * cfg.d * 4
     if flags:
         assert st["bytes_moved"] < st["bytes_one_by_one"] and s.num_items < len(ev)
+        if flags == B.A2_SCHED_CHAIN:  # chaining moves fewer rows in fewer batches than gradient fusion alone
+            f = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+            assert st["bytes_moved"] < f.stats(cfg.d, 4)["bytes_moved"] and s.num_batches < f.num_batches
+            two = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags, max_workers_per_item=2)
+            assert all(two.item(k).c < 0 for k in range(two.num_items))
+            assert st["bytes_moved"] <= two.stats(cfg.d, 4)["bytes_moved"] <= f.stats(cfg.d, 4)["bytes_moved"]
     else:
         assert st["bytes_moved"] == st["bytes_one_by_one"] and s.num_items == len(ev)
 
@@ -109,6 +117,35 @@ def test_fusion_folds_pending_gradients_and_respects_caps():
     assert sorted(np.concatenate([s2.batch_events(b) for b in range(s2.num_batches)])) == [0, 1, 2, 3, 4]
     s3 = B.Schedule(2, 2, [1.0, 2.0, 3.0], [0, 0, 0], [-1, -1, 1], [0, 1, -1], flags=B.A2_SCHED_FUSE)
     assert s3.num_items == 2 and s3.item(0).slot_a == 0 and s3.item(1).slot_a == 1
+
+
+def test_chaining_appends_to_the_item_that_holds_the_rows_and_takes_a_third_worker():
+    # comm(0,1); gradient on 1; comm(0,1) again -> one item, nothing re-read; then comm(1,2) with 2 free earlier
+    # -> worker 2 joins as the third worker; then comm(2,3): 3 is free earlier, but the item is full -> new item
+    times = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0]
+    wi, wj, sl = [0, 1, 1, 2, 2, 3], [1, -1, 0, 1, 3, -1], [-1, 1, -1, -1, -1, 3]
+    s = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN)
+    assert s.num_items == 2 and s.num_batches == 2
+    it = s.item(0)
+    evs, kinds = s.ops(it.first_op, it.n_ops)
+    assert (it.a, it.b, it.c, it.slot_a, it.slot_b, it.slot_c) == (0, 1, 2, -1, 1, -1)
+    assert list(evs) == [0, 1, 2, 3]
+    assert list(kinds) == [B.A2_OP_COMM, B.A2_OP_GRAD_B, B.A2_OP_COMM, B.A2_OP_COMM_BC]
+    tail = s.item(1)
+    evs, kinds = s.ops(tail.first_op, tail.n_ops)
+    # the trailing gradient of worker 3 goes into the item that already holds its rows
+    assert (tail.a, tail.b, tail.c, tail.slot_b) == (2, 3, -1, 3) and list(evs) == [4, 5]
+    assert list(kinds) == [B.A2_OP_COMM, B.A2_OP_GRAD_B]
+    assert np.array_equal(s.t_final(4), [3.0, 4.0, 5.0, 6.0])
+    # two workers per item at most: the third comm opens a new item
+    s2 = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=2)
+    assert s2.num_items == 3 and all(s2.item(k).c < 0 for k in range(3))
+    # a gradient row of another slot cannot share the item's single row per worker
+    s3 = B.Schedule(2, 2, [1.0, 2.0, 3.0, 4.0], [0, 0, 0, 0], [1, -1, -1, 1], [-1, 0, 1, -1], flags=B.A2_SCHED_CHAIN)
+    rows = [(s3.item(k).slot_a, s3.item(k).n_ops) for k in range(s3.num_items)]
+    assert rows == [(0, 2), (1, 2)]
+    with pytest.raises(B.A2Error):
+        B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=4)
 
 
 def test_empty_stream_and_start_times():
@@ -167,7 +204,7 @@ def test_resident_schedule_is_one_batch_in_stream_order():
     sim.apply_stream(ev)
     assert np.array_equal(s.t_final(cfg.n), sim.t)
     with pytest.raises(B.A2Error):
-        B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=4)
+        B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=8)
 
 
 def test_fifo_stream_with_ties_replays_exactly():
@@ -178,7 +215,7 @@ def test_fifo_stream_with_ties_replays_exactly():
     x0, G = rng.standard_normal((n, d)), rng.standard_normal((n, d))
     ref = OracleSim(x0, 0.3, 0.5, 1.1, 0.05, grads=G)
     ref.apply_stream(ev)
-    for flags in (0, B.A2_SCHED_FUSE):
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN):
         s = B.Schedule(n, n, ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
         sim = OracleSim(x0, 0.3, 0.5, 1.1, 0.05, grads=G)
         for b in range(s.num_batches):
@@ -209,19 +246,21 @@ def test_random_streams_property():
                 wi.append(i); wj.append(j); sl.append(-1)
             else:
                 wi.append(i); wj.append(-1); sl.append(draw(st.integers(0, n_slots - 1)))
-        flags = draw(st.sampled_from([0, B.A2_SCHED_FUSE]))
+        flags = draw(st.sampled_from([0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_CHAIN]))
         cap = draw(st.sampled_from([0, 2, 3, 5]))
-        return n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32), flags, cap
+        kw = draw(st.sampled_from([0, 2, 3]))
+        return (n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32),
+                flags, cap, kw)
 
     @settings(max_examples=150, deadline=None)
     @given(streams())
     def check(case):
-        n, n_slots, times, wi, wj, sl, flags, cap = case
+        n, n_slots, times, wi, wj, sl, flags, cap, kw = case
         rng = np.random.default_rng(len(times) * 31 + n)
         x0, G = rng.standard_normal((n, 3)), rng.standard_normal((n_slots, 3))
         ref = OracleSim(x0, 0.4, 0.5, 1.7, 0.1, grads=G)
         ref.apply(times, wi, wj, sl)
-        s = B.Schedule(n, n_slots, times, wi, wj, sl, flags=flags, max_ops_per_item=cap)
+        s = B.Schedule(n, n_slots, times, wi, wj, sl, flags=flags, max_ops_per_item=cap, max_workers_per_item=kw)
         sim = OracleSim(x0, 0.4, 0.5, 1.7, 0.1, grads=G)
         seen = []
         for b in range(s.num_batches):
@@ -229,10 +268,14 @@ def test_random_streams_property():
             used = set()
             for k in range(first, first + cnt):
                 it = s.item(k)
-                ws = {it.a} | ({it.b} if it.b >= 0 else set())
+                ws = set(it.workers())
                 assert not (ws & used) and (cap == 0 or it.n_ops <= max(cap, 1))
+                assert len(ws) <= (kw or 3) and (flags == B.A2_SCHED_CHAIN or len(ws) <= 2)
                 used |= ws
-                evs, _ = s.ops(it.first_op, it.n_ops)
+                evs, kinds = s.ops(it.first_op, it.n_ops)
+                slots = {B.A2_OP_GRAD_A: it.slot_a, B.A2_OP_GRAD_B: it.slot_b, B.A2_OP_GRAD_C: it.slot_c}
+                for x, kd in zip(evs, kinds):  # one gradient row per worker and item
+                    assert kd not in slots or sl[x] == slots[kd]
                 e = evs[np.argsort(times[evs], kind="stable")]
                 # inside an item a worker's own events are already in stream order
                 for w in ws:
