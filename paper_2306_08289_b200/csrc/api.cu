@@ -360,6 +360,9 @@ int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_t
     if (!h) return fail(nullptr, A2_ENOMEM, "out of host memory");
     h->n = n; h->d = d; h->eta = eta; h->alpha = alpha; h->alpha_tilde = alpha_tilde; h->gamma = gamma;
     h->dtype = storage_dtype;
+    // bf16 rows: the three-worker instance needs 126 registers for its nine widened rows, which leaves too few
+    // bytes in flight (4.85 against 6.15 TB/s measured on 64 rows of 25.6e6 columns); two workers per item there
+    if (storage_dtype == A2_BF16) h->item_workers = 2;
     if (const char* v = std::getenv("A2CID2_ITEM_WORKERS")) {  // tuning override
         const int k = std::atoi(v);
         if (k >= 2 && k <= a2::kMaxItemWorkers) h->item_workers = k;

@@ -70,7 +70,7 @@ def test_full_size_sampled_columns_every_batch(name):
     xw, gw = _fill(eng, cfg, cols)
     chk = P.Checker(xw, P.oracle_params(cfg), cfg.gamma, gw, cfg.storage)
     ev = W.config_events(cfg)
-    plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)  # the schedule the benchmark times
     nb = plan.sched.num_batches
     worst = {}
     for b in range(nb):
