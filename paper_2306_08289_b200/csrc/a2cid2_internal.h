@@ -115,6 +115,7 @@ struct DeviceInfo {
     int event_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // [storage type][128-bit / 256-bit accesses]
     int event3_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the three-worker instances
     int plain_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the kernel of the dynamic without x~
+    int plain3_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};
     int consensus_ctas_per_sm = 0;
 };
 

@@ -250,8 +250,6 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     }
     for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
         const LaunchRange& R = pk.launches[(size_t)l];
-        if (R.three && h->variant == A2_NO_MOMENTUM)
-            return fail(h, A2_ESTATE, "this plan holds three-worker items, which the A2_NO_MOMENTUM kernels do not take");
         a2::EventLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.items = d_items + R.item0;
@@ -360,9 +358,6 @@ int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_t
     if (!h) return fail(nullptr, A2_ENOMEM, "out of host memory");
     h->n = n; h->d = d; h->eta = eta; h->alpha = alpha; h->alpha_tilde = alpha_tilde; h->gamma = gamma;
     h->dtype = storage_dtype;
-    // bf16 rows: the three-worker instance needs 126 registers for its nine widened rows, which leaves too few
-    // bytes in flight (4.85 against 6.15 TB/s measured on 64 rows of 25.6e6 columns); two workers per item there
-    if (storage_dtype == A2_BF16) h->item_workers = 2;
     if (const char* v = std::getenv("A2CID2_ITEM_WORKERS")) {  // tuning override
         const int k = std::atoi(v);
         if (k >= 2 && k <= a2::kMaxItemWorkers) h->item_workers = k;
@@ -523,8 +518,8 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
     const double t0 = now_ms();
     a2cid2_sched* s = nullptr;
     std::string err;
-    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0,
-                            h->variant == A2_NO_MOMENTUM ? 2 : h->item_workers, &s, err);
+    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, h->item_workers,
+                            &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     return submit_schedule(h, s, stats, t0);
 }
@@ -643,7 +638,7 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
     a2cid2_sched* s = nullptr;
     std::string err;
     rc = a2::build_schedule(h->n, h->n_slots, t_start ? t_start : h->t.data(), n_events, times, wi, wj, grad_slot, flags,
-                            0, h->variant == A2_NO_MOMENTUM ? 2 : h->item_workers, &s, err);
+                            0, h->item_workers, &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     a2cid2_plan* p = new (std::nothrow) a2cid2_plan();
     if (!p) { a2cid2_sched_destroy(s); return fail(h, A2_ENOMEM, "out of host memory"); }

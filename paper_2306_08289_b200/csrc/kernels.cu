@@ -381,14 +381,14 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
 // flow between events, so times play no part on the device and a mixing-only operation does nothing.
 // ---------------------------------------------------------------------------------------------
 #ifndef A2_PLAIN_UNROLL
-#define A2_PLAIN_UNROLL 2  // 256-bit vectors per thread and tile
+#define A2_PLAIN_UNROLL 1  // 256-bit vectors per thread and tile
 #endif
 #ifndef A2_PLAIN_UNROLL_128
-#define A2_PLAIN_UNROLL_128 4  // the same bytes per thread with 128-bit vectors
+#define A2_PLAIN_UNROLL_128 2  // the same bytes per thread with 128-bit vectors
 #endif
 template <int BYTES> struct PlainCfg { static constexpr int UNROLL = BYTES == 32 ? A2_PLAIN_UNROLL : A2_PLAIN_UNROLL_128; };
 
-template <typename T, int BYTES, int UNROLL>
+template <typename T, int BYTES, int UNROLL, int KW>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
@@ -409,13 +409,17 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
         const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
         const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
         const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
+        T* const pxc = X + (long long)(has_c ? it.c : it.a) * p.pitch;
         const T* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
         const T* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+        const T* const pgc = G + (long long)(has_gc ? it.slot_c : 0) * p.pitch;
 
-        float xa[UNROLL][N], xb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N];
+        constexpr int UC = KW == 3 ? UNROLL : 1, NC = KW == 3 ? N : 1;
+        float xa[UNROLL][N], xb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N], xc[UC][NC], gc[UC][NC];
         bool live[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -424,11 +428,19 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
             const long long off = v * N;
 #pragma unroll
             for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
+            if constexpr (KW == 3) {
+#pragma unroll
+                for (int k = 0; k < NC; ++k) { xc[u][k] = 0.f; gc[u][k] = 0.f; }
+            }
             if (live[u]) {
                 V::load(pxa + off, xa[u]);
                 if (has_b) V::load(pxb + off, xb[u]);
                 if (has_ga) V::load(pga + off, ga[u]);
                 if (has_gb) V::load(pgb + off, gb[u]);
+                if constexpr (KW == 3) {
+                    if (has_c) V::load(pxc + off, xc[u]);
+                    if (has_gc) V::load(pgc + off, gc[u]);
+                }
             }
         }
         bool dirty = false;
@@ -436,6 +448,25 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
             const int kind = s_kind[o];
             if (kind == A2_OP_MIX_A) continue;
             dirty = true;
+            if (KW == 3 && (kind == A2_OP_GRAD_C || kind == A2_OP_COMM_AC || kind == A2_OP_COMM_BC)) {
+#pragma unroll
+                for (int u = 0; u < UC; ++u)
+#pragma unroll
+                    for (int k = 0; k < NC; ++k) {
+                        if (kind == A2_OP_GRAD_C) {
+                            xc[u][k] = __fmaf_rn(ngamma, gc[u][k], xc[u][k]);
+                        } else if (kind == A2_OP_COMM_AC) {
+                            const float m = __fsub_rn(xa[u][k], xc[u][k]);
+                            xa[u][k] = __fmaf_rn(-alpha, m, xa[u][k]);
+                            xc[u][k] = __fmaf_rn(alpha, m, xc[u][k]);
+                        } else {
+                            const float m = __fsub_rn(xb[u][k], xc[u][k]);
+                            xb[u][k] = __fmaf_rn(-alpha, m, xb[u][k]);
+                            xc[u][k] = __fmaf_rn(alpha, m, xc[u][k]);
+                        }
+                    }
+                continue;
+            }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
@@ -457,6 +488,9 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
             if (live[u] && dirty) {
                 V::store(pxa + off, xa[u]);
                 if (has_b) V::store(pxb + off, xb[u]);
+                if constexpr (KW == 3) {
+                    if (has_c) V::store(pxc + off, xc[u]);
+                }
             }
         }
     }
@@ -469,6 +503,9 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
 #ifndef A2_PLAIN_BF16_UNROLL
 #define A2_PLAIN_BF16_UNROLL 1  // 256-bit vectors per thread and tile (the 128-bit kernel takes twice as many)
 #endif
+#ifndef A2_PLAIN_BF16_GROUP
+#define A2_PLAIN_BF16_GROUP 2
+#endif
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
@@ -477,7 +514,7 @@ __device__ __forceinline__ uint32_t bf16_pack(float lo, float hi) {  // round to
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int WORDS, int UNROLL>
+template <int WORDS, int UNROLL, int KW>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const EventArgs p) {
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
@@ -496,11 +533,16 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
         const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
         const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
+        const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
         const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
         __nv_bfloat16* const pxa = X + (long long)it.a * p.pitch;
         __nv_bfloat16* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
         const __nv_bfloat16* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
         const __nv_bfloat16* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
+        __nv_bfloat16* const pxc = X + (long long)(has_c ? it.c : it.a) * p.pitch;
+        const __nv_bfloat16* const pgc = G + (long long)(has_gc ? it.slot_c : 0) * p.pitch;
+        constexpr int UC = KW == 3 ? UNROLL : 1, WC = KW == 3 ? WORDS : 1;
+        uint32_t xc[UC][WC], gc[UC][WC];
 
         uint32_t xa[UNROLL][WORDS], xb[UNROLL][WORDS], ga[UNROLL][WORDS], gb[UNROLL][WORDS];
         bool live[UNROLL];
@@ -511,6 +553,14 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
             const long long off = v * (2 * WORDS);
 #pragma unroll
             for (int k = 0; k < WORDS; ++k) { xa[u][k] = 0u; xb[u][k] = 0u; ga[u][k] = 0u; gb[u][k] = 0u; }
+            if constexpr (KW == 3) {
+#pragma unroll
+                for (int k = 0; k < WC; ++k) { xc[u][k] = 0u; gc[u][k] = 0u; }
+                if (live[u]) {
+                    if (has_c) Words<WORDS>::ld(pxc + off, xc[u]);
+                    if (has_gc) Words<WORDS>::ld(pgc + off, gc[u]);
+                }
+            }
             if (live[u]) {
                 Words<WORDS>::ld(pxa + off, xa[u]);
                 if (has_b) Words<WORDS>::ld(pxb + off, xb[u]);
@@ -521,32 +571,64 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
         const int o_begin = it.op_first, o_end = it.op_first + it.op_count;
         bool dirty = false;
         for (int o = o_begin; o < o_end; ++o) dirty |= s_kind[o] != A2_OP_MIX_A;
+        constexpr int WG = A2_PLAIN_BF16_GROUP < WORDS ? A2_PLAIN_BF16_GROUP : WORDS;  // words widened and updated together
+        constexpr int E = 2 * WG, EC = KW == 3 ? E : 1;
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
 #pragma unroll
-            for (int k = 0; k < WORDS; ++k) {
-                float a0 = bf16_lo(xa[u][k]), a1 = bf16_hi(xa[u][k]);
-                float b0 = bf16_lo(xb[u][k]), b1 = bf16_hi(xb[u][k]);
-                const float ga0 = bf16_lo(ga[u][k]), ga1 = bf16_hi(ga[u][k]);
-                const float gb0 = bf16_lo(gb[u][k]), gb1 = bf16_hi(gb[u][k]);
+            for (int k0 = 0; k0 < WORDS; k0 += WG) {
+                float a[E], b[E], fa[E], fb[E], c[EC], fc[EC];
+#pragma unroll
+                for (int w = 0; w < WG; ++w) {
+                    a[2 * w] = bf16_lo(xa[u][k0 + w]); a[2 * w + 1] = bf16_hi(xa[u][k0 + w]);
+                    b[2 * w] = bf16_lo(xb[u][k0 + w]); b[2 * w + 1] = bf16_hi(xb[u][k0 + w]);
+                    fa[2 * w] = bf16_lo(ga[u][k0 + w]); fa[2 * w + 1] = bf16_hi(ga[u][k0 + w]);
+                    fb[2 * w] = bf16_lo(gb[u][k0 + w]); fb[2 * w + 1] = bf16_hi(gb[u][k0 + w]);
+                    if constexpr (KW == 3) {
+                        c[2 * w] = bf16_lo(xc[u][k0 + w]); c[2 * w + 1] = bf16_hi(xc[u][k0 + w]);
+                        fc[2 * w] = bf16_lo(gc[u][k0 + w]); fc[2 * w + 1] = bf16_hi(gc[u][k0 + w]);
+                    }
+                }
                 for (int o = o_begin; o < o_end; ++o) {
                     const int kind = s_kind[o];
                     if (kind == A2_OP_GRAD_A) {
-                        a0 = __fmaf_rn(ngamma, ga0, a0);
-                        a1 = __fmaf_rn(ngamma, ga1, a1);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) a[e] = __fmaf_rn(ngamma, fa[e], a[e]);
                     } else if (kind == A2_OP_GRAD_B) {
-                        b0 = __fmaf_rn(ngamma, gb0, b0);
-                        b1 = __fmaf_rn(ngamma, gb1, b1);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) b[e] = __fmaf_rn(ngamma, fb[e], b[e]);
                     } else if (kind == A2_OP_COMM) {
-                        const float m0 = __fsub_rn(a0, b0), m1 = __fsub_rn(a1, b1);
-                        a0 = __fmaf_rn(-alpha, m0, a0);
-                        a1 = __fmaf_rn(-alpha, m1, a1);
-                        b0 = __fmaf_rn(alpha, m0, b0);
-                        b1 = __fmaf_rn(alpha, m1, b1);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            const float m = __fsub_rn(a[e], b[e]);
+                            a[e] = __fmaf_rn(-alpha, m, a[e]);
+                            b[e] = __fmaf_rn(alpha, m, b[e]);
+                        }
+                    } else if (KW == 3 && kind == A2_OP_GRAD_C) {
+#pragma unroll
+                        for (int e = 0; e < EC; ++e) c[e] = __fmaf_rn(ngamma, fc[e], c[e]);
+                    } else if (KW == 3 && kind == A2_OP_COMM_AC) {
+#pragma unroll
+                        for (int e = 0; e < EC; ++e) {
+                            const float m = __fsub_rn(a[e], c[e]);
+                            a[e] = __fmaf_rn(-alpha, m, a[e]);
+                            c[e] = __fmaf_rn(alpha, m, c[e]);
+                        }
+                    } else if (KW == 3 && kind == A2_OP_COMM_BC) {
+#pragma unroll
+                        for (int e = 0; e < EC; ++e) {
+                            const float m = __fsub_rn(b[e], c[e]);
+                            b[e] = __fmaf_rn(-alpha, m, b[e]);
+                            c[e] = __fmaf_rn(alpha, m, c[e]);
+                        }
                     }
                 }
-                xa[u][k] = bf16_pack(a0, a1);
-                xb[u][k] = bf16_pack(b0, b1);
+#pragma unroll
+                for (int w = 0; w < WG; ++w) {
+                    xa[u][k0 + w] = bf16_pack(a[2 * w], a[2 * w + 1]);
+                    xb[u][k0 + w] = bf16_pack(b[2 * w], b[2 * w + 1]);
+                    if constexpr (KW == 3) xc[u][k0 + w] = bf16_pack(c[2 * w], c[2 * w + 1]);
+                }
             }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -554,7 +636,139 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
             if (live[u] && dirty) {
                 Words<WORDS>::st(pxa + off, xa[u]);
                 if (has_b) Words<WORDS>::st(pxb + off, xb[u]);
+                if constexpr (KW == 3) {
+                    if (has_c) Words<WORDS>::st(pxc + off, xc[u]);
+                }
             }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Three-worker items on bf16 rows. Nine rows widened to fp32 take 126 registers and leave too few bytes in
+// flight, so this instance keeps the rows packed (two columns per 32-bit register) while the loads are
+// in flight and takes one pair of columns at a time through the item's operations: widen, apply every
+// operation in order, round, pack. Per element the arithmetic is that of k_apply_events on bf16 rows.
+// ---------------------------------------------------------------------------------------------
+#ifndef A2_BF16_PACKED_GROUP
+#define A2_BF16_PACKED_GROUP 2  // 32-bit words (pairs of columns) widened and updated together
+#endif
+template <int WORDS, int WG>
+__global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_packed(const EventArgs p) {
+    __shared__ DevItem s_items[kMaxItemsPerLaunch];
+    __shared__ float s_ca[kMaxOpsPerLaunch];
+    __shared__ float s_cb[kMaxOpsPerLaunch];
+    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
+        const DevOp op = p.ops[o];
+        s_kind[o] = (unsigned char)op.kind;
+        const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC;
+        s_ca[o] = (float)mix_coeff(p.eta, op.t - op.t_prev_a);
+        s_cb[o] = comm ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
+    }
+    __syncthreads();
+
+    __nv_bfloat16* const X = static_cast<__nv_bfloat16*>(p.x);
+    __nv_bfloat16* const Xt = static_cast<__nv_bfloat16*>(p.xt);
+    const __nv_bfloat16* const G = static_cast<const __nv_bfloat16*>(p.g);
+    const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
+    const bool before = p.msg_before_mix != 0;
+    const long long n_units = (long long)p.n_items * p.n_tiles;
+    const int n_it = p.n_items;
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int rem = (int)(unit % n_it);
+        const long long tile = unit / n_it;
+        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+        const bool has_b = it.b >= 0, has_c = it.c >= 0;
+        const bool has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0, has_gc = it.slot_c >= 0;
+        const long long v = tile * (long long)kEventThreads + threadIdx.x;
+        if (v >= p.n_vec) continue;
+        const long long off = v * (2 * WORDS);
+        const long long ra = (long long)it.a * p.pitch + off;
+        const long long rb = (long long)(has_b ? it.b : it.a) * p.pitch + off;
+        const long long rc = (long long)(has_c ? it.c : it.a) * p.pitch + off;
+
+        uint32_t xa[WORDS], xta[WORDS], xb[WORDS], xtb[WORDS], xc[WORDS], xtc[WORDS], ga[WORDS], gb[WORDS], gc[WORDS];
+#pragma unroll
+        for (int k = 0; k < WORDS; ++k) { xb[k] = 0u; xtb[k] = 0u; xc[k] = 0u; xtc[k] = 0u; ga[k] = 0u; gb[k] = 0u; gc[k] = 0u; }
+        Words<WORDS>::ld(X + ra, xa);
+        Words<WORDS>::ld(Xt + ra, xta);
+        if (has_b) {
+            Words<WORDS>::ld(X + rb, xb);
+            Words<WORDS>::ld(Xt + rb, xtb);
+        }
+        if (has_c) {
+            Words<WORDS>::ld(X + rc, xc);
+            Words<WORDS>::ld(Xt + rc, xtc);
+        }
+        if (has_ga) Words<WORDS>::ld(G + (long long)it.slot_a * p.pitch + off, ga);
+        if (has_gb) Words<WORDS>::ld(G + (long long)it.slot_b * p.pitch + off, gb);
+        if (has_gc) Words<WORDS>::ld(G + (long long)it.slot_c * p.pitch + off, gc);
+
+        const int o_begin = it.op_first, o_end = it.op_first + it.op_count;
+        constexpr int E = 2 * WG;  // columns taken through the operations together
+#pragma unroll
+        for (int k0 = 0; k0 < WORDS; k0 += WG) {
+            float a[E], ta[E], b[E], tb[E], c[E], tc[E], fa[E], fb[E], fc[E];
+#pragma unroll
+            for (int w = 0; w < WG; ++w) {
+                a[2 * w] = bf16_lo(xa[k0 + w]); a[2 * w + 1] = bf16_hi(xa[k0 + w]);
+                ta[2 * w] = bf16_lo(xta[k0 + w]); ta[2 * w + 1] = bf16_hi(xta[k0 + w]);
+                b[2 * w] = bf16_lo(xb[k0 + w]); b[2 * w + 1] = bf16_hi(xb[k0 + w]);
+                tb[2 * w] = bf16_lo(xtb[k0 + w]); tb[2 * w + 1] = bf16_hi(xtb[k0 + w]);
+                c[2 * w] = bf16_lo(xc[k0 + w]); c[2 * w + 1] = bf16_hi(xc[k0 + w]);
+                tc[2 * w] = bf16_lo(xtc[k0 + w]); tc[2 * w + 1] = bf16_hi(xtc[k0 + w]);
+                fa[2 * w] = bf16_lo(ga[k0 + w]); fa[2 * w + 1] = bf16_hi(ga[k0 + w]);
+                fb[2 * w] = bf16_lo(gb[k0 + w]); fb[2 * w + 1] = bf16_hi(gb[k0 + w]);
+                fc[2 * w] = bf16_lo(gc[k0 + w]); fc[2 * w + 1] = bf16_hi(gc[k0 + w]);
+            }
+            for (int o = o_begin; o < o_end; ++o) {
+                const int kind = s_kind[o];
+                const float ca = s_ca[o];
+                if (kind == A2_OP_GRAD_A) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) grad_elem<false>(a[e], ta[e], ca, ngamma, fa[e]);
+                } else if (kind == A2_OP_GRAD_B) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) grad_elem<false>(b[e], tb[e], ca, ngamma, fb[e]);
+                } else if (kind == A2_OP_GRAD_C) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) grad_elem<false>(c[e], tc[e], ca, ngamma, fc[e]);
+                } else if (kind == A2_OP_MIX_A) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) grad_elem<false>(a[e], ta[e], ca, ngamma, 0.f);
+                } else {
+                    const float cb = s_cb[o];
+                    if (kind == A2_OP_COMM) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) comm_elem<false>(a[e], ta[e], b[e], tb[e], ca, cb, alpha, alpha_t, before);
+                    } else if (kind == A2_OP_COMM_AC) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) comm_elem<false>(a[e], ta[e], c[e], tc[e], ca, cb, alpha, alpha_t, before);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) comm_elem<false>(b[e], tb[e], c[e], tc[e], ca, cb, alpha, alpha_t, before);
+                    }
+                }
+            }
+#pragma unroll
+            for (int w = 0; w < WG; ++w) {
+                xa[k0 + w] = bf16_pack(a[2 * w], a[2 * w + 1]); xta[k0 + w] = bf16_pack(ta[2 * w], ta[2 * w + 1]);
+                xb[k0 + w] = bf16_pack(b[2 * w], b[2 * w + 1]); xtb[k0 + w] = bf16_pack(tb[2 * w], tb[2 * w + 1]);
+                xc[k0 + w] = bf16_pack(c[2 * w], c[2 * w + 1]); xtc[k0 + w] = bf16_pack(tc[2 * w], tc[2 * w + 1]);
+            }
+        }
+        Words<WORDS>::st(X + ra, xa);
+        Words<WORDS>::st(Xt + ra, xta);
+        if (has_b) {
+            Words<WORDS>::st(X + rb, xb);
+            Words<WORDS>::st(Xt + rb, xtb);
+        }
+        if (has_c) {
+            Words<WORDS>::st(X + rc, xc);
+            Words<WORDS>::st(Xt + rc, xtc);
         }
     }
 }
@@ -668,7 +882,7 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     return (int)cudaGetLastError();
 }
 
-template <typename T, int BYTES>
+template <typename T, int BYTES, int KW>
 int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr int U = PlainCfg<BYTES>::UNROLL;
     constexpr int N = Vec<T, BYTES>::N;
@@ -681,15 +895,15 @@ int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t str
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    const int per_sm = dev.plain_ctas_per_sm[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
+    const int per_sm = (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
     long long grid = (long long)dev.sm_count * per_sm;
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events_plain<T, BYTES, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    k_apply_events_plain<T, BYTES, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
-template <int WORDS>
+template <int WORDS, int KW>
 int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr int U = A2_PLAIN_BF16_UNROLL * (8 / WORDS);
     EventArgs a;
@@ -701,10 +915,10 @@ int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t 
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    long long grid = (long long)dev.sm_count * dev.plain_ctas_per_sm[1][WORDS == 8 ? 1 : 0];
+    long long grid = (long long)dev.sm_count * (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[1][WORDS == 8 ? 1 : 0];
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events_plain_bf16<WORDS, U><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    k_apply_events_plain_bf16<WORDS, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -725,12 +939,14 @@ cudaError_t event_occupancy(int* out) {
     return e;
 }
 
-template <typename T, int BYTES>
+template <typename T, int BYTES, int KW>
 cudaError_t plain_occupancy(int* out) {
     int occ = 0;
     const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &occ, k_apply_events_plain<T, BYTES, PlainCfg<BYTES>::UNROLL>, kEventThreads, 0);
-    *out = occ > EventCtas<T>::PER_SM ? EventCtas<T>::PER_SM : (occ > 0 ? occ : 1);
+        &occ, k_apply_events_plain<T, BYTES, PlainCfg<BYTES>::UNROLL, KW>, kEventThreads, 0);
+    // fp32 rows of 25.6e6 columns, one 256-bit vector per thread: two-worker items 2 CTAs/SM 5.65 TB/s, 3: 6.59,
+    // 4: 6.18; three-worker items 2: 4.76, 3: 5.98, 4: 4.68 (two vectors per thread and 2 CTAs: 6.59 and 5.70)
+    *out = occ > 3 ? 3 : (occ > 0 ? occ : 1);
     return e;
 }
 
@@ -784,25 +1000,51 @@ int query_device(DeviceInfo* info) {
     info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
     if ((e = event_occupancy<float, 16, 3>(&info->event3_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<float, 32, 3>(&info->event3_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
-    if ((e = event_occupancy<__nv_bfloat16, 16, 3>(&info->event3_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
-    info->event3_ctas_per_sm[1][1] = info->event3_ctas_per_sm[1][0];
-    if ((e = plain_occupancy<float, 16>(&info->plain_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
-    if ((e = plain_occupancy<float, 32>(&info->plain_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     {
         int occ = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<4, 2 * A2_PLAIN_BF16_UNROLL>,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_bf16_packed<4, A2_BF16_PACKED_GROUP>, kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        // measured on 64 bf16 rows of 25.6e6 columns, chained schedule: 128-bit accesses 2 CTAs/SM 5.02 TB/s, 3: 5.88,
+        // 4: 4.99; 256-bit accesses 2: 6.05, 3: 5.47
+        info->event3_ctas_per_sm[1][0] = occ > 3 ? 3 : (occ > 0 ? occ : 1);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_bf16_packed<8, A2_BF16_PACKED_GROUP>, kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->event3_ctas_per_sm[1][1] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
+    }
+    if ((e = plain_occupancy<float, 16, 2>(&info->plain_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = plain_occupancy<float, 32, 2>(&info->plain_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    if ((e = plain_occupancy<float, 16, 3>(&info->plain3_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
+    if ((e = plain_occupancy<float, 32, 3>(&info->plain3_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
+    {
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<4, 2 * A2_PLAIN_BF16_UNROLL, 2>,
                                                           kEventThreads, 0);
         if (e != cudaSuccess) return (int)e;
         info->plain_ctas_per_sm[1][0] = occ > 4 ? 4 : (occ > 0 ? occ : 1);
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<8, A2_PLAIN_BF16_UNROLL>,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<8, A2_PLAIN_BF16_UNROLL, 2>,
                                                           kEventThreads, 0);
         if (e != cudaSuccess) return (int)e;
         info->plain_ctas_per_sm[1][1] = occ > 4 ? 4 : (occ > 0 ? occ : 1);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<4, 2 * A2_PLAIN_BF16_UNROLL, 3>,
+                                                          kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->plain3_ctas_per_sm[1][0] = occ > 3 ? 3 : (occ > 0 ? occ : 1);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_plain_bf16<8, A2_PLAIN_BF16_UNROLL, 3>,
+                                                          kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        // bf16 rows of 25.6e6 columns, 256-bit accesses, chained schedule: 2 CTAs/SM 5.37 TB/s, 3: 6.36, 4: 5.12
+        info->plain3_ctas_per_sm[1][1] = occ > 3 ? 3 : (occ > 0 ? occ : 1);
     }
     if (const char* v = std::getenv("A2CID2_PLAIN_CTAS_PER_SM")) {  // tuning override, as for the event kernel
         const int k = std::atoi(v);
         if (k > 0)
             for (auto& row : info->plain_ctas_per_sm)
+                for (int& c : row) c = k;
+    }
+    if (const char* v = std::getenv("A2CID2_PLAIN3_CTAS_PER_SM")) {  // the same for the three-worker instances
+        const int k = std::atoi(v);
+        if (k > 0)
+            for (auto& row : info->plain3_ctas_per_sm)
                 for (int& c : row) c = k;
     }
     info->consensus_ctas_per_sm = 8;  // capacity of the partial-sum scratch, CTAs per SM
@@ -821,6 +1063,23 @@ int query_device(DeviceInfo* info) {
     return 0;
 }
 
+template <int WORDS>
+int launch_bf16_packed(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
+    EventArgs a;
+    a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
+    a.n_vec = (L.d + 2 * WORDS - 1) / (2 * WORDS);
+    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
+    a.n_tiles = (int)((a.n_vec + kEventThreads - 1) / kEventThreads);
+    a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
+    a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
+    const long long n_units = (long long)a.n_items * a.n_tiles;
+    long long grid = (long long)dev.sm_count * dev.event3_ctas_per_sm[1][WORDS == 8 ? 1 : 0];
+    if (grid > n_units) grid = n_units;
+    if (grid < 1) return 0;
+    k_apply_events_bf16_packed<WORDS, A2_BF16_PACKED_GROUP><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    return (int)cudaGetLastError();
+}
+
 int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.n_items <= 0) return 0;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -830,13 +1089,23 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
             static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
             const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.g);
             const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;
-            return wide_bf16 ? launch_plain_bf16<8>(L, dev, stream) : launch_plain_bf16<4>(L, dev, stream);
+            if (L.three_workers)
+                return wide_bf16 ? launch_plain_bf16<8, 3>(L, dev, stream) : launch_plain_bf16<4, 3>(L, dev, stream);
+            return wide_bf16 ? launch_plain_bf16<8, 2>(L, dev, stream) : launch_plain_bf16<4, 2>(L, dev, stream);
         }
-        return wide_x ? launch_plain_t<float, 32>(L, dev, stream) : launch_plain_t<float, 16>(L, dev, stream);
+        if (L.three_workers)
+            return wide_x ? launch_plain_t<float, 32, 3>(L, dev, stream) : launch_plain_t<float, 16, 3>(L, dev, stream);
+        return wide_x ? launch_plain_t<float, 32, 2>(L, dev, stream) : launch_plain_t<float, 16, 2>(L, dev, stream);
     }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
     if (L.three_workers) {
-        if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16, 3>(L, dev, stream);
+        if (L.dtype == A2_BF16) {
+            static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+            const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.xt) |
+                                   reinterpret_cast<uintptr_t>(L.g);
+            const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;
+            return wide_bf16 ? launch_bf16_packed<8>(L, dev, stream) : launch_bf16_packed<4>(L, dev, stream);
+        }
         return wide ? launch_events_t<float, 32, 3>(L, dev, stream) : launch_events_t<float, 16, 3>(L, dev, stream);
     }
     if (L.dtype == A2_BF16) return launch_events_t<__nv_bfloat16, 16, 2>(L, dev, stream);

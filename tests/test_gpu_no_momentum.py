@@ -10,7 +10,7 @@ from tests import parity as P
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 def test_cfg1_full_every_batch(flags):
     cfg = W.CONFIGS["cfg1"]
     eng, chk = P.make_small(cfg, momentum=False)
@@ -27,7 +27,7 @@ def test_cfg1_full_every_batch(flags):
     ("cfg4", 4_097, 4000),    # one column past a tile of the two-vector kernel
     ("cfg5", 16_389, 4000),   # bf16
 ])
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 def test_scaled_configs_every_batch(name, d, n_events, flags):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     eng, chk = P.make_small(cfg, momentum=False)
@@ -44,7 +44,7 @@ def test_degenerate_sizes(n, d, storage):
     cfg = W.WorkloadConfig(name=f"tiny{n}x{d}", n=n, graph="ring", d=d, storage=storage,
                            n_events=300 if storage == "f32" else 120,
                            x0_std=1.0, g_std=0.5, gamma=0.05, edge_rate=1.0, fixed_params=(0.7, 0.5, 1.5), seed=78)
-    for flags in (0, B.A2_SCHED_FUSE):
+    for flags in (0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN):
         eng, chk = P.make_small(cfg, momentum=False)
         P.run_batches_and_check(eng, chk, W.config_events(cfg), flags, every=7)
         eng.close()
@@ -61,7 +61,7 @@ def test_rows_on_16_byte_boundaries_only(name):
     eng.write_state(xs)
     eng.write_grads(gs)
     chk = P.Checker(xw, P.oracle_params(cfg), cfg.gamma, gw, cfg.storage, variant=B.A2_NO_MOMENTUM)
-    P.run_batches_and_check(eng, chk, W.config_events(cfg), B.A2_SCHED_FUSE, every=9)
+    P.run_batches_and_check(eng, chk, W.config_events(cfg), B.A2_SCHED_CHAIN, every=9)
     eng.close()
 
 
@@ -100,7 +100,7 @@ def test_whole_plan_as_a_graph_and_the_refusals():
     cfg = W.CONFIGS["cfg1"].scaled(n_events=2000)
     eng, chk = P.make_small(cfg, momentum=False)
     ev = W.config_events(cfg)
-    plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+    plan = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)
     assert plan.sched.num_batches >= 4  # long enough to be recorded as a CUDA graph
     plan.run()
     chk.plain.apply_stream(ev)
