@@ -2,9 +2,11 @@
 //
 //   event kernel      one launch per batch of worker-disjoint items. A work unit is (item, column
 //                     tile); a persistent grid strides over the units. For a unit the item's rows
-//                     (x_a, x~_a, x_b, x~_b and the gradient rows it needs) are read once with
-//                     128-bit loads, the item's operations are applied in registers in event
-//                     order, and the state rows are written once. Purely HBM-bound streaming work.
+//                     (x, x~ of its two or three workers and the gradient rows it needs) are read
+//                     once with 256- or 128-bit loads, the item's operations are applied in
+//                     registers in event order, and the state rows are written once. HBM-bound
+//                     streaming work. Separate instances for two- and three-worker items, for bf16
+//                     rows kept packed in registers, and for the dynamic without x~.
 //   consensus kernel  per column: sum_i (x_i - xbar)^2 from shifted sums, fp64 across columns,
 //                     warp shuffle + block reduce, per-block partials, fixed-order final sum.
 //
