@@ -176,6 +176,131 @@ __device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, floa
     xtb = __fadd_rn(xtb, __fmaf_rn(alpha_t, m, __fmaf_rn(alpha_t, m_lo, -ub)));
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same two updates on a PAIR of elements with sm_100's packed fp32 instructions (add/sub/mul/fma
+// .rn.f32x2: two IEEE single-precision results per issued instruction, each rounded like the scalar
+// form). The kernels with several events per row are short of issue slots, not of FP32 lanes; results
+// are bit-identical to grad_elem / comm_elem (negations are moved, which round-to-nearest commutes with).
+// ---------------------------------------------------------------------------------------------
+#ifndef A2_F32X2_FP32
+#define A2_F32X2_FP32 0  // fp32 rows: measured 1-3 % slower than the scalar forms (6.15 against 6.32 TB/s)
+#endif
+#ifndef A2_F32X2_BF16
+#define A2_F32X2_BF16 1  // bf16 rows, whose kernels issue twice as much per byte: 1-2 % faster
+#endif
+using f32x2 = unsigned long long;
+__device__ __forceinline__ f32x2 pk2(float lo, float hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+
+struct GradK {  // per-operation constants of a gradient event, both lanes equal
+    f32x2 c, nc, ngamma;
+    __device__ __forceinline__ GradK(float c_, float ngamma_) : c(pk2(c_, c_)), nc(pk2(-c_, -c_)), ngamma(pk2(ngamma_, ngamma_)) {}
+};
+template <bool ONE_ROUNDING>
+__device__ __forceinline__ void grad_pair(float& x0, float& x1, float& xt0, float& xt1, const GradK& K, float g0, float g1) {
+    f32x2 x = pk2(x0, x1), xt = pk2(xt0, xt1);
+    const f32x2 g = pk2(g0, g1);
+    const f32x2 dlt = sub2(x, xt);
+    if (!ONE_ROUNDING) {
+        x = fma2(K.ngamma, g, fma2(K.nc, dlt, x));
+        xt = fma2(K.ngamma, g, fma2(K.c, dlt, xt));
+    } else {
+        const f32x2 tg = mul2(K.ngamma, g);
+        x = add2(x, fma2(K.nc, dlt, tg));
+        xt = add2(xt, fma2(K.c, dlt, tg));
+    }
+    upk2(x, x0, x1);
+    upk2(xt, xt0, xt1);
+}
+
+struct CommK {  // per-operation constants of a communication event
+    f32x2 nca, ncb, alpha, nalpha, alpha_t, nalpha_t;
+    __device__ __forceinline__ CommK(float ca, float cb, float a, float at)
+        : nca(pk2(-ca, -ca)), ncb(pk2(-cb, -cb)), alpha(pk2(a, a)), nalpha(pk2(-a, -a)), alpha_t(pk2(at, at)), nalpha_t(pk2(-at, -at)) {}
+};
+template <bool COMPENSATED>
+__device__ __forceinline__ void comm_pair(float& xa0, float& xa1, float& xta0, float& xta1, float& xb0, float& xb1,
+                                          float& xtb0, float& xtb1, const CommK& K, bool msg_before_mix) {
+    f32x2 xa = pk2(xa0, xa1), xta = pk2(xta0, xta1), xb = pk2(xb0, xb1), xtb = pk2(xtb0, xtb1);
+    const f32x2 ua = mul2(K.nca, sub2(xa, xta));
+    const f32x2 ub = mul2(K.ncb, sub2(xb, xtb));
+    if (!COMPENSATED) {
+        const f32x2 m_pre = sub2(xa, xb);
+        xa = add2(xa, ua);
+        xta = sub2(xta, ua);
+        xb = add2(xb, ub);
+        xtb = sub2(xtb, ub);
+        const f32x2 m0 = msg_before_mix ? m_pre : sub2(xa, xb);
+        xa = fma2(K.nalpha, m0, xa);
+        xta = fma2(K.nalpha_t, m0, xta);
+        xb = fma2(K.alpha, m0, xb);
+        xtb = fma2(K.alpha_t, m0, xtb);
+    } else {
+        const f32x2 raw = sub2(xa, xb);  // xa + (-xb)
+        f32x2 bv = sub2(raw, xa);
+        f32x2 av = sub2(raw, bv);
+        const f32x2 e_raw = sub2(sub2(xa, av), add2(xb, bv));  // (xa - av) + (-xb - bv)
+        f32x2 m = raw, m_lo = e_raw;
+        if (!msg_before_mix) {
+            const f32x2 du = sub2(ua, ub);
+            m = add2(raw, du);
+            bv = sub2(m, raw);
+            av = sub2(m, bv);
+            m_lo = add2(e_raw, add2(sub2(raw, av), sub2(du, bv)));
+        }
+        xa = add2(xa, fma2(K.nalpha, m, fma2(K.nalpha, m_lo, ua)));
+        xta = sub2(xta, fma2(K.alpha_t, m, fma2(K.alpha_t, m_lo, ua)));     // + (-alpha~ m - alpha~ m_lo - ua)
+        xb = add2(xb, fma2(K.alpha, m, fma2(K.alpha, m_lo, ub)));
+        xtb = sub2(xtb, fma2(K.nalpha_t, m, fma2(K.nalpha_t, m_lo, ub)));  // + (alpha~ m + alpha~ m_lo - ub)
+    }
+    upk2(xa, xa0, xa1);
+    upk2(xta, xta0, xta1);
+    upk2(xb, xb0, xb1);
+    upk2(xtb, xtb0, xtb1);
+}
+
+// One operation on whole register rows of NE elements (NE even). PRECISE: the one-rounding / compensated forms
+// (fp32 storage); PACKED: two elements per instruction.
+template <bool PRECISE, bool PACKED, int NE>
+__device__ __forceinline__ void grad_row(float (&x)[NE], float (&xt)[NE], float c, float ngamma, const float (&g)[NE]) {
+    if constexpr (PACKED) {
+        const GradK K(c, ngamma);
+#pragma unroll
+        for (int k = 0; k < NE; k += 2) grad_pair<PRECISE>(x[k], x[k + 1], xt[k], xt[k + 1], K, g[k], g[k + 1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < NE; ++k) grad_elem<PRECISE>(x[k], xt[k], c, ngamma, g[k]);
+    }
+}
+template <bool PRECISE, bool PACKED, int NE>
+__device__ __forceinline__ void mix_row(float (&x)[NE], float (&xt)[NE], float c, float ngamma) {
+    if constexpr (PACKED) {
+        const GradK K(c, ngamma);
+#pragma unroll
+        for (int k = 0; k < NE; k += 2) grad_pair<PRECISE>(x[k], x[k + 1], xt[k], xt[k + 1], K, 0.f, 0.f);
+    } else {
+#pragma unroll
+        for (int k = 0; k < NE; ++k) grad_elem<PRECISE>(x[k], xt[k], c, ngamma, 0.f);
+    }
+}
+template <bool PRECISE, bool PACKED, int NE>
+__device__ __forceinline__ void comm_row(float (&xa)[NE], float (&xta)[NE], float (&xb)[NE], float (&xtb)[NE], float ca, float cb,
+                                         float alpha, float alpha_t, bool msg_before_mix) {
+    if constexpr (PACKED) {
+        const CommK K(ca, cb, alpha, alpha_t);
+#pragma unroll
+        for (int k = 0; k < NE; k += 2)
+            comm_pair<PRECISE>(xa[k], xa[k + 1], xta[k], xta[k + 1], xb[k], xb[k + 1], xtb[k], xtb[k + 1], K, msg_before_mix);
+    } else {
+#pragma unroll
+        for (int k = 0; k < NE; ++k) comm_elem<PRECISE>(xa[k], xta[k], xb[k], xtb[k], ca, cb, alpha, alpha_t, msg_before_mix);
+    }
+}
+
 __device__ __forceinline__ double mix_coeff(double eta, double dt) { return -0.5 * expm1(-2.0 * eta * dt); }
 
 // ---------------------------------------------------------------------------------------------
@@ -232,7 +357,8 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     // 1 % FASTER with the 64-bit division per unit and the zero fill left in (6.37 against 6.30 TB/s on 64 rows
     // of 25.6e6 columns): it is bound by DRAM alone and the extra work between units spaces its bursts of loads;
     // so it keeps them.
-    constexpr bool kRecompute = sizeof(T) == 4;
+    // (The three-worker instance issues more per byte and gains 3 % from leaving them out: 6.18 -> 6.38 TB/s.)
+    constexpr bool kRecompute = sizeof(T) == 4 && KW == 2;
     const int n_it = p.n_items;
     int rem = (int)(blockIdx.x % (unsigned)n_it);
     long long tile = blockIdx.x / (unsigned)n_it;
@@ -302,56 +428,38 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
             }
         }
 
+        constexpr bool kPrecise = sizeof(T) == 4;
+        constexpr bool kPacked = sizeof(T) == 4 ? (A2_F32X2_FP32 != 0) : (A2_F32X2_BF16 != 0);
+        const bool before = p.msg_before_mix != 0;
         for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
             const int kind = s_kind[o];
+            const float ca = s_ca[o];
             if (kind == A2_OP_GRAD_A) {
-                const float c = s_ca[o];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
-#pragma unroll
-                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], c, ngamma, ga[u][k]);
+                for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xa[u], xta[u], ca, ngamma, ga[u]);
             } else if (kind == A2_OP_GRAD_B) {
-                const float c = s_ca[o];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
-#pragma unroll
-                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], c, ngamma, gb[u][k]);
-            } else if (KW == 3 && kind == A2_OP_GRAD_C) {
-                const float c = s_ca[o];
-#pragma unroll
-                for (int u = 0; u < UC; ++u)
-#pragma unroll
-                    for (int k = 0; k < NC; ++k) grad_elem<sizeof(T) == 4>(xc[u][k], xtc[u][k], c, ngamma, gc[u][k]);
-            } else if (KW == 3 && kind == A2_OP_COMM_AC) {
-                const float ca = s_ca[o], cb = s_cb[o];
-#pragma unroll
-                for (int u = 0; u < UC; ++u)
-#pragma unroll
-                    for (int k = 0; k < NC; ++k)
-                        comm_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], xc[u][k], xtc[u][k], ca, cb, alpha, alpha_t,
-                                                  p.msg_before_mix != 0);
-            } else if (KW == 3 && kind == A2_OP_COMM_BC) {
-                const float ca = s_ca[o], cb = s_cb[o];
-#pragma unroll
-                for (int u = 0; u < UC; ++u)
-#pragma unroll
-                    for (int k = 0; k < NC; ++k)
-                        comm_elem<sizeof(T) == 4>(xb[u][k], xtb[u][k], xc[u][k], xtc[u][k], ca, cb, alpha, alpha_t,
-                                                  p.msg_before_mix != 0);
+                for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xb[u], xtb[u], ca, ngamma, gb[u]);
             } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
-                const float c = s_ca[o];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
+                for (int u = 0; u < UNROLL; ++u) mix_row<kPrecise, kPacked>(xa[u], xta[u], ca, ngamma);
+            } else if (kind == A2_OP_COMM) {
+                const float cb = s_cb[o];
 #pragma unroll
-                    for (int k = 0; k < N; ++k) grad_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], c, ngamma, 0.f);
-            } else {
-                const float ca = s_ca[o], cb = s_cb[o];
+                for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xa[u], xta[u], xb[u], xtb[u], ca, cb, alpha, alpha_t, before);
+            } else if constexpr (KW == 3) {
+                if (kind == A2_OP_GRAD_C) {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
+                    for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xc[u], xtc[u], ca, ngamma, gc[u]);
+                } else if (kind == A2_OP_COMM_AC) {
+                    const float cb = s_cb[o];
 #pragma unroll
-                    for (int k = 0; k < N; ++k)
-                        comm_elem<sizeof(T) == 4>(xa[u][k], xta[u][k], xb[u][k], xtb[u][k], ca, cb, alpha, alpha_t,
-                                                  p.msg_before_mix != 0);
+                    for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xa[u], xta[u], xc[u], xtc[u], ca, cb, alpha, alpha_t, before);
+                } else {
+                    const float cb = s_cb[o];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xb[u], xtb[u], xc[u], xtc[u], ca, cb, alpha, alpha_t, before);
+                }
             }
         }
 
@@ -726,33 +834,23 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_packed(cons
                 fb[2 * w] = bf16_lo(gb[k0 + w]); fb[2 * w + 1] = bf16_hi(gb[k0 + w]);
                 fc[2 * w] = bf16_lo(gc[k0 + w]); fc[2 * w + 1] = bf16_hi(gc[k0 + w]);
             }
+            constexpr bool kPk = A2_F32X2_BF16 != 0;
             for (int o = o_begin; o < o_end; ++o) {
                 const int kind = s_kind[o];
                 const float ca = s_ca[o];
                 if (kind == A2_OP_GRAD_A) {
-#pragma unroll
-                    for (int e = 0; e < E; ++e) grad_elem<false>(a[e], ta[e], ca, ngamma, fa[e]);
+                    grad_row<false, kPk>(a, ta, ca, ngamma, fa);
                 } else if (kind == A2_OP_GRAD_B) {
-#pragma unroll
-                    for (int e = 0; e < E; ++e) grad_elem<false>(b[e], tb[e], ca, ngamma, fb[e]);
+                    grad_row<false, kPk>(b, tb, ca, ngamma, fb);
                 } else if (kind == A2_OP_GRAD_C) {
-#pragma unroll
-                    for (int e = 0; e < E; ++e) grad_elem<false>(c[e], tc[e], ca, ngamma, fc[e]);
+                    grad_row<false, kPk>(c, tc, ca, ngamma, fc);
                 } else if (kind == A2_OP_MIX_A) {
-#pragma unroll
-                    for (int e = 0; e < E; ++e) grad_elem<false>(a[e], ta[e], ca, ngamma, 0.f);
+                    mix_row<false, kPk>(a, ta, ca, ngamma);
                 } else {
                     const float cb = s_cb[o];
-                    if (kind == A2_OP_COMM) {
-#pragma unroll
-                        for (int e = 0; e < E; ++e) comm_elem<false>(a[e], ta[e], b[e], tb[e], ca, cb, alpha, alpha_t, before);
-                    } else if (kind == A2_OP_COMM_AC) {
-#pragma unroll
-                        for (int e = 0; e < E; ++e) comm_elem<false>(a[e], ta[e], c[e], tc[e], ca, cb, alpha, alpha_t, before);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < E; ++e) comm_elem<false>(b[e], tb[e], c[e], tc[e], ca, cb, alpha, alpha_t, before);
-                    }
+                    if (kind == A2_OP_COMM) comm_row<false, kPk>(a, ta, b, tb, ca, cb, alpha, alpha_t, before);
+                    else if (kind == A2_OP_COMM_AC) comm_row<false, kPk>(a, ta, c, tc, ca, cb, alpha, alpha_t, before);
+                    else comm_row<false, kPk>(b, tb, c, tc, ca, cb, alpha, alpha_t, before);
                 }
             }
 #pragma unroll
