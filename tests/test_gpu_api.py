@@ -181,8 +181,9 @@ def test_bind_rejects_bad_buffers():
     L.a2cid2_destroy(h)
 
 
+@pytest.mark.parametrize("flags", [B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
 @pytest.mark.parametrize("storage", ["f32", "bf16"])
-def test_rows_aligned_to_16_bytes_only_take_the_128_bit_kernels(storage):
+def test_rows_aligned_to_16_bytes_only_take_the_128_bit_kernels(storage, flags):
     """Rows on 32-byte boundaries run the 256-bit kernels, rows that are only 16-byte aligned the
     128-bit ones; the arithmetic per element is the same, so the states agree bit for bit."""
     cfg = _small(storage, d=5_003, n_events=600)
@@ -195,7 +196,7 @@ def test_rows_aligned_to_16_bytes_only_take_the_128_bit_kernels(storage):
         assert (eng.x.data_ptr() % 32 == 16) == narrow
         eng.write_state(xs)
         eng.write_grads(gs)
-        eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
+        eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=flags)
         t_eval = float(ev.times[-1]) + 0.5
         outs.append((eng.read_state(), eng.consensus_distance(), eng.consensus_distance(t_eval)))
         eng.close()
