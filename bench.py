@@ -47,7 +47,7 @@ NOMINAL_HBM_GBS = 8000.0
 # d = 2e6 case), as a ratio to the bytes the launch's items must move: reads 1.000, writes 0.88
 # (the rest was still in L2 when the small launches ended). None once the kernel has changed
 # since the counters were taken.
-NCU_TRAFFIC_RATIO = 0.950
+NCU_TRAFFIC_RATIO = 0.951
 
 
 def parse_args():
