@@ -75,10 +75,11 @@ enum {
                            all in one item is appended to that item, whose rows then serve one
                            more event without crossing HBM again; (2) a communication between a
                            worker that is free earlier and one whose latest events sit in an item
-                           of two workers joins that item as its third worker, so the shared
-                           worker's rows are not written and read again in between. Every
-                           worker's own order is kept and the arithmetic per event is unchanged;
-                           batches get fewer and items longer (up to three workers)            */
+                           with room joins that item as one more worker, so the shared worker's
+                           rows are not written and read again in between. Every worker's own
+                           order is kept and the arithmetic per event is unchanged; batches get
+                           fewer and items longer (up to four workers with fp32 rows and the
+                           momentum buffer, three otherwise)                                    */
 };
 
 /* Kinds of elementary operation inside an item. */
@@ -89,7 +90,11 @@ enum {
     A2_OP_MIX_A = 3,  /* mixing only (a2cid2_flush)                                              */
     A2_OP_GRAD_C = 4,
     A2_OP_COMM_AC = 5,
-    A2_OP_COMM_BC = 6
+    A2_OP_COMM_BC = 6,
+    A2_OP_GRAD_D = 7,
+    A2_OP_COMM_AD = 8,
+    A2_OP_COMM_BD = 9,
+    A2_OP_COMM_CD = 10
 };
 
 /* Variants of the dynamic. */
@@ -106,7 +111,7 @@ enum {
                               rows. A2_SCHED_RESIDENT is not available (A2_EINVAL).               */
 };
 
-/* One item of a batch: all the work done on one worker (b = c = -1), a pair, or three workers. */
+/* One item of a batch: all the work done on one worker (b = c = d = -1) or on two to four workers. */
 typedef struct a2cid2_item_info {
     int32_t a, b;           /* worker rows; b = -1 for a gradient-only item                    */
     int32_t slot_a, slot_b; /* gradient rows read for worker a / b, or -1                       */
@@ -114,6 +119,7 @@ typedef struct a2cid2_item_info {
     int32_t n_ops;          /* operations applied, in order, while the rows sit in registers    */
     int32_t batch;          /* batch (dependency level) the item belongs to                     */
     int32_t c, slot_c;      /* third worker and its gradient row (A2_SCHED_CHAIN), or -1         */
+    int32_t d, slot_d;      /* fourth worker and its gradient row, or -1                         */
 } a2cid2_item_info;
 
 /* Counters of one a2cid2_apply_events / a2cid2_plan_run call (all device figures are what the
@@ -274,8 +280,8 @@ void a2cid2_plan_destroy(a2cid2_plan_t* p);
  * gradient-only item at the end of the stream, or when max_ops_per_item is reached or the
  * gradient slot changes). With A2_SCHED_CHAIN items also take later events of workers they already
  * hold, and a third worker (see the flag). t_last[n] are the workers' times at the start
- * (NULL = zeros). max_ops_per_item <= 0 selects the default; max_workers_per_item is 2 or 3
- * (<= 0: 3) and only matters with A2_SCHED_CHAIN. Validation and error codes as in
+ * (NULL = zeros). max_ops_per_item <= 0 selects the default; max_workers_per_item is 2, 3 or 4
+ * (<= 0: 4) and only matters with A2_SCHED_CHAIN. Validation and error codes as in
  * a2cid2_apply_events. */
 int a2cid2_sched_create(int32_t n, int32_t n_grad_slots, const double* t_last, int64_t n_events,
                         const double* times, const int32_t* wi, const int32_t* wj, const int32_t* grad_slot,

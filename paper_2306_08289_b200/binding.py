@@ -22,6 +22,7 @@ A2_SCHED_FUSE = 1
 A2_SCHED_RESIDENT = 2
 A2_SCHED_CHAIN = 4
 A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A, A2_OP_GRAD_C, A2_OP_COMM_AC, A2_OP_COMM_BC = 0, 1, 2, 3, 4, 5, 6
+A2_OP_GRAD_D, A2_OP_COMM_AD, A2_OP_COMM_BD, A2_OP_COMM_CD = 7, 8, 9, 10
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX, A2_NO_MOMENTUM = 0, 1, 2
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
@@ -31,10 +32,10 @@ ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ER
 class ItemInfo(C.Structure):
     _fields_ = [("a", C.c_int32), ("b", C.c_int32), ("slot_a", C.c_int32), ("slot_b", C.c_int32),
                 ("first_op", C.c_int64), ("n_ops", C.c_int32), ("batch", C.c_int32),
-                ("c", C.c_int32), ("slot_c", C.c_int32)]
+                ("c", C.c_int32), ("slot_c", C.c_int32), ("d", C.c_int32), ("slot_d", C.c_int32)]
 
     def workers(self):
-        return [w for w in (self.a, self.b, self.c) if w >= 0]
+        return [w for w in (self.a, self.b, self.c, self.d) if w >= 0]
 
 
 class Stats(C.Structure):

@@ -22,11 +22,11 @@ struct SchedOp {
     double t_prev_b;  // same for the second worker of a communication
 };
 
-constexpr int kMaxItemWorkers = 3;
+constexpr int kMaxItemWorkers = 4;
 
 struct SchedItem {
-    int32_t a, b, c;  // workers; b, c = -1 when absent
-    int32_t slot_a, slot_b, slot_c;
+    int32_t a, b, c, d;  // workers; b, c, d = -1 when absent
+    int32_t slot_a, slot_b, slot_c, slot_d;
     int64_t first_op;
     int32_t n_ops;
     int32_t batch;
@@ -76,7 +76,7 @@ void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, in
 
 // ---- device descriptors (layout shared by host packing and the event kernel) ---------------
 struct DevItem {
-    int32_t a, b, c, slot_a, slot_b, slot_c;
+    int32_t a, b, c, d, slot_a, slot_b, slot_c, slot_d;
     int32_t op_first;  // relative to the launch's first op
     int32_t op_count;
 };
@@ -107,13 +107,14 @@ struct EventLaunch {
     float alpha, alpha_tilde, gamma;
     int32_t variant;
     int32_t dtype;
-    bool three_workers;  // some item holds a third worker: the three-worker instance of the kernel is needed
+    int32_t max_workers;  // most workers any item of the launch holds (2, 3 or 4): selects the kernel instance
 };
 
 struct DeviceInfo {
     int sm_count = 0;
     int event_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // [storage type][128-bit / 256-bit accesses]
     int event3_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the three-worker instances
+    int event4_ctas_per_sm[2] = {0, 0};               // four-worker instances (fp32 rows only): 128-bit / 256-bit
     int plain_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};  // the same for the kernel of the dynamic without x~
     int plain3_ctas_per_sm[2][2] = {{0, 0}, {0, 0}};
     int consensus_ctas_per_sm = 0;

@@ -1,6 +1,7 @@
 // C ABI of the engine: handle, plans, validation, descriptor upload, launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <chrono>
 #include <cmath>
 #include <cstdio>
@@ -31,7 +32,7 @@ namespace {
 struct LaunchRange {
     int64_t item0, item1;  // items of the plan covered by this launch
     int64_t op0, op1;
-    bool three = false;  // some item of the launch holds a third worker
+    int workers = 2;  // most workers any item of the launch holds
 };
 
 // Grow-only pinned + device buffer pair used to ship the descriptors of one apply_events call.
@@ -53,7 +54,7 @@ struct a2cid2 {
     double eta = 0, alpha = 0, alpha_tilde = 0, gamma = 0;
     int32_t dtype = A2_F32;
     int32_t variant = A2_MSG_AFTER_MIX;
-    int32_t item_workers = a2::kMaxItemWorkers;  // most workers A2_SCHED_CHAIN puts into one item
+    int32_t item_workers = a2::kMaxItemWorkers;  // most workers A2_SCHED_CHAIN puts into one item (before the kernels' limits)
     // borrowed buffers
     void* x = nullptr;
     void* xt = nullptr;
@@ -153,11 +154,12 @@ void make_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches, st
         int64_t i = s.batch_first[(size_t)b];
         const int64_t iend = s.batch_first[(size_t)b + 1];
         while (i < iend) {
-            LaunchRange L{i, i, s.items[(size_t)i].first_op, s.items[(size_t)i].first_op, false};
+            LaunchRange L{i, i, s.items[(size_t)i].first_op, s.items[(size_t)i].first_op, 2};
             while (L.item1 < iend && (L.item1 - L.item0) < a2::kMaxItemsPerLaunch &&
                    (L.op1 - L.op0) + s.items[(size_t)L.item1].n_ops <= a2::kMaxOpsPerLaunch) {
                 L.op1 += s.items[(size_t)L.item1].n_ops;
-                L.three = L.three || s.items[(size_t)L.item1].c >= 0;
+                const a2::SchedItem& si = s.items[(size_t)L.item1];
+                L.workers = std::max(L.workers, si.d >= 0 ? 4 : (si.c >= 0 ? 3 : 2));
                 L.item1 += 1;
             }
             launches.push_back(L);
@@ -207,12 +209,13 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
         for (const LaunchRange& L : pk.launches)
             for (int64_t k = L.item0; k < L.item1; ++k) {
                 const a2::SchedItem& it = s.items[(size_t)k];
-                di[k] = DevItem{it.a, it.b, it.c, it.slot_a, it.slot_b, it.slot_c, (int32_t)(it.first_op - L.op0), it.n_ops};
+                di[k] = DevItem{it.a, it.b, it.c, it.d, it.slot_a, it.slot_b, it.slot_c, it.slot_d,
+                                (int32_t)(it.first_op - L.op0), it.n_ops};
             }
     } else {
         for (size_t k = 0; k < s.items.size(); ++k) {  // one operation per item; slot_b carries the cache index
             const a2::SchedItem& it = s.items[k];
-            di[k] = DevItem{it.a, it.b, -1, it.slot_a, pk.cache_idx[k], -1, (int32_t)k, 1};
+            di[k] = DevItem{it.a, it.b, -1, -1, it.slot_a, pk.cache_idx[k], -1, -1, (int32_t)k, 1};
         }
         if (!pk.chunks.empty())
             std::memcpy(static_cast<char*>(dst) + pk.chunks_off, pk.chunks.data(), pk.chunks.size() * sizeof(a2::ResChunk));
@@ -250,6 +253,8 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     }
     for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
         const LaunchRange& R = pk.launches[(size_t)l];
+        if (R.workers > ((h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3))
+            return fail(h, A2_ESTATE, "this plan holds four-worker items, which the kernels of the current variant do not take");
         a2::EventLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.items = d_items + R.item0;
@@ -259,11 +264,18 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.eta = h->eta;
         L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
         L.variant = h->variant; L.dtype = h->dtype;
-        L.three_workers = R.three;
+        L.max_workers = R.workers;
         const int rc = a2::launch_events(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
     return A2_OK;
+}
+
+// Most workers per item the kernels of the handle's storage type and variant take: four with fp32 rows and the
+// momentum buffer, three with bf16 rows or without x~.
+int32_t item_workers(const a2cid2* h) {
+    const int32_t cap = (h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3;
+    return h->item_workers < cap ? h->item_workers : cap;
 }
 
 constexpr int64_t kGraphMinLaunches = 4;
@@ -318,16 +330,17 @@ void advance_times(const a2cid2_sched& s, int64_t b0, int64_t b1, std::vector<do
         for (int32_t o = 0; o < it.n_ops; ++o) {
             const a2::SchedOp& op = s.ops[(size_t)(it.first_op + o)];
             const int32_t k = op.kind;
-            if (k == A2_OP_GRAD_A || k == A2_OP_MIX_A || k == A2_OP_COMM || k == A2_OP_COMM_AC) t[(size_t)it.a] = op.t;
-            if (k == A2_OP_GRAD_B || k == A2_OP_COMM || k == A2_OP_COMM_BC) t[(size_t)it.b] = op.t;
-            if (k == A2_OP_GRAD_C || k == A2_OP_COMM_AC || k == A2_OP_COMM_BC) t[(size_t)it.c] = op.t;
+            if (k == A2_OP_GRAD_A || k == A2_OP_MIX_A || k == A2_OP_COMM || k == A2_OP_COMM_AC || k == A2_OP_COMM_AD) t[(size_t)it.a] = op.t;
+            if (k == A2_OP_GRAD_B || k == A2_OP_COMM || k == A2_OP_COMM_BC || k == A2_OP_COMM_BD) t[(size_t)it.b] = op.t;
+            if (k == A2_OP_GRAD_C || k == A2_OP_COMM_AC || k == A2_OP_COMM_BC || k == A2_OP_COMM_CD) t[(size_t)it.c] = op.t;
+            if (k == A2_OP_GRAD_D || k == A2_OP_COMM_AD || k == A2_OP_COMM_BD || k == A2_OP_COMM_CD) t[(size_t)it.d] = op.t;
         }
     }
 }
 
 bool needs_gradients(const a2cid2_sched& s) {
     for (const a2::SchedItem& it : s.items)
-        if (it.slot_a >= 0 || it.slot_b >= 0 || it.slot_c >= 0) return true;
+        if (it.slot_a >= 0 || it.slot_b >= 0 || it.slot_c >= 0 || it.slot_d >= 0) return true;
     return false;
 }
 
@@ -518,7 +531,7 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
     const double t0 = now_ms();
     a2cid2_sched* s = nullptr;
     std::string err;
-    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, h->item_workers,
+    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, item_workers(h),
                             &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     return submit_schedule(h, s, stats, t0);
@@ -542,7 +555,7 @@ int a2cid2_flush(a2cid2_t* h, double t_flush) {
     s->t_final = h->t;
     for (int32_t w = 0; w < h->n; ++w) {  // one batch: a mixing-only item per worker that is behind
         if (h->t[(size_t)w] == t_flush) continue;
-        s->items.push_back(a2::SchedItem{w, -1, -1, -1, -1, -1, (int64_t)s->ops.size(), 1, 0});
+        s->items.push_back(a2::SchedItem{w, -1, -1, -1, -1, -1, -1, -1, (int64_t)s->ops.size(), 1, 0});
         s->ops.push_back(a2::SchedOp{-1, A2_OP_MIX_A, t_flush, h->t[(size_t)w], 0.0});
         s->t_final[(size_t)w] = t_flush;
     }
@@ -638,7 +651,7 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
     a2cid2_sched* s = nullptr;
     std::string err;
     rc = a2::build_schedule(h->n, h->n_slots, t_start ? t_start : h->t.data(), n_events, times, wi, wj, grad_slot, flags,
-                            0, h->item_workers, &s, err);
+                            0, item_workers(h), &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     a2cid2_plan* p = new (std::nothrow) a2cid2_plan();
     if (!p) { a2cid2_sched_destroy(s); return fail(h, A2_ENOMEM, "out of host memory"); }
@@ -754,7 +767,7 @@ int a2cid2_sched_item(const a2cid2_sched_t* s, int64_t item, a2cid2_item_info* o
     if (!s || !out) return fail(nullptr, A2_EINVAL, "NULL argument");
     if (item < 0 || item >= (int64_t)s->items.size()) return fail(nullptr, A2_ERANGE, "item out of range");
     const a2::SchedItem& it = s->items[(size_t)item];
-    *out = a2cid2_item_info{it.a, it.b, it.slot_a, it.slot_b, it.first_op, it.n_ops, it.batch, it.c, it.slot_c};
+    *out = a2cid2_item_info{it.a, it.b, it.slot_a, it.slot_b, it.first_op, it.n_ops, it.batch, it.c, it.slot_c, it.d, it.slot_d};
     return A2_OK;
 }
 

@@ -322,9 +322,10 @@ struct EventArgs {
     int msg_before_mix;
 };
 
-// KW = 2 or 3: workers an item may hold (three-worker items come from A2_SCHED_CHAIN schedules).
-template <typename T, int BYTES, int UNROLL, int KW>
-__global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs p) {
+// KW = 2, 3 or 4: workers an item may hold (items of more than two workers come from A2_SCHED_CHAIN schedules).
+// THREADS: threads per CTA (the four-worker instance trades threads for registers).
+template <typename T, int BYTES, int UNROLL, int KW, int THREADS = kEventThreads>
+__global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
@@ -332,11 +333,12 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
     __shared__ float s_cb[kMaxOpsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
 
-    for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
-    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
+    for (int i = threadIdx.x; i < p.n_items; i += THREADS) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += THREADS) {
         const DevOp op = p.ops[o];
         s_kind[o] = (unsigned char)op.kind;
-        const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC;
+        const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC ||
+                          op.kind == A2_OP_COMM_AD || op.kind == A2_OP_COMM_BD || op.kind == A2_OP_COMM_CD;
         s_ca[o] = (float)mix_coeff(p.eta, op.t - op.t_prev_a);  // the operation's first (or only) worker
         s_cb[o] = comm ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
     }
@@ -379,8 +381,9 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
         const int item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
         const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
-        const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
-        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
+        const bool has_c = KW >= 3 && it.c >= 0, has_gc = KW >= 3 && it.slot_c >= 0;
+        const bool has_d = KW >= 4 && it.d >= 0, has_gd = KW >= 4 && it.slot_d >= 0;
+        const long long v0 = tile * (long long)(THREADS * UNROLL) + threadIdx.x;
 
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxta = Xt + (long long)it.a * p.pitch;
@@ -391,20 +394,24 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
         const T* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
         const T* const pgb = G + (long long)(has_gb ? it.slot_b : 0) * p.pitch;
         const T* const pgc = G + (long long)(has_gc ? it.slot_c : 0) * p.pitch;
+        T* const pxd = X + (long long)(has_d ? it.d : it.a) * p.pitch;
+        T* const pxtd = Xt + (long long)(has_d ? it.d : it.a) * p.pitch;
+        const T* const pgd = G + (long long)(has_gd ? it.slot_d : 0) * p.pitch;
 
-        constexpr int UC = KW == 3 ? UNROLL : 1, NC = KW == 3 ? N : 1;  // no registers for a worker the instance never has
+        constexpr int UC = KW >= 3 ? UNROLL : 1, NC = KW >= 3 ? N : 1;  // no registers for a worker the instance never has
+        constexpr int UD = KW >= 4 ? UNROLL : 1, ND = KW >= 4 ? N : 1;
         float xa[UNROLL][N], xta[UNROLL][N], xb[UNROLL][N], xtb[UNROLL][N], ga[UNROLL][N], gb[UNROLL][N];
-        float xc[UC][NC], xtc[UC][NC], gc[UC][NC];
+        float xc[UC][NC], xtc[UC][NC], gc[UC][NC], xd[UD][ND], xtd[UD][ND], gd[UD][ND];
         bool live[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const long long v = v0 + (long long)u * kEventThreads;
+            const long long v = v0 + (long long)u * THREADS;
             live[u] = v < p.n_vec;
             const long long off = v * N;
             if (kRecompute) {
 #pragma unroll
                 for (int k = 0; k < N; ++k) { xb[u][k] = 0.f; xtb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; xa[u][k] = 0.f; xta[u][k] = 0.f; }
-                if constexpr (KW == 3) {
+                if constexpr (KW >= 3) {
 #pragma unroll
                     for (int k = 0; k < NC; ++k) { xc[u][k] = 0.f; xtc[u][k] = 0.f; gc[u][k] = 0.f; }
                 }
@@ -418,12 +425,19 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 }
                 if (has_ga) V::load(pga + off, ga[u]);
                 if (has_gb) V::load(pgb + off, gb[u]);
-                if constexpr (KW == 3) {
+                if constexpr (KW >= 3) {
                     if (has_c) {
                         V::load(pxc + off, xc[u]);
                         V::load(pxtc + off, xtc[u]);
                     }
                     if (has_gc) V::load(pgc + off, gc[u]);
+                }
+                if constexpr (KW >= 4) {
+                    if (has_d) {
+                        V::load(pxd + off, xd[u]);
+                        V::load(pxtd + off, xtd[u]);
+                    }
+                    if (has_gd) V::load(pgd + off, gd[u]);
                 }
             }
         }
@@ -447,7 +461,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                 const float cb = s_cb[o];
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xa[u], xta[u], xb[u], xtb[u], ca, cb, alpha, alpha_t, before);
-            } else if constexpr (KW == 3) {
+            } else if constexpr (KW >= 3) {
                 if (kind == A2_OP_GRAD_C) {
 #pragma unroll
                     for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xc[u], xtc[u], ca, ngamma, gc[u]);
@@ -455,17 +469,34 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                     const float cb = s_cb[o];
 #pragma unroll
                     for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xa[u], xta[u], xc[u], xtc[u], ca, cb, alpha, alpha_t, before);
-                } else {
+                } else if (kind == A2_OP_COMM_BC) {
                     const float cb = s_cb[o];
 #pragma unroll
                     for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xb[u], xtb[u], xc[u], xtc[u], ca, cb, alpha, alpha_t, before);
+                } else if constexpr (KW >= 4) {
+                    if (kind == A2_OP_GRAD_D) {
+#pragma unroll
+                        for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xd[u], xtd[u], ca, ngamma, gd[u]);
+                    } else {
+                        const float cb = s_cb[o];
+                        if (kind == A2_OP_COMM_AD) {
+#pragma unroll
+                            for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xa[u], xta[u], xd[u], xtd[u], ca, cb, alpha, alpha_t, before);
+                        } else if (kind == A2_OP_COMM_BD) {
+#pragma unroll
+                            for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xb[u], xtb[u], xd[u], xtd[u], ca, cb, alpha, alpha_t, before);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < UNROLL; ++u) comm_row<kPrecise, kPacked>(xc[u], xtc[u], xd[u], xtd[u], ca, cb, alpha, alpha_t, before);
+                        }
+                    }
                 }
             }
         }
 
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const long long off = (v0 + (long long)u * kEventThreads) * N;
+            const long long off = (v0 + (long long)u * THREADS) * N;
             if (live[u]) {
                 V::store(pxa + off, xa[u]);
                 V::store(pxta + off, xta[u]);
@@ -473,10 +504,16 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events(const EventArgs 
                     V::store(pxb + off, xb[u]);
                     V::store(pxtb + off, xtb[u]);
                 }
-                if constexpr (KW == 3) {
+                if constexpr (KW >= 3) {
                     if (has_c) {
                         V::store(pxc + off, xc[u]);
                         V::store(pxtc + off, xtc[u]);
+                    }
+                }
+                if constexpr (KW >= 4) {
+                    if (has_d) {
+                        V::store(pxd + off, xd[u]);
+                        V::store(pxtd + off, xtd[u]);
                     }
                 }
             }
@@ -961,24 +998,31 @@ __global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __re
     }
 }
 
-template <typename T, int BYTES, int KW>
+#ifndef A2_EVENT4_THREADS
+#define A2_EVENT4_THREADS 192  // threads per CTA of the four-worker instance
+#endif
+#ifndef A2_EVENT4_UNROLL_128
+#define A2_EVENT4_UNROLL_128 1
+#endif
+
+template <typename T, int BYTES, int KW, int THREADS = kEventThreads, int U = EventCfg<T, BYTES>::UNROLL>
 int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
-    constexpr int U = EventCfg<T, BYTES>::UNROLL;
     constexpr int N = Vec<T, BYTES>::N;
     EventArgs a;
     a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
     a.n_vec = (L.d + N - 1) / N;
     a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
-    const long long vec_per_tile = (long long)kEventThreads * U;
+    const long long vec_per_tile = (long long)THREADS * U;
     a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    const int per_sm = (KW == 3 ? dev.event3_ctas_per_sm : dev.event_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
+    const int per_sm = KW == 4 ? dev.event4_ctas_per_sm[BYTES == 32 ? 1 : 0]
+                               : (KW == 3 ? dev.event3_ctas_per_sm : dev.event_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
     long long grid = (long long)dev.sm_count * per_sm;
     if (grid > n_units) grid = n_units;
     if (grid < 1) return 0;
-    k_apply_events<T, BYTES, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    k_apply_events<T, BYTES, U, KW, THREADS><<<(unsigned)grid, THREADS, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -1098,6 +1142,21 @@ int query_device(DeviceInfo* info) {
     if ((e = event_occupancy<float, 32, 2>(&info->event_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<__nv_bfloat16, 16, 2>(&info->event_ctas_per_sm[1][0])) != cudaSuccess) return (int)e;
     info->event_ctas_per_sm[1][1] = info->event_ctas_per_sm[1][0];
+    {
+        int occ = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+            &occ, k_apply_events<float, 16, A2_EVENT4_UNROLL_128, 4, kEventThreads>, kEventThreads, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->event4_ctas_per_sm[0] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events<float, 32, 1, 4, A2_EVENT4_THREADS>,
+                                                          A2_EVENT4_THREADS, 0);
+        if (e != cudaSuccess) return (int)e;
+        info->event4_ctas_per_sm[1] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
+        if (const char* v = std::getenv("A2CID2_EVENT4_CTAS_PER_SM")) {  // tuning override
+            const int k = std::atoi(v);
+            if (k > 0) info->event4_ctas_per_sm[0] = info->event4_ctas_per_sm[1] = k;
+        }
+    }
     if ((e = event_occupancy<float, 16, 3>(&info->event3_ctas_per_sm[0][0])) != cudaSuccess) return (int)e;
     if ((e = event_occupancy<float, 32, 3>(&info->event3_ctas_per_sm[0][1])) != cudaSuccess) return (int)e;
     {
@@ -1189,16 +1248,21 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
             static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
             const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.g);
             const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;
-            if (L.three_workers)
+            if (L.max_workers >= 3)
                 return wide_bf16 ? launch_plain_bf16<8, 3>(L, dev, stream) : launch_plain_bf16<4, 3>(L, dev, stream);
             return wide_bf16 ? launch_plain_bf16<8, 2>(L, dev, stream) : launch_plain_bf16<4, 2>(L, dev, stream);
         }
-        if (L.three_workers)
+        if (L.max_workers >= 3)
             return wide_x ? launch_plain_t<float, 32, 3>(L, dev, stream) : launch_plain_t<float, 16, 3>(L, dev, stream);
         return wide_x ? launch_plain_t<float, 32, 2>(L, dev, stream) : launch_plain_t<float, 16, 2>(L, dev, stream);
     }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
-    if (L.three_workers) {
+    if (L.max_workers >= 4 && L.dtype != A2_BF16) {
+        static const bool narrow4 = std::getenv("A2CID2_EVENT4_128BIT") != nullptr;  // tuning override
+        if (wide && !narrow4) return launch_events_t<float, 32, 4, A2_EVENT4_THREADS, 1>(L, dev, stream);
+        return launch_events_t<float, 16, 4, kEventThreads, A2_EVENT4_UNROLL_128>(L, dev, stream);
+    }
+    if (L.max_workers >= 3) {
         if (L.dtype == A2_BF16) {
             static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
             const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.xt) |

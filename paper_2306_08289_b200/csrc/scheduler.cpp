@@ -39,7 +39,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     if (n_events > 0 && (!times || !wi || !wj || !slot)) { err = "event arrays are NULL"; return A2_EINVAL; }
     if (flags & ~uint32_t(A2_SCHED_FUSE | A2_SCHED_RESIDENT | A2_SCHED_CHAIN)) { err = "unknown scheduling flag"; return A2_EINVAL; }
     if (max_workers_per_item <= 0) max_workers_per_item = kMaxItemWorkers;
-    if (max_workers_per_item < 2 || max_workers_per_item > kMaxItemWorkers) { err = "an item holds 2 or 3 workers"; return A2_EINVAL; }
+    if (max_workers_per_item < 2 || max_workers_per_item > kMaxItemWorkers) { err = "an item holds 2 to 4 workers"; return A2_EINVAL; }
     if (max_ops_per_item <= 0) max_ops_per_item = kDefaultMaxOpsPerItem;
     if (max_ops_per_item > kMaxOpsPerLaunch) max_ops_per_item = kMaxOpsPerLaunch;
     const bool resident = (flags & A2_SCHED_RESIDENT) != 0;
@@ -106,7 +106,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
 
         auto new_item = [&](int32_t a, int32_t b, int32_t batch) -> int64_t {
             Build bd;
-            bd.it = SchedItem{a, b, -1, -1, -1, -1, 0, 0, batch};
+            bd.it = SchedItem{a, b, -1, -1, -1, -1, -1, -1, 0, 0, batch};
             items.push_back(bd);
             return (int64_t)items.size() - 1;
         };
@@ -119,8 +119,10 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             bd.tail = o;
             bd.it.n_ops += 1;
         };
-        auto local_of = [&](const SchedItem& it, int32_t w) -> int { return it.a == w ? 0 : (it.b == w ? 1 : 2); };
-        auto slot_ref = [&](SchedItem& it, int l) -> int32_t& { return l == 0 ? it.slot_a : (l == 1 ? it.slot_b : it.slot_c); };
+        auto local_of = [&](const SchedItem& it, int32_t w) -> int { return it.a == w ? 0 : (it.b == w ? 1 : (it.c == w ? 2 : 3)); };
+        auto slot_ref = [&](SchedItem& it, int l) -> int32_t& {
+            return l == 0 ? it.slot_a : (l == 1 ? it.slot_b : (l == 2 ? it.slot_c : it.slot_d));
+        };
         // can the held-back gradient events of worker w go into item k (which holds w)?
         auto slot_ok = [&](int64_t k, int32_t w) -> bool {
             const Pending& p = pend[(size_t)w];
@@ -136,7 +138,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             SchedItem& it = items[(size_t)k].it;
             const int l = local_of(it, w);
             slot_ref(it, l) = p.slot;
-            const int32_t kind = l == 0 ? A2_OP_GRAD_A : (l == 1 ? A2_OP_GRAD_B : A2_OP_GRAD_C);
+            const int32_t kind = l == 0 ? A2_OP_GRAD_A : (l == 1 ? A2_OP_GRAD_B : (l == 2 ? A2_OP_GRAD_C : A2_OP_GRAD_D));
             for (int64_t e : p.events) {
                 add_op(k, SchedOp{e, kind, times[e], tcur[(size_t)w], 0.0});
                 tcur[(size_t)w] = times[e];
@@ -150,7 +152,11 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             int li = local_of(it, i), lj = local_of(it, j);
             int32_t wa = i, wb = j;
             if (li > lj) { std::swap(li, lj); std::swap(wa, wb); }  // the update is symmetric in the two workers
-            const int32_t kind = lj == 1 ? A2_OP_COMM : (li == 0 ? A2_OP_COMM_AC : A2_OP_COMM_BC);
+            static const int32_t kPair[4][4] = {{-1, A2_OP_COMM, A2_OP_COMM_AC, A2_OP_COMM_AD},
+                                                {-1, -1, A2_OP_COMM_BC, A2_OP_COMM_BD},
+                                                {-1, -1, -1, A2_OP_COMM_CD},
+                                                {-1, -1, -1, -1}};
+            const int32_t kind = kPair[li][lj];
             add_op(k, SchedOp{e, kind, times[e], tcur[(size_t)wa], tcur[(size_t)wb]});
             tcur[(size_t)i] = times[e];
             tcur[(size_t)j] = times[e];
@@ -202,11 +208,11 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
                 if (level[(size_t)i] != level[(size_t)j]) {
                     const int32_t hi = level[(size_t)i] > level[(size_t)j] ? i : j, lo = hi == i ? j : i;
                     const int64_t kh = last_item[(size_t)hi];
-                    const int held = kh < 0 ? 0 : (items[(size_t)kh].it.b < 0 ? 1 : (items[(size_t)kh].it.c < 0 ? 2 : 3));
+                    const int held = kh < 0 ? 0 : (items[(size_t)kh].it.b < 0 ? 1 : (items[(size_t)kh].it.c < 0 ? 2 : (items[(size_t)kh].it.d < 0 ? 3 : 4)));
                     if (kh >= 0 && held + 1 <= max_workers_per_item && slot_ok(kh, hi) &&
                         items[(size_t)kh].it.n_ops + need <= max_ops_per_item) {
                         SchedItem& it = items[(size_t)kh].it;
-                        if (it.b < 0) it.b = lo; else it.c = lo;
+                        if (it.b < 0) it.b = lo; else if (it.c < 0) it.c = lo; else it.d = lo;
                         push_pending(kh, i);
                         push_pending(kh, j);
                         push_comm(kh, e, i, j);
@@ -310,15 +316,17 @@ void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, in
     for (int64_t k = i0; k < i1; ++k) {
         const SchedItem& it = s.items[(size_t)k];
         const int64_t per_worker = momentum ? 2 : 1;  // x and x~, or x alone
-        const int64_t state_rows = (1 + (it.b >= 0 ? 1 : 0) + (it.c >= 0 ? 1 : 0)) * per_worker;
+        const int64_t state_rows = (1 + (it.b >= 0 ? 1 : 0) + (it.c >= 0 ? 1 : 0) + (it.d >= 0 ? 1 : 0)) * per_worker;
         bool touches_state = momentum;  // without x~ a mixing-only item moves nothing
         for (int32_t o = 0; o < it.n_ops && !touches_state; ++o)
             touches_state = s.ops[(size_t)(it.first_op + o)].kind != A2_OP_MIX_A;
         if (touches_state)
-            rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0) + (it.slot_c >= 0 ? 1 : 0);
+            rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0) + (it.slot_c >= 0 ? 1 : 0) +
+                          (it.slot_d >= 0 ? 1 : 0);
         for (int32_t o = 0; o < it.n_ops; ++o) {
             const int32_t kind = s.ops[(size_t)(it.first_op + o)].kind;
-            if (kind == A2_OP_COMM || kind == A2_OP_COMM_AC || kind == A2_OP_COMM_BC) { st.n_comm += 1; rows_single += momentum ? 8 : 4; }
+            if (kind == A2_OP_COMM || kind == A2_OP_COMM_AC || kind == A2_OP_COMM_BC || kind == A2_OP_COMM_AD ||
+                kind == A2_OP_COMM_BD || kind == A2_OP_COMM_CD) { st.n_comm += 1; rows_single += momentum ? 8 : 4; }
             else if (kind == A2_OP_MIX_A) { rows_single += momentum ? 4 : 0; }
             else { st.n_grad += 1; rows_single += momentum ? 5 : 3; }
         }

@@ -54,11 +54,13 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
             assert it.batch == b and it.n_ops >= 1
             ws = set(it.workers())
             assert len(ws) == len(it.workers()) and not (ws & used)
-            assert (it.c < 0 or it.b >= 0) and (flags == B.A2_SCHED_CHAIN or it.c < 0)
+            assert (it.c < 0 or it.b >= 0) and (it.d < 0 or it.c >= 0) and (flags == B.A2_SCHED_CHAIN or it.c < 0)
             used |= ws
             evs, kinds = s.ops(it.first_op, it.n_ops)
-            pairs = {B.A2_OP_COMM: (it.a, it.b), B.A2_OP_COMM_AC: (it.a, it.c), B.A2_OP_COMM_BC: (it.b, it.c)}
-            grads = {B.A2_OP_GRAD_A: (it.a, it.slot_a), B.A2_OP_GRAD_B: (it.b, it.slot_b), B.A2_OP_GRAD_C: (it.c, it.slot_c)}
+            pairs = {B.A2_OP_COMM: (it.a, it.b), B.A2_OP_COMM_AC: (it.a, it.c), B.A2_OP_COMM_BC: (it.b, it.c),
+                     B.A2_OP_COMM_AD: (it.a, it.d), B.A2_OP_COMM_BD: (it.b, it.d), B.A2_OP_COMM_CD: (it.c, it.d)}
+            grads = {B.A2_OP_GRAD_A: (it.a, it.slot_a), B.A2_OP_GRAD_B: (it.b, it.slot_b), B.A2_OP_GRAD_C: (it.c, it.slot_c),
+                     B.A2_OP_GRAD_D: (it.d, it.slot_d)}
             for e, kd in zip(evs, kinds):
                 if kd in pairs:
                     # the pair may be stored the other way round: the update is symmetric in its two workers
@@ -84,8 +86,11 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
             f = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
             assert st["bytes_moved"] < f.stats(cfg.d, 4)["bytes_moved"] and s.num_batches < f.num_batches
             two = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags, max_workers_per_item=2)
+            three = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags, max_workers_per_item=3)
             assert all(two.item(k).c < 0 for k in range(two.num_items))
-            assert st["bytes_moved"] <= two.stats(cfg.d, 4)["bytes_moved"] <= f.stats(cfg.d, 4)["bytes_moved"]
+            assert all(three.item(k).d < 0 for k in range(three.num_items))
+            assert (st["bytes_moved"] <= three.stats(cfg.d, 4)["bytes_moved"] <= two.stats(cfg.d, 4)["bytes_moved"]
+                    <= f.stats(cfg.d, 4)["bytes_moved"])
     else:
         assert st["bytes_moved"] == st["bytes_one_by_one"] and s.num_items == len(ev)
 
@@ -121,10 +126,11 @@ def test_fusion_folds_pending_gradients_and_respects_caps():
 
 def test_chaining_appends_to_the_item_that_holds_the_rows_and_takes_a_third_worker():
     # comm(0,1); gradient on 1; comm(0,1) again -> one item, nothing re-read; then comm(1,2) with 2 free earlier
-    # -> worker 2 joins as the third worker; then comm(2,3): 3 is free earlier, but the item is full -> new item
+    # -> worker 2 joins as the third worker; then comm(2,3): 3 is free earlier, but with three workers per item
+    # the item is full -> new item
     times = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0]
     wi, wj, sl = [0, 1, 1, 2, 2, 3], [1, -1, 0, 1, 3, -1], [-1, 1, -1, -1, -1, 3]
-    s = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN)
+    s = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=3)
     assert s.num_items == 2 and s.num_batches == 2
     it = s.item(0)
     evs, kinds = s.ops(it.first_op, it.n_ops)
@@ -137,6 +143,13 @@ def test_chaining_appends_to_the_item_that_holds_the_rows_and_takes_a_third_work
     assert (tail.a, tail.b, tail.c, tail.slot_b) == (2, 3, -1, 3) and list(evs) == [4, 5]
     assert list(kinds) == [B.A2_OP_COMM, B.A2_OP_GRAD_B]
     assert np.array_equal(s.t_final(4), [3.0, 4.0, 5.0, 6.0])
+    # four workers per item (the default): everything fits one item, worker 3 is its fourth
+    s4 = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN)
+    it4 = s4.item(0)
+    evs, kinds = s4.ops(it4.first_op, it4.n_ops)
+    assert s4.num_items == 1 and (it4.a, it4.b, it4.c, it4.d, it4.slot_b, it4.slot_d) == (0, 1, 2, 3, 1, 3)
+    assert list(evs) == [0, 1, 2, 3, 4, 5]
+    assert list(kinds) == [B.A2_OP_COMM, B.A2_OP_GRAD_B, B.A2_OP_COMM, B.A2_OP_COMM_BC, B.A2_OP_COMM_CD, B.A2_OP_GRAD_D]
     # two workers per item at most: the third comm opens a new item
     s2 = B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=2)
     assert s2.num_items == 3 and all(s2.item(k).c < 0 for k in range(3))
@@ -145,7 +158,7 @@ def test_chaining_appends_to_the_item_that_holds_the_rows_and_takes_a_third_work
     rows = [(s3.item(k).slot_a, s3.item(k).n_ops) for k in range(s3.num_items)]
     assert rows == [(0, 2), (1, 2)]
     with pytest.raises(B.A2Error):
-        B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=4)
+        B.Schedule(4, 4, times, wi, wj, sl, flags=B.A2_SCHED_CHAIN, max_workers_per_item=5)
 
 
 def test_empty_stream_and_start_times():
@@ -248,7 +261,7 @@ def test_random_streams_property():
                 wi.append(i); wj.append(-1); sl.append(draw(st.integers(0, n_slots - 1)))
         flags = draw(st.sampled_from([0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_CHAIN]))
         cap = draw(st.sampled_from([0, 2, 3, 5]))
-        kw = draw(st.sampled_from([0, 2, 3]))
+        kw = draw(st.sampled_from([0, 2, 3, 4]))
         return (n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32),
                 flags, cap, kw)
 
@@ -270,10 +283,10 @@ def test_random_streams_property():
                 it = s.item(k)
                 ws = set(it.workers())
                 assert not (ws & used) and (cap == 0 or it.n_ops <= max(cap, 1))
-                assert len(ws) <= (kw or 3) and (flags == B.A2_SCHED_CHAIN or len(ws) <= 2)
+                assert len(ws) <= (kw or 4) and (flags == B.A2_SCHED_CHAIN or len(ws) <= 2)
                 used |= ws
                 evs, kinds = s.ops(it.first_op, it.n_ops)
-                slots = {B.A2_OP_GRAD_A: it.slot_a, B.A2_OP_GRAD_B: it.slot_b, B.A2_OP_GRAD_C: it.slot_c}
+                slots = {B.A2_OP_GRAD_A: it.slot_a, B.A2_OP_GRAD_B: it.slot_b, B.A2_OP_GRAD_C: it.slot_c, B.A2_OP_GRAD_D: it.slot_d}
                 for x, kd in zip(evs, kinds):  # one gradient row per worker and item
                     assert kd not in slots or sl[x] == slots[kd]
                 e = evs[np.argsort(times[evs], kind="stable")]
