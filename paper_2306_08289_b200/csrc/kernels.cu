@@ -185,6 +185,10 @@ __device__ __forceinline__ void comm_elem(float& xa, float& xta, float& xb, floa
 #ifndef A2_F32X2_FP32
 #define A2_F32X2_FP32 0  // fp32 rows: measured 1-3 % slower than the scalar forms (6.15 against 6.32 TB/s)
 #endif
+#ifndef A2_F32X2_FP32_KW4
+#define A2_F32X2_FP32_KW4 1  // ... except in the four-worker instance with 256-bit accesses, which is short of issue
+                             // slots: 37.4k -> 40.4k events/s (5.74 -> 6.25 TB/s) on the 64-worker ring
+#endif
 #ifndef A2_F32X2_BF16
 #define A2_F32X2_BF16 1  // bf16 rows, whose kernels issue twice as much per byte: 1-2 % faster
 #endif
@@ -443,7 +447,8 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
         }
 
         constexpr bool kPrecise = sizeof(T) == 4;
-        constexpr bool kPacked = sizeof(T) == 4 ? (A2_F32X2_FP32 != 0) : (A2_F32X2_BF16 != 0);
+        constexpr bool kPacked = sizeof(T) == 4 ? ((KW >= 4 && BYTES == 32) ? (A2_F32X2_FP32_KW4 != 0) : (A2_F32X2_FP32 != 0))
+                                                : (A2_F32X2_BF16 != 0);
         const bool before = p.msg_before_mix != 0;
         for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
             const int kind = s_kind[o];
@@ -1002,7 +1007,7 @@ __global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __re
 #define A2_EVENT4_THREADS 192  // threads per CTA of the four-worker instance
 #endif
 #ifndef A2_EVENT4_UNROLL_128
-#define A2_EVENT4_UNROLL_128 1
+#define A2_EVENT4_UNROLL_128 2
 #endif
 
 template <typename T, int BYTES, int KW, int THREADS = kEventThreads, int U = EventCfg<T, BYTES>::UNROLL>
