@@ -43,11 +43,11 @@ from paper_2306_08289_b200.distutil import Ranks, aggregate_throughput  # noqa: 
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per event-kernel launch from the committed ncu
-# summary (profiles/k_apply_events_cfg4_d2m.md: three launches of the three-worker instance on a
-# d = 2e6 case), as a ratio to the bytes the launch's items must move: reads 1.000, writes 0.88
+# summary (profiles/k_apply_events_cfg4_d2m.md: two launches of the four-worker instance on a
+# d = 2e6 case), as a ratio to the bytes the launch's items must move: reads 1.000, writes 0.93
 # (the rest was still in L2 when the small launches ended). None once the kernel has changed
 # since the counters were taken.
-NCU_TRAFFIC_RATIO = 0.951
+NCU_TRAFFIC_RATIO = 0.973
 
 
 def parse_args():
