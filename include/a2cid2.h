@@ -279,7 +279,7 @@ void a2cid2_plan_destroy(a2cid2_plan_t* p);
  * back and applied, in order, inside the next communication item of that worker (or in a
  * gradient-only item at the end of the stream, or when max_ops_per_item is reached or the
  * gradient slot changes). With A2_SCHED_CHAIN items also take later events of workers they already
- * hold, and a third worker (see the flag). t_last[n] are the workers' times at the start
+ * hold, and further workers (see the flag). t_last[n] are the workers' times at the start
  * (NULL = zeros). max_ops_per_item <= 0 selects the default; max_workers_per_item is 2, 3 or 4
  * (<= 0: 4) and only matters with A2_SCHED_CHAIN. Validation and error codes as in
  * a2cid2_apply_events. */
