@@ -251,10 +251,11 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;
     }
+    for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l)  // before anything is launched
+        if (pk.launches[(size_t)l].workers > ((h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3))
+            return fail(h, A2_ESTATE, "this plan holds four-worker items, which the kernels of the current variant do not take");
     for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
         const LaunchRange& R = pk.launches[(size_t)l];
-        if (R.workers > ((h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3))
-            return fail(h, A2_ESTATE, "this plan holds four-worker items, which the kernels of the current variant do not take");
         a2::EventLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.items = d_items + R.item0;

@@ -278,3 +278,27 @@ def test_plan_graph_follows_a_change_of_variant():
     p.close()
     eng.close()
     assert all(np.array_equal(u, v) for u, v in zip(want, got))
+
+
+def test_a_plan_with_four_worker_items_is_refused_by_a_variant_whose_kernels_take_three():
+    """Plans are scheduled for the kernels of the variant they were made under; the no-momentum kernels take
+    three workers per item, so a four-worker plan must be refused there, before anything is launched."""
+    cfg = _small(n_events=600)
+    ev = W.config_events(cfg)
+    eng, _ = P.make_small(cfg)
+    p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)
+    assert max(len(p.sched.item(k).workers()) for k in range(p.sched.num_items)) == 4
+    before = eng.read_state()
+    eng.set_variant(B.A2_NO_MOMENTUM)
+    with pytest.raises(B.A2Error) as e:
+        p.run()
+    assert e.value.code == B.A2_ESTATE
+    assert all(np.array_equal(u, v) for u, v in zip(before, eng.read_state()))
+    # a plan made under the variant holds at most three workers per item and runs
+    q = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)
+    assert max(len(q.sched.item(k).workers()) for k in range(q.sched.num_items)) == 3
+    q.run()
+    eng.sync()
+    p.close()
+    q.close()
+    eng.close()
