@@ -228,6 +228,14 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
     }
 }
 
+// Most workers per item the kernels of the handle's storage type and variant take: four with fp32 rows and the
+// momentum buffer, three with bf16 rows or without x~.
+int32_t kernel_item_workers(const a2cid2* h) { return (h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3; }
+int32_t item_workers(const a2cid2* h) {
+    const int32_t cap = kernel_item_workers(h);
+    return h->item_workers < cap ? h->item_workers : cap;
+}
+
 // Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
 int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev, int64_t b0, int64_t b1,
                   cudaStream_t stream) {
@@ -252,7 +260,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         return A2_OK;
     }
     for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l)  // before anything is launched
-        if (pk.launches[(size_t)l].workers > ((h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3))
+        if (pk.launches[(size_t)l].workers > kernel_item_workers(h))
             return fail(h, A2_ESTATE, "this plan holds four-worker items, which the kernels of the current variant do not take");
     for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
         const LaunchRange& R = pk.launches[(size_t)l];
@@ -270,13 +278,6 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
     return A2_OK;
-}
-
-// Most workers per item the kernels of the handle's storage type and variant take: four with fp32 rows and the
-// momentum buffer, three with bf16 rows or without x~.
-int32_t item_workers(const a2cid2* h) {
-    const int32_t cap = (h->dtype == A2_F32 && h->variant != A2_NO_MOMENTUM) ? 4 : 3;
-    return h->item_workers < cap ? h->item_workers : cap;
 }
 
 constexpr int64_t kGraphMinLaunches = 4;
