@@ -265,7 +265,7 @@ def test_random_streams_property():
         return (n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32),
                 flags, cap, kw)
 
-    @settings(max_examples=150, deadline=None)
+    @settings(max_examples=400, deadline=None)
     @given(streams())
     def check(case):
         n, n_slots, times, wi, wj, sl, flags, cap, kw = case
