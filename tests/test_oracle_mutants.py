@@ -37,6 +37,13 @@ MUTANTS = {
                                   "a2o_plain_comm(xi, xj, d, alpha);\n                tl[i] = t;"),
     "plain_grad_touches_tilde": ("a2o_plain_grad(xi, g, d, gamma);", "a2o_plain_grad(xi, g, d, gamma); a2o_plain_grad(xti, g, d, gamma);"),
     "consensus_at_ignores_flow": ("mean += x - c * (x - xt);", "mean += x;"),
+    # the branch that follows Algorithm 1 as printed (message before the mixing line)
+    "printed_order_sign_of_mixing_on_j": ("xj[k] = (xj[k] - cj * dj) + alpha * m;", "xj[k] = (xj[k] + cj * dj) + alpha * m;"),
+    "printed_order_message_after_mixing": ("const double m = xi[k] - xj[k]; /* from the un-mixed buffers */",
+                                           "const double m = (xi[k] - ci * (xi[k] - xti[k])) - (xj[k] - cj * (xj[k] - xtj[k]));"),
+    "printed_order_swapped_coeffs": ("xi[k] = (xi[k] - ci * di) - alpha * m;\n                    xti[k] = (xti[k] + ci * di) - alpha_t * m;",
+                                     "xi[k] = (xi[k] - ci * di) - alpha_t * m;\n                    xti[k] = (xti[k] + ci * di) - alpha * m;"),
+    "printed_order_tilde_mixed_with_wrong_sign": ("xti[k] = (xti[k] + ci * di) - alpha_t * m;", "xti[k] = (xti[k] - ci * di) - alpha_t * m;"),
 }
 
 # pins that take the simulator class, and pins that use OracleSim directly
@@ -54,7 +61,13 @@ DETECTORS = [
     lambda: pins.test_hand_example(pins.OracleSim),
     lambda: pins.test_plain_dynamic_is_a_product_of_gossip_matrices(pins.OracleSim, 0.3),
     lambda: pins.test_plain_dynamic_is_the_full_one_without_drift(),
+    lambda: pins.test_algorithm1_ordering_against_series_exponential(pins.OracleSim, 4, 3, "ring"),
+    lambda: pins.test_hand_example_algorithm1_ordering(pins.OracleSim),
 ]
+
+# mistakes planted in the branch of Algorithm 1's printed ordering must be caught by the pins of that
+# branch, which do not consult the NumPy twin
+PRINTED_ORDER_DETECTORS = (13, 14)
 
 
 def _caught():
@@ -85,3 +98,5 @@ def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
     monkeypatch.setattr(sim_mod, "_lib", sim_mod.load(str(so)))
     caught = _caught()
     assert caught, f"no pin noticed the planted mistake '{name}'"
+    if name.startswith("printed_order_"):
+        assert set(caught) & set(PRINTED_ORDER_DETECTORS), caught

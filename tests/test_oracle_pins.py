@@ -301,6 +301,82 @@ def test_brute_force_matrix_exponential(Sim, n, d, graph):
     np.testing.assert_allclose(fxt, bxt, rtol=1e-10, atol=1e-11)
 
 
+# ---- Algorithm 1 as printed (variant 1): message formed before the mixing line ---------------
+def _algorithm1_lazy_reference(x0, xt0, G, ev, eta, alpha, at, gamma):
+    """Algorithm 1, worker by worker, in the order its two loops print the steps, with the matrix
+    exponential of exp((t - t_i) [[-eta, eta],[eta, -eta]]) summed from its Taylor series (no closed
+    form). Communication loop: the message x^i - x^j is formed first, from the stored rows; then each
+    of the two workers applies the exponential over its own elapsed time; then the jumps -alpha m /
+    -alpha~ m on worker i and, roles swapped (symmetric communications, Sec. 3.1), +alpha m / +alpha~ m
+    on worker j. Gradient loop: the exponential, then -gamma g on both buffers."""
+    X, Xt = np.array(x0, dtype=np.float64), np.array(xt0, dtype=np.float64)
+    tl = np.zeros(X.shape[0])
+    A = np.array([[-eta, eta], [eta, -eta]])
+
+    def flow(w, t):
+        E = _expm_taylor((t - tl[w]) * A)
+        X[w], Xt[w] = E[0, 0] * X[w] + E[0, 1] * Xt[w], E[1, 0] * X[w] + E[1, 1] * Xt[w]
+        tl[w] = t
+
+    for t, i, j, sl in zip(ev.times, ev.wi, ev.wj, ev.slot):
+        if j < 0:
+            flow(i, t)
+            X[i] -= gamma * G[sl]
+            Xt[i] -= gamma * G[sl]
+        else:
+            m = X[i] - X[j]  # before either worker is mixed
+            flow(i, t)
+            flow(j, t)
+            X[i] -= alpha * m
+            Xt[i] -= at * m
+            X[j] += alpha * m
+            Xt[j] += at * m
+    return X, Xt, tl
+
+
+@pytest.mark.parametrize("n,d,graph", [(2, 3, "ring"), (4, 3, "ring"), (5, 2, "complete")])
+@pytest.mark.parametrize("Sim", SIMS)
+def test_algorithm1_ordering_against_series_exponential(Sim, n, d, graph):
+    """Variant 1 against a lazy per-worker run written here from Algorithm 1's printed order, with a
+    Taylor-series matrix exponential; x~ starts away from x so that the very first mixing matters."""
+    r = np.random.default_rng(23)
+    x0, xt0, G = r.standard_normal((n, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    edges = W.make_edges(graph, n)
+    ev = W.poisson_events(n, edges, np.full(len(edges), 0.9), 150, seed=5)
+    eta, alpha, at, gamma = 0.55, 0.4, 1.7, 0.05
+    s = Sim(x0, eta, alpha, at, gamma, grads=G, xt0=xt0, variant=1)
+    s.apply(ev.times, ev.wi, ev.wj, ev.slot)
+    rx, rxt, rt = _algorithm1_lazy_reference(x0, xt0, G, ev, eta, alpha, at, gamma)
+    np.testing.assert_allclose(s.X, rx, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(s.Xt, rxt, rtol=1e-10, atol=1e-11)
+    assert np.array_equal(s.t, rt)
+    # and the ordering is not the one of Eq. (dynamic): the same stream under variant 0 ends elsewhere
+    s0 = Sim(x0, eta, alpha, at, gamma, grads=G, xt0=xt0, variant=0)
+    s0.apply(ev.times, ev.wi, ev.wj, ev.slot)
+    assert np.abs(s0.X - rx).max() > 1e-3
+
+
+@pytest.mark.parametrize("Sim", SIMS)
+def test_hand_example_algorithm1_ordering(Sim):
+    # n=2, d=1, eta = ln(2)/2, alpha = 1/2, alpha~ = 2; stored x = (4, 0), x~ = (0, 8), both at t = 0.
+    # One communication (0, 1) at t = 1: e = exp(-2 eta) = 1/2, c = (1 - e)/2 = 1/4 for both workers.
+    # Algorithm 1 as printed:
+    #   message first, from the stored rows:           m = 4 - 0 = 4
+    #   worker 0 mixed:  x - x~ =  4:  x = 4 - 1 = 3,  x~ = 0 + 1 = 1
+    #   worker 1 mixed:  x - x~ = -8:  x = 0 + 2 = 2,  x~ = 8 - 2 = 6
+    #   jumps:  x_0 = 3 - 4/2 = 1,  x~_0 = 1 - 2*4 = -7,  x_1 = 2 + 4/2 = 4,  x~_1 = 6 + 2*4 = 14
+    # (Eq. (dynamic)'s ordering would take m = 3 - 2 = 1 and end at x = (2.5, 2.5), x~ = (-1, 8).)
+    s = Sim(np.array([[4.0], [0.0]]), math.log(2.0) / 2.0, 0.5, 2.0, 0.0, xt0=np.array([[0.0], [8.0]]), variant=1)
+    s.apply(*_one([1.0], [0], [1], [-1]))
+    np.testing.assert_allclose(s.X[:, 0], [1.0, 4.0], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(s.Xt[:, 0], [-7.0, 14.0], rtol=0, atol=1e-14)
+    assert list(s.t) == [1.0, 1.0]
+    s0 = Sim(np.array([[4.0], [0.0]]), math.log(2.0) / 2.0, 0.5, 2.0, 0.0, xt0=np.array([[0.0], [8.0]]), variant=0)
+    s0.apply(*_one([1.0], [0], [1], [-1]))
+    np.testing.assert_allclose(s0.X[:, 0], [2.5, 2.5], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(s0.Xt[:, 0], [-1.0, 8.0], rtol=0, atol=1e-14)
+
+
 def test_consensus_at_common_time_matches_flushed_state_and_definition():
     """App. A: ||pi x||_F^2 with pi = I - 11^T/n, written out as a projection."""
     cfg = W.CONFIGS["cfg1"].scaled(d=6, n_events=200)
