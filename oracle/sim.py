@@ -115,13 +115,20 @@ class OracleSim:
         self.X, self.Xt = self.flushed(t_flush)
         self.t[:] = t_flush
 
-    def round_rows(self, workers):
-        """Model of bf16 *storage*: the rows of these workers are rounded to bfloat16, as happens
-        whenever an implementation that keeps its state in bf16 writes them back. The arithmetic
+    def round_rows(self, workers, fmt="bf16"):
+        """Model of reduced-precision *storage*: the rows of these workers are rounded to the storage
+        format (bfloat16, or IEEE binary32 with fmt="f32"; both to nearest even), as happens whenever
+        an implementation that keeps its state in that format writes them back. The arithmetic
         between two stores stays fp64."""
         w = np.unique(np.asarray(workers, dtype=np.int64))
-        self.X[w] = round_to_bf16(self.X[w])
-        self.Xt[w] = round_to_bf16(self.Xt[w])
+        if fmt == "bf16":
+            self.X[w] = round_to_bf16(self.X[w])
+            self.Xt[w] = round_to_bf16(self.Xt[w])
+        elif fmt == "f32":
+            self.X[w] = self.X[w].astype(np.float32).astype(np.float64)
+            self.Xt[w] = self.Xt[w].astype(np.float32).astype(np.float64)
+        else:
+            raise ValueError(fmt)
 
     def consensus(self, t_eval=None):
         if t_eval is None:

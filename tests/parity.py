@@ -11,16 +11,22 @@ bf16 storage -- bar 2e-2, applied norm-wise against the plain fp64 run:
   Element-wise the bar is below what the storage format can hold: one bf16 store costs up to
   2^-8 = 3.9e-3 of an element, x~ integrates alpha~ times the rounding errors of x at every
   averaging, and an ideal bf16-storage run (fp64 arithmetic, exact round-to-nearest-even at
-  every store) already sits at 3-6e-2 in the element-wise metric after a few hundred events.
-  So that a wrong element cannot hide inside a norm, every element is still compared
-    * with the fp64 run *with the storage modelled* (the checker's rows rounded to bf16 wherever
-      the engine writes them back, i.e. after every item): bound 5e-2 (a few bf16 ulps: the two
-      runs differ where fp32 and fp64 arithmetic round a store to different neighbours, and
-      those one-ulp differences are integrated like any other perturbation);
-    * with the plain fp64 run: bound 0.3 (rows of >= 256 columns, like the norm: on a row of one or two
-      columns the floor of the metric is the element itself, and what the storage format loses over a few
-      hundred events is then measured against a value that has shrunk towards zero -- an ideal
-      bf16-storage run of 2 workers x 1 column is already 0.38 away from the fp64 run).
+  every store) already sits at 3-6e-2 in the element-wise metric after a few hundred events
+  (tests/test_oracle_pins.py::test_what_bf16_storage_alone_costs).
+  So that a wrong element cannot hide inside a norm, every element is compared with the fp64 run
+  *with the storage modelled* (the checker's rows rounded to bf16 at the engine's documented storage
+  points, i.e. when an item's rows are written back), in bf16 units in the last place of the
+  element's own magnitude:
+      |gpu_k - ref_k| / ulp_bf16(max(|ref_k|, rms(ref row))),   ulp_bf16(v) = 2^(floor(log2 v) - 7).
+  Two correct implementations that differ only in the precision of the arithmetic between two stores
+  (fp32 on the GPU, fp64 in the checker) round a store to different neighbours once in a few thousand
+  stores, and such one-ulp differences are then carried along like any perturbation. The bound is what
+  tests/test_parity_bounds_cpu.py measures between two such implementations on the CPU (fp64 against
+  NumPy float32 arithmetic: at most 4 ulps and 98 % of the elements identical after 10,000 events on
+  2e5 elements, the tail falling tenfold per ulp), extended along that tail to the 3e9 elements of the
+  full-size runs: BF16_ULP_BOUND = 8 ulps on any element, at least BF16_MIN_EXACT = 95 % of the
+  elements bit-equal and BF16_MIN_WITHIN_1 = 99.5 % within one ulp (the two fractions on rows of
+  >= 256 columns).
 """
 from __future__ import annotations
 
@@ -32,8 +38,9 @@ from paper_2306_08289_b200 import binding as B
 from paper_2306_08289_b200 import workload as W
 
 TOL = {"f32": 1e-5, "bf16": 2e-2}
-BF16_ELEM_STORED_BOUND = 5e-2
-BF16_ELEM_PLAIN_BOUND = 0.3
+BF16_ULP_BOUND = 8.0
+BF16_MIN_EXACT = 0.95
+BF16_MIN_WITHIN_1 = 0.995
 BF16_NORM_MIN_COLS = 256
 TILE_COLS = {"f32": 256 * 8, "bf16": 256 * 8}  # columns per work unit of the event kernel
 
@@ -52,6 +59,27 @@ def row_norm_err(gpu, ref):
     num = np.sqrt(((gpu - ref) ** 2).sum(axis=1))
     den = np.maximum(np.sqrt((ref * ref).sum(axis=1)), 1e-300)
     return float((num / den).max()) if ref.size else 0.0
+
+
+def ulp_bf16(v):
+    """Spacing of bfloat16 (8 significant bits) at magnitude v > 0."""
+    return np.exp2(np.floor(np.log2(v)) - 7.0)
+
+
+def bf16_ulp_distance(gpu, ref):
+    """Per element: |gpu - ref| in bf16 ulps of max(|ref|, rms of ref's row)."""
+    ref = np.asarray(ref, dtype=np.float64)
+    gpu = np.asarray(gpu, dtype=np.float64)
+    rms = np.sqrt((ref * ref).mean(axis=1, keepdims=True))
+    mag = np.maximum(np.abs(ref), np.maximum(rms, 1e-300))
+    return np.abs(gpu - ref) / ulp_bf16(mag)
+
+
+def ulp_histogram(u):
+    """Counts of elements off by exactly 0, at most 1, at most 2, and more than 2 ulps; and the maximum."""
+    u = np.asarray(u)
+    return {"n": int(u.size), "eq": int((u == 0).sum()), "le1": int((u <= 1).sum()), "le2": int((u <= 2).sum()),
+            "gt2": int((u > 2).sum()), "max": float(u.max()) if u.size else 0.0}
 
 
 def widen(a, storage):
@@ -109,12 +137,18 @@ class Checker:
         if st is None:
             assert out["elem_plain"] <= TOL["f32"], f"parity {where}: {out}"
         else:
-            out["elem_stored"] = max(rel_err(x, sel(st.X)), rel_err(xt, sel(st.Xt)))
             out["norm_plain"] = max(row_norm_err(x, sel(pl.X)), row_norm_err(xt, sel(pl.Xt)))
+            u = np.concatenate([bf16_ulp_distance(x, sel(st.X)).ravel(), bf16_ulp_distance(xt, sel(st.Xt)).ravel()])
+            h = ulp_histogram(u)
+            out["ulps_stored_max"] = h["max"]
+            out["not_exact"] = 1.0 - h["eq"] / max(1, h["n"])
+            out["beyond_1_ulp"] = 1.0 - h["le1"] / max(1, h["n"])
+            self.last_histogram = h
+            assert h["max"] <= BF16_ULP_BOUND, f"parity {where}: {out}"
             if x.shape[1] >= BF16_NORM_MIN_COLS:
                 assert out["norm_plain"] <= TOL["bf16"], f"parity {where}: {out}"
-                assert out["elem_plain"] <= BF16_ELEM_PLAIN_BOUND, f"parity {where}: {out}"
-            assert out["elem_stored"] <= BF16_ELEM_STORED_BOUND, f"parity {where}: {out}"
+                assert out["not_exact"] <= 1.0 - BF16_MIN_EXACT, f"parity {where}: {out}"
+                assert out["beyond_1_ulp"] <= 1.0 - BF16_MIN_WITHIN_1, f"parity {where}: {out}"
         return out
 
 
