@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--config", default="cfg4", choices=sorted(W.CONFIGS))
     ap.add_argument("--d", type=int, default=None, help="override the row width (for quick checks)")
     ap.add_argument("--events-per-step", type=int, default=500)
+    ap.add_argument("--grad-pool", type=int, default=None,
+                    help="gradient rows per worker, used round-robin by its gradient events (default: the workload's own)")
     ap.add_argument("--no-fuse", action="store_true", help="one event per item (no gradient fusion)")
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -214,6 +216,10 @@ def main():
     cfg = W.CONFIGS[args.config]
     if args.d is not None:
         cfg = cfg.scaled(d=args.d, name=f"{cfg.name}-d{args.d}")
+    if args.grad_pool is not None:
+        from dataclasses import replace
+
+        cfg = replace(cfg, grad_pool=int(args.grad_pool))
     if args.impl == "reference":
         # rank 0 alone times the CPU checker; the other ranks have nothing to do and no group is formed
         if int(os.environ.get("RANK", "0")) == 0:

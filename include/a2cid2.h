@@ -71,7 +71,7 @@ enum {
                               With bf16 storage the tile is kept in fp32 and rounded once, at the
                               end of the call. The schedule then has a single batch holding every
                               event in stream order. Overrides the other flags.                */
-    A2_SCHED_CHAIN = 4u /* A2_SCHED_FUSE, and further: (1) an event whose workers' latest events are
+    A2_SCHED_CHAIN = 4u, /* A2_SCHED_FUSE, and further: (1) an event whose workers' latest events are
                            all in one item is appended to that item, whose rows then serve one
                            more event without crossing HBM again; (2) a communication between a
                            worker that is free earlier and one whose latest events sit in an item
@@ -80,6 +80,16 @@ enum {
                            order is kept and the arithmetic per event is unchanged; batches get
                            fewer and items longer (up to four workers with fp32 rows and the
                            momentum buffer, three otherwise)                                    */
+    A2_SCHED_ROW_PER_OP = 8u /* with A2_SCHED_FUSE or A2_SCHED_CHAIN: the gradient events an item applies to
+                           one worker may each name their own gradient row -- the paper's stochastic
+                           gradients are fresh draws at every step (Sec. 3.2; Algorithm 1 computes g_i anew
+                           in every iteration of its first loop). The item records the worker's first row
+                           (slot_a .. slot_d) and, per gradient operation, the row to fetch next
+                           (a2cid2_sched_op_reloads); the event kernel fetches it right after the operation
+                           has used the previous one. Without the flag a change of row ends the item, so
+                           that one row per worker and item suffices. The engine sets the flag by itself
+                           wherever its kernels can follow it (fp32 rows) and clears it elsewhere (bf16
+                           rows, whose kernels keep packed rows in registers for the whole item).        */
 };
 
 /* Kinds of elementary operation inside an item. */
@@ -111,10 +121,24 @@ enum {
                               rows. A2_SCHED_RESIDENT is not available (A2_EINVAL).               */
 };
 
+/* How a whole event stream (a2cid2_apply_events, a whole a2cid2_plan_run) is put on the GPU. */
+enum {
+    A2_LAUNCH_AUTO = 0,          /* the library chooses (column slices)                                  */
+    A2_LAUNCH_PER_BATCH = 1,     /* one kernel launch per batch of worker-disjoint items; the CTAs of a launch
+                                    share out its (item, column tile) units round robin                      */
+    A2_LAUNCH_COLUMN_SLICES = 2  /* launches that hold the items of several consecutive batches: every CTA owns a
+                                    contiguous range of columns and applies all items, in schedule order, to
+                                    that range alone. Legal because every operation of the method is element-wise
+                                    over the parameter dimension (Eq. (dynamic) couples workers, never columns):
+                                    what an item needs from an earlier one was written by the same thread. No
+                                    CTA ever waits for another. The results are the same bits in all modes.  */
+};
+
 /* One item of a batch: all the work done on one worker (b = c = d = -1) or on two to four workers. */
 typedef struct a2cid2_item_info {
     int32_t a, b;           /* worker rows; b = -1 for a gradient-only item                    */
-    int32_t slot_a, slot_b; /* gradient rows read for worker a / b, or -1                       */
+    int32_t slot_a, slot_b; /* gradient row read up front for worker a / b (that of its first gradient
+                               operation in the item), or -1                                    */
     int64_t first_op;       /* index of the item's first elementary operation                   */
     int32_t n_ops;          /* operations applied, in order, while the rows sit in registers    */
     int32_t batch;          /* batch (dependency level) the item belongs to                     */
@@ -129,7 +153,8 @@ typedef struct a2cid2_stats {
     int64_t n_batches;  /* dependency levels                                                    */
     int64_t n_launches; /* event-kernel launches (a batch is split if it exceeds a launch's caps) */
     int64_t n_items;
-    int64_t bytes_moved;       /* rows read + rows written by the items, times d, times element size */
+    int64_t bytes_moved;       /* rows read + rows written by the items (every gradient row fetched counts,
+                                  also one fetched in the middle of an item), times d, times element size */
     int64_t bytes_one_by_one;  /* the same stream applied one event per item: comm 8 rows, gradient 5
                                   (4 and 3 under A2_NO_MOMENTUM)                                   */
     int64_t descriptor_bytes;  /* host-to-device bytes of the descriptors                        */
@@ -150,6 +175,10 @@ int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_t
 /* Select A2_MSG_AFTER_MIX (default), A2_MSG_BEFORE_MIX or A2_NO_MOMENTUM for later events.
  * A2_ESTATE when leaving A2_NO_MOMENTUM while no x~ buffer is bound. */
 int a2cid2_set_variant(a2cid2_t* h, int32_t variant);
+
+/* Select how whole streams are launched (A2_LAUNCH_*; default A2_LAUNCH_AUTO). A range of a plan's batches
+ * (a2cid2_plan_run with a first batch or a count) is always run with one launch per batch. */
+int a2cid2_set_launch_mode(a2cid2_t* h, int32_t mode);
 
 /* Lend the device buffers: x and x_tilde are [n, row_pitch_elems], grads is
  * [n_grad_slots, row_pitch_elems] (may be NULL with n_grad_slots = 0 if no gradient event is
@@ -300,6 +329,11 @@ int a2cid2_sched_item(const a2cid2_sched_t* s, int64_t item, a2cid2_item_info* o
 /* Operations [first_op, first_op + n_ops): the index of the event each one applies (into the
  * arrays given to a2cid2_sched_create) and its kind (A2_OP_*). Either output may be NULL. */
 int a2cid2_sched_ops(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, int64_t* event_index, int32_t* kind);
+
+/* For gradient operations [first_op, first_op + n_ops): the gradient row that is fetched into the worker's
+ * gradient registers after the operation (A2_SCHED_ROW_PER_OP), or -1; -1 for every other operation. The row
+ * a gradient operation itself uses is the one its event names. */
+int a2cid2_sched_op_reloads(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, int32_t* reload);
 
 /* Workers' times after the whole schedule has run. */
 int a2cid2_sched_t_final(const a2cid2_sched_t* s, double* t_out);

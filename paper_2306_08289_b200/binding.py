@@ -21,9 +21,11 @@ A2_F32, A2_BF16 = 0, 1
 A2_SCHED_FUSE = 1
 A2_SCHED_RESIDENT = 2
 A2_SCHED_CHAIN = 4
+A2_SCHED_ROW_PER_OP = 8
 A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A, A2_OP_GRAD_C, A2_OP_COMM_AC, A2_OP_COMM_BC = 0, 1, 2, 3, 4, 5, 6
 A2_OP_GRAD_D, A2_OP_COMM_AD, A2_OP_COMM_BD, A2_OP_COMM_CD = 7, 8, 9, 10
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX, A2_NO_MOMENTUM = 0, 1, 2
+A2_LAUNCH_AUTO, A2_LAUNCH_PER_BATCH, A2_LAUNCH_COLUMN_SLICES = 0, 1, 2
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
                A2_ECUDA: "A2_ECUDA", A2_ESTATE: "A2_ESTATE"}
@@ -63,6 +65,7 @@ _vp = C.c_void_p
 SIGNATURES = {
     "a2cid2_create": (C.c_int, [C.c_int32, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int32, C.POINTER(_vp)]),
     "a2cid2_set_variant": (C.c_int, [_vp, C.c_int32]),
+    "a2cid2_set_launch_mode": (C.c_int, [_vp, C.c_int32]),
     "a2cid2_bind": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp]),
     "a2cid2_write_state": (C.c_int, [_vp, _vp, _vp, _dp]),
     "a2cid2_write_grads": (C.c_int, [_vp, C.c_int32, C.c_int32, _vp]),
@@ -88,6 +91,7 @@ SIGNATURES = {
     "a2cid2_sched_batch_items": (C.c_int, [_vp, C.c_int64, _lp, _lp]),
     "a2cid2_sched_item": (C.c_int, [_vp, C.c_int64, C.POINTER(ItemInfo)]),
     "a2cid2_sched_ops": (C.c_int, [_vp, C.c_int64, C.c_int64, _lp, _ip]),
+    "a2cid2_sched_op_reloads": (C.c_int, [_vp, C.c_int64, C.c_int64, _ip]),
     "a2cid2_sched_t_final": (C.c_int, [_vp, _dp]),
     "a2cid2_sched_stats": (C.c_int, [_vp, C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.POINTER(Stats)]),
     "a2cid2_sched_destroy": (None, [_vp]),
@@ -212,6 +216,12 @@ class Schedule:
         _check(lib().a2cid2_sched_ops(self._h, first_op, n_ops, _ptr(ev, _lp), _ptr(kind, _ip)))
         return ev, kind
 
+    def op_reloads(self, first_op, n_ops):
+        """Per operation: the gradient row fetched into the worker's registers after it, or -1."""
+        out = np.empty(n_ops, dtype=np.int32)
+        _check(lib().a2cid2_sched_op_reloads(self._h, first_op, n_ops, _ptr(out, _ip)))
+        return out
+
     def batch_events(self, b):
         """Event indices applied by batch b, item by item, in the order they are applied."""
         first, cnt = self.batch_items(b)
@@ -315,6 +325,9 @@ class Engine:
     # -- state ---------------------------------------------------------------------------------
     def set_variant(self, variant):
         _check(lib().a2cid2_set_variant(self._h, variant), self._h)
+
+    def set_launch_mode(self, mode):
+        _check(lib().a2cid2_set_launch_mode(self._h, mode), self._h)
 
     def write_state(self, x, x_tilde=None, t=None):
         x = np.ascontiguousarray(x, dtype=self.np_dtype)

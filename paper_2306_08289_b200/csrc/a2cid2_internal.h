@@ -20,6 +20,9 @@ struct SchedOp {
     double t;         // event time
     double t_prev_a;  // time the operation's first (or only) worker was last updated before it
     double t_prev_b;  // same for the second worker of a communication
+    int32_t reload = -1;  // gradient operations: the row to load into the worker's gradient registers once this
+                          // operation has used them (the row of the worker's next gradient operation in the item,
+                          // when it differs), or -1
 };
 
 constexpr int kMaxItemWorkers = 4;
@@ -83,7 +86,7 @@ struct DevItem {
 
 struct DevOp {
     int32_t kind;
-    int32_t pad;
+    int32_t reload;   // gradient row to fetch into the worker's gradient registers after this operation, or -1
     double t;         // event time
     double t_prev_a;  // last-event time, before this op, of its first (or only) worker
     double t_prev_b;  // of the second worker of a communication
@@ -108,6 +111,8 @@ struct EventLaunch {
     int32_t variant;
     int32_t dtype;
     int32_t max_workers;  // most workers any item of the launch holds (2, 3 or 4): selects the kernel instance
+    int32_t op_base = 0;  // index, in the plan, of the launch's first operation
+    bool slice = false;   // column-slice launch: the items may span several batches, each CTA owns a range of columns
 };
 
 struct DeviceInfo {

@@ -55,6 +55,7 @@ struct a2cid2 {
     int32_t dtype = A2_F32;
     int32_t variant = A2_MSG_AFTER_MIX;
     int32_t item_workers = a2::kMaxItemWorkers;  // most workers A2_SCHED_CHAIN puts into one item (before the kernels' limits)
+    int32_t launch_mode = A2_LAUNCH_AUTO;
     // borrowed buffers
     void* x = nullptr;
     void* xt = nullptr;
@@ -87,6 +88,7 @@ struct Packed {
     // batched mode
     std::vector<LaunchRange> launches;
     std::vector<int64_t> batch_launch_first;  // launches of batch b: [first[b], first[b+1])
+    std::vector<LaunchRange> slice_launches;  // the whole schedule as column-slice launches (items of several batches each)
     // resident mode
     bool resident = false;
     int32_t cache_rows = 0;
@@ -169,6 +171,25 @@ void make_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches, st
     batch_first[(size_t)nb] = (int64_t)launches.size();
 }
 
+// The whole schedule cut into launches at the per-launch caps only: in a column-slice launch every CTA walks the
+// items in schedule order over columns of its own, so batch boundaries need no launch boundary.
+void make_slice_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches) {
+    const int64_t n = (int64_t)s.items.size();
+    int64_t i = 0;
+    while (i < n) {
+        LaunchRange L{i, i, s.items[(size_t)i].first_op, s.items[(size_t)i].first_op, 2};
+        while (L.item1 < n && (L.item1 - L.item0) < a2::kMaxItemsPerLaunch &&
+               (L.op1 - L.op0) + s.items[(size_t)L.item1].n_ops <= a2::kMaxOpsPerLaunch) {
+            const a2::SchedItem& si = s.items[(size_t)L.item1];
+            L.op1 += si.n_ops;
+            L.workers = std::max(L.workers, si.d >= 0 ? 4 : (si.c >= 0 ? 3 : 2));
+            L.item1 += 1;
+        }
+        launches.push_back(L);
+        i = L.item1;
+    }
+}
+
 size_t align16(size_t v) { return (v + 15) & ~size_t(15); }
 
 // Decide how the schedule is launched and lay its descriptors out. Resident schedules need the
@@ -181,6 +202,7 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
         return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT is not available for the A2_NO_MOMENTUM variant");
     if (!pk.resident) {
         make_launches(s, pk.launches, pk.batch_launch_first);
+        make_slice_launches(s, pk.slice_launches);
     } else {
         pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
         if (pk.cache_rows <= 0)
@@ -210,7 +232,7 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
             for (int64_t k = L.item0; k < L.item1; ++k) {
                 const a2::SchedItem& it = s.items[(size_t)k];
                 di[k] = DevItem{it.a, it.b, it.c, it.d, it.slot_a, it.slot_b, it.slot_c, it.slot_d,
-                                (int32_t)(it.first_op - L.op0), it.n_ops};
+                                (int32_t)it.first_op, it.n_ops};  // counted from the plan's first operation
             }
     } else {
         for (size_t k = 0; k < s.items.size(); ++k) {  // one operation per item; slot_b carries the cache index
@@ -224,7 +246,7 @@ void write_descriptors(const a2cid2_sched& s, const Packed& pk, void* dst) {
     }
     for (size_t o = 0; o < s.ops.size(); ++o) {
         const a2::SchedOp& op = s.ops[o];
-        dop[o] = DevOp{op.kind, 0, op.t, op.t_prev_a, op.t_prev_b};
+        dop[o] = DevOp{op.kind, op.reload, op.t, op.t_prev_a, op.t_prev_b};
     }
 }
 
@@ -234,6 +256,21 @@ int32_t kernel_item_workers(const a2cid2* h) { return (h->dtype == A2_F32 && h->
 int32_t item_workers(const a2cid2* h) {
     const int32_t cap = kernel_item_workers(h);
     return h->item_workers < cap ? h->item_workers : cap;
+}
+
+// Scheduling flags as the engine uses them: an item may change a worker's gradient row between two of its
+// gradient operations exactly where the event kernels fetch rows operation by operation (fp32 rows).
+uint32_t engine_flags(const a2cid2* h, uint32_t flags) {
+    if (h->dtype == A2_F32) return flags | A2_SCHED_ROW_PER_OP;
+    return flags & ~uint32_t(A2_SCHED_ROW_PER_OP);
+}
+
+// Column-slice launches serve a schedule that is run whole (any batch boundary inside a launch is then harmless);
+// a range of batches is run with one launch per batch.
+bool uses_slices(const a2cid2* h, const a2cid2_sched& s, int64_t b0, int64_t b1) {
+    const int64_t nb = (int64_t)s.batch_first.size() - 1;
+    if ((s.flags & A2_SCHED_RESIDENT) || b0 != 0 || b1 != nb) return false;
+    return h->launch_mode != A2_LAUNCH_PER_BATCH;
 }
 
 // Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
@@ -259,11 +296,15 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;
     }
-    for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l)  // before anything is launched
-        if (pk.launches[(size_t)l].workers > kernel_item_workers(h))
+    const std::vector<LaunchRange>& list = uses_slices(h, s, b0, b1) ? pk.slice_launches : pk.launches;
+    const bool slices = &list == &pk.slice_launches;
+    const int64_t l0 = slices ? 0 : pk.batch_launch_first[(size_t)b0];
+    const int64_t l1 = slices ? (int64_t)list.size() : pk.batch_launch_first[(size_t)b1];
+    for (int64_t l = l0; l < l1; ++l)  // before anything is launched
+        if (list[(size_t)l].workers > kernel_item_workers(h))
             return fail(h, A2_ESTATE, "this plan holds four-worker items, which the kernels of the current variant do not take");
-    for (int64_t l = pk.batch_launch_first[(size_t)b0]; l < pk.batch_launch_first[(size_t)b1]; ++l) {
-        const LaunchRange& R = pk.launches[(size_t)l];
+    for (int64_t l = l0; l < l1; ++l) {
+        const LaunchRange& R = list[(size_t)l];
         a2::EventLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.items = d_items + R.item0;
@@ -274,6 +315,8 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.alpha = (float)h->alpha; L.alpha_tilde = (float)h->alpha_tilde; L.gamma = (float)h->gamma;
         L.variant = h->variant; L.dtype = h->dtype;
         L.max_workers = R.workers;
+        L.op_base = (int32_t)R.op0;
+        L.slice = slices;
         const int rc = a2::launch_events(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
@@ -306,6 +349,12 @@ int ensure_plan_graph(a2cid2* h, a2cid2_plan* p) {
     return A2_OK;
 }
 
+// Launches a whole run of the plan takes under the handle's launch mode.
+int64_t whole_run_launches(const a2cid2* h, const a2cid2_plan* p) {
+    const int64_t nb = (int64_t)p->sched->batch_first.size() - 1;
+    return uses_slices(h, *p->sched, 0, nb) ? (int64_t)p->pk.slice_launches.size() : (int64_t)p->pk.launches.size();
+}
+
 int run_plan_graph(a2cid2* h, a2cid2_plan* p) {
     const int rc = ensure_plan_graph(h, p);
     if (rc != A2_OK) return rc;
@@ -321,7 +370,8 @@ void fill_stats(const a2cid2* h, const a2cid2_sched& s, const Packed& pk, int64_
         st->n_launches = b1 > b0 ? 2 : 0;
         st->bytes_moved = b1 > b0 ? ((int64_t)4 * h->n + (int64_t)pk.g_rows.size()) * h->d * eb : 0;
     } else {
-        st->n_launches = pk.batch_launch_first[(size_t)b1] - pk.batch_launch_first[(size_t)b0];
+        st->n_launches = uses_slices(h, s, b0, b1) ? (int64_t)pk.slice_launches.size()
+                                                   : pk.batch_launch_first[(size_t)b1] - pk.batch_launch_first[(size_t)b0];
     }
 }
 
@@ -390,6 +440,15 @@ int a2cid2_set_variant(a2cid2_t* h, int32_t variant) {
         return fail(h, A2_ESTATE, "this variant needs an x_tilde buffer and none is bound");
     h->variant = variant;
     h->bind_epoch += 1;
+    return A2_OK;
+}
+
+int a2cid2_set_launch_mode(a2cid2_t* h, int32_t mode) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (mode != A2_LAUNCH_AUTO && mode != A2_LAUNCH_PER_BATCH && mode != A2_LAUNCH_COLUMN_SLICES)
+        return fail(h, A2_EINVAL, "unknown launch mode");
+    h->launch_mode = mode;
+    h->bind_epoch += 1;  // recorded plan graphs hold the launches of the previous mode
     return A2_OK;
 }
 
@@ -533,7 +592,7 @@ int a2cid2_apply_events(a2cid2_t* h, int64_t n_events, const double* times, cons
     const double t0 = now_ms();
     a2cid2_sched* s = nullptr;
     std::string err;
-    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, flags, 0, item_workers(h),
+    rc = a2::build_schedule(h->n, h->n_slots, h->t.data(), n_events, times, wi, wj, grad_slot, engine_flags(h, flags), 0, item_workers(h),
                             &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     return submit_schedule(h, s, stats, t0);
@@ -652,8 +711,8 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
     *out = nullptr;
     a2cid2_sched* s = nullptr;
     std::string err;
-    rc = a2::build_schedule(h->n, h->n_slots, t_start ? t_start : h->t.data(), n_events, times, wi, wj, grad_slot, flags,
-                            0, item_workers(h), &s, err);
+    rc = a2::build_schedule(h->n, h->n_slots, t_start ? t_start : h->t.data(), n_events, times, wi, wj, grad_slot,
+                            engine_flags(h, flags), 0, item_workers(h), &s, err);
     if (rc != A2_OK) return fail(h, rc, err);
     a2cid2_plan* p = new (std::nothrow) a2cid2_plan();
     if (!p) { a2cid2_sched_destroy(s); return fail(h, A2_ENOMEM, "out of host memory"); }
@@ -677,7 +736,7 @@ int a2cid2_plan_create(a2cid2_t* h, const double* t_start, int64_t n_events, con
             return fail_cuda(h, e, "plan descriptor upload");
         }
     }
-    if (!p->pk.resident && (int64_t)p->pk.launches.size() >= kGraphMinLaunches) {
+    if (!p->pk.resident && whole_run_launches(h, p) >= kGraphMinLaunches) {
         rc = ensure_plan_graph(h, p);  // recorded now, so that running the plan is a single submission
         if (rc != A2_OK) {
             if (p->d_desc) cudaFree(p->d_desc);
@@ -709,7 +768,7 @@ int a2cid2_plan_run(a2cid2_t* h, a2cid2_plan_t* p, int64_t first_batch, int64_t 
         // batch. The graph was recorded on a private stream when the plan was made and is recorded again only if
         // the bound buffers, the stream or the variant have changed since.
         const bool whole = first_batch == 0 && b1 == nb;
-        if (whole && !p->pk.resident && (int64_t)p->pk.launches.size() >= kGraphMinLaunches) {
+        if (whole && !p->pk.resident && whole_run_launches(h, p) >= kGraphMinLaunches) {
             rc = run_plan_graph(h, p);
         } else {
             rc = queue_batches(h, *p->sched, p->pk, p->d_desc, first_batch, b1, h->stream);
@@ -780,6 +839,13 @@ int a2cid2_sched_ops(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, i
         if (event_index) event_index[k] = s->ops[(size_t)(first_op + k)].event;
         if (kind) kind[k] = s->ops[(size_t)(first_op + k)].kind;
     }
+    return A2_OK;
+}
+
+int a2cid2_sched_op_reloads(const a2cid2_sched_t* s, int64_t first_op, int64_t n_ops, int32_t* reload) {
+    if (!s || !reload) return fail(nullptr, A2_EINVAL, "NULL argument");
+    if (first_op < 0 || n_ops < 0 || first_op + n_ops > (int64_t)s->ops.size()) return fail(nullptr, A2_ERANGE, "op range out of bounds");
+    for (int64_t k = 0; k < n_ops; ++k) reload[k] = s->ops[(size_t)(first_op + k)].reload;
     return A2_OK;
 }
 

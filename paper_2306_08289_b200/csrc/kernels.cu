@@ -324,11 +324,55 @@ struct EventArgs {
     double eta;
     float alpha, alpha_tilde, gamma;
     int msg_before_mix;
+    int op_base;      // index, in the plan, of the launch's first operation (DevItem::op_first counts from the plan's)
+    int slice_vec;    // column-slice launches: vectors of a row owned by one CTA (a multiple of 4); else 0
+};
+
+// How a launch walks its (item, column tile) units.
+//   round robin (SLICE = false)  one launch per batch of worker-disjoint items; unit u = (tile u / n_items, item
+//       skewed by the tile index), CTA b takes units b, b + grid, ...: at any moment all CTAs stream through the
+//       same few rows.
+//   column slices (SLICE = true)  the launch's items may come from SEVERAL consecutive batches. CTA b owns the
+//       vectors [b * slice_vec, (b + 1) * slice_vec) of every row and walks ALL items, in order, over that range
+//       alone, the same thread always on the same columns. Every operation of the method is element-wise over
+//       the parameter dimension (Eq. (dynamic) couples workers, never columns), so what an item needs from an
+//       earlier item was written by the same thread: no grid-wide order is needed, hence no flag, no wait and
+//       no launch boundary between batches. Every CTA does the same work, whatever the items cost.
+template <bool SLICE, int TILE_VEC>
+struct UnitWalk {
+    long long v_lo, v_end;  // vectors of a row this CTA may touch
+    int my_tiles, n_it;
+    long long first, step, end;
+    __device__ __forceinline__ UnitWalk(const EventArgs& p) {
+        n_it = p.n_items;
+        if (SLICE) {
+            v_lo = (long long)blockIdx.x * p.slice_vec;
+            v_end = v_lo + p.slice_vec < p.n_vec ? v_lo + p.slice_vec : p.n_vec;
+            my_tiles = v_end > v_lo ? (int)((v_end - v_lo + TILE_VEC - 1) / TILE_VEC) : 0;
+            first = 0; step = 1; end = (long long)n_it * my_tiles;
+        } else {
+            v_lo = 0; v_end = p.n_vec; my_tiles = p.n_tiles;
+            first = blockIdx.x; step = gridDim.x; end = (long long)n_it * p.n_tiles;
+        }
+    }
+    // unit -> item index and the first vector of the unit's tile
+    __device__ __forceinline__ void map(long long unit, int& item_idx, long long& tile_v0) const {
+        if (SLICE) {
+            item_idx = (int)(unit / my_tiles);
+            tile_v0 = v_lo + (unit % my_tiles) * (long long)TILE_VEC;
+        } else {
+            const int rem = (int)(unit % n_it);
+            const long long tile = unit / n_it;
+            const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+            item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
+            tile_v0 = tile * (long long)TILE_VEC;
+        }
+    }
 };
 
 // KW = 2, 3 or 4: workers an item may hold (items of more than two workers come from A2_SCHED_CHAIN schedules).
 // THREADS: threads per CTA (the four-worker instance trades threads for registers).
-template <typename T, int BYTES, int UNROLL, int KW, int THREADS = kEventThreads>
+template <typename T, int BYTES, int UNROLL, int KW, int THREADS = kEventThreads, bool SLICE = false>
 __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
@@ -336,11 +380,13 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     __shared__ float s_ca[kMaxOpsPerLaunch];
     __shared__ float s_cb[kMaxOpsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    __shared__ int s_reload[kMaxOpsPerLaunch];  // gradient row to fetch after a gradient operation, or -1
 
     for (int i = threadIdx.x; i < p.n_items; i += THREADS) s_items[i] = p.items[i];
     for (int o = threadIdx.x; o < p.n_ops; o += THREADS) {
         const DevOp op = p.ops[o];
         s_kind[o] = (unsigned char)op.kind;
+        s_reload[o] = op.reload;
         const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC ||
                           op.kind == A2_OP_COMM_AD || op.kind == A2_OP_COMM_BD || op.kind == A2_OP_COMM_CD;
         s_ca[o] = (float)mix_coeff(p.eta, op.t - op.t_prev_a);  // the operation's first (or only) worker
@@ -352,7 +398,6 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     T* const Xt = static_cast<T*>(p.xt);
     const T* const G = static_cast<const T*>(p.g);
     const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
-    const long long n_units = (long long)p.n_items * p.n_tiles;
 
     // unit -> (tile = unit / n_items, item = (unit % n_items + tile) % n_items). The skew by the tile index
     // makes every CTA walk through ALL items of the batch: without it a CTA whose stride shares a factor with
@@ -365,6 +410,8 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     // so it keeps them.
     // (The three-worker instance issues more per byte and gains 3 % from leaving them out: 6.18 -> 6.38 TB/s.)
     constexpr bool kRecompute = sizeof(T) == 4 && KW == 2;
+    const UnitWalk<SLICE, THREADS * UNROLL> walk(p);
+    const long long v_end = walk.v_end;
     const int n_it = p.n_items;
     int rem = (int)(blockIdx.x % (unsigned)n_it);
     long long tile = blockIdx.x / (unsigned)n_it;
@@ -372,22 +419,24 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     const int step_rem = (int)(gridDim.x % (unsigned)n_it);
     const long long step_tile = gridDim.x / (unsigned)n_it;
     const int step_skew = (int)((unsigned long long)step_tile % (unsigned)n_it);
-    for (long long unit = blockIdx.x; unit < n_units;
-         unit += gridDim.x, rem += step_rem, tile += step_tile, skew += step_skew) {
-        if (kRecompute) {
-            rem = (int)(unit % n_it);
-            tile = unit / n_it;
-            skew = (int)((unsigned)tile % (unsigned)n_it);
+    for (long long unit = walk.first; unit < walk.end;
+         unit += walk.step, rem += step_rem, tile += step_tile, skew += step_skew) {
+        int item_idx;
+        long long tile_v0;
+        if (SLICE || kRecompute) {
+            walk.map(unit, item_idx, tile_v0);
         } else {
             if (rem >= n_it) { rem -= n_it; tile += 1; skew += 1; }
             if (skew >= n_it) skew -= n_it;
+            item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
+            tile_v0 = tile * (long long)(THREADS * UNROLL);
         }
-        const int item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
         const DevItem it = s_items[item_idx];
+        const long long v0 = tile_v0 + threadIdx.x;
+        if (SLICE && tile_v0 + (long long)(threadIdx.x & ~31u) >= v_end) continue;  // nothing of this warp's is inside the slice
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
         const bool has_c = KW >= 3 && it.c >= 0, has_gc = KW >= 3 && it.slot_c >= 0;
         const bool has_d = KW >= 4 && it.d >= 0, has_gd = KW >= 4 && it.slot_d >= 0;
-        const long long v0 = tile * (long long)(THREADS * UNROLL) + threadIdx.x;
 
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxta = Xt + (long long)it.a * p.pitch;
@@ -410,7 +459,7 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const long long v = v0 + (long long)u * THREADS;
-            live[u] = v < p.n_vec;
+            live[u] = v < v_end;
             const long long off = v * N;
             if (kRecompute) {
 #pragma unroll
@@ -450,15 +499,30 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
         constexpr bool kPacked = sizeof(T) == 4 ? ((KW >= 4 && BYTES == 32) ? (A2_F32X2_FP32_KW4 != 0) : (A2_F32X2_FP32 != 0))
                                                 : (A2_F32X2_BF16 != 0);
         const bool before = p.msg_before_mix != 0;
-        for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
+        const int o_first = it.op_first - p.op_base;
+        for (int o = o_first; o < o_first + it.op_count; ++o) {
             const int kind = s_kind[o];
             const float ca = s_ca[o];
+            // A gradient operation whose worker needs another row for its next one (fresh gradients, Sec. 3.2)
+            // fetches it into the same registers as soon as it has used them: the load is in flight while the
+            // item's following operations run.
+            auto refetch = [&](auto& grow) {
+                const int rl = s_reload[o];
+                if (rl >= 0) {
+                    const T* const pg = G + (long long)rl * p.pitch;
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u)
+                        if (live[u]) V::load(pg + (v0 + (long long)u * THREADS) * N, grow[u]);
+                }
+            };
             if (kind == A2_OP_GRAD_A) {
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xa[u], xta[u], ca, ngamma, ga[u]);
+                refetch(ga);
             } else if (kind == A2_OP_GRAD_B) {
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xb[u], xtb[u], ca, ngamma, gb[u]);
+                refetch(gb);
             } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) mix_row<kPrecise, kPacked>(xa[u], xta[u], ca, ngamma);
@@ -470,6 +534,7 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
                 if (kind == A2_OP_GRAD_C) {
 #pragma unroll
                     for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xc[u], xtc[u], ca, ngamma, gc[u]);
+                    refetch(gc);
                 } else if (kind == A2_OP_COMM_AC) {
                     const float cb = s_cb[o];
 #pragma unroll
@@ -482,6 +547,7 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
                     if (kind == A2_OP_GRAD_D) {
 #pragma unroll
                         for (int u = 0; u < UNROLL; ++u) grad_row<kPrecise, kPacked>(xd[u], xtd[u], ca, ngamma, gd[u]);
+                        refetch(gd);
                     } else {
                         const float cb = s_cb[o];
                         if (kind == A2_OP_COMM_AD) {
@@ -540,29 +606,34 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
 #endif
 template <int BYTES> struct PlainCfg { static constexpr int UNROLL = BYTES == 32 ? A2_PLAIN_UNROLL : A2_PLAIN_UNROLL_128; };
 
-template <typename T, int BYTES, int UNROLL, int KW>
+template <typename T, int BYTES, int UNROLL, int KW, bool SLICE = false>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const EventArgs p) {
     using V = Vec<T, BYTES>;
     constexpr int N = V::N;
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    __shared__ int s_reload[kMaxOpsPerLaunch];
     for (int i = threadIdx.x; i < p.n_items; i += kEventThreads) s_items[i] = p.items[i];
-    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) s_kind[o] = (unsigned char)p.ops[o].kind;
+    for (int o = threadIdx.x; o < p.n_ops; o += kEventThreads) {
+        s_kind[o] = (unsigned char)p.ops[o].kind;
+        s_reload[o] = p.ops[o].reload;
+    }
     __syncthreads();
 
     T* const X = static_cast<T*>(p.x);
     const T* const G = static_cast<const T*>(p.g);
     const float alpha = p.alpha, ngamma = -p.gamma;
-    const long long n_units = (long long)p.n_items * p.n_tiles;
-    const int n_it = p.n_items;
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int rem = (int)(unit % n_it);
-        const long long tile = unit / n_it;
-        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
-        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+    const UnitWalk<SLICE, kEventThreads * UNROLL> walk(p);
+    const long long v_end = walk.v_end;
+    for (long long unit = walk.first; unit < walk.end; unit += walk.step) {
+        int item_idx;
+        long long tile_v0;
+        walk.map(unit, item_idx, tile_v0);
+        const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
         const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
-        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
+        const long long v0 = tile_v0 + threadIdx.x;
+        if (SLICE && tile_v0 + (long long)(threadIdx.x & ~31u) >= v_end) continue;
         T* const pxa = X + (long long)it.a * p.pitch;
         T* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
         T* const pxc = X + (long long)(has_c ? it.c : it.a) * p.pitch;
@@ -576,7 +647,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const long long v = v0 + (long long)u * kEventThreads;
-            live[u] = v < p.n_vec;
+            live[u] = v < v_end;
             const long long off = v * N;
 #pragma unroll
             for (int k = 0; k < N; ++k) { xa[u][k] = 0.f; xb[u][k] = 0.f; ga[u][k] = 0.f; gb[u][k] = 0.f; }
@@ -596,10 +667,20 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
             }
         }
         bool dirty = false;
-        for (int o = it.op_first; o < it.op_first + it.op_count; ++o) {
+        const int o_first = it.op_first - p.op_base;
+        for (int o = o_first; o < o_first + it.op_count; ++o) {
             const int kind = s_kind[o];
             if (kind == A2_OP_MIX_A) continue;
             dirty = true;
+            auto refetch = [&](auto& grow) {  // the worker's next gradient row, when it is another one
+                const int rl = s_reload[o];
+                if (rl >= 0) {
+                    const T* const pg = G + (long long)rl * p.pitch;
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u)
+                        if (live[u]) V::load(pg + (v0 + (long long)u * kEventThreads) * N, grow[u]);
+                }
+            };
             if (KW == 3 && (kind == A2_OP_GRAD_C || kind == A2_OP_COMM_AC || kind == A2_OP_COMM_BC)) {
 #pragma unroll
                 for (int u = 0; u < UC; ++u)
@@ -617,6 +698,9 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
                             xc[u][k] = __fmaf_rn(alpha, m, xc[u][k]);
                         }
                     }
+                if constexpr (KW == 3) {
+                    if (kind == A2_OP_GRAD_C) refetch(gc);
+                }
                 continue;
             }
 #pragma unroll
@@ -633,6 +717,8 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
                         xb[u][k] = __fmaf_rn(alpha, m, xb[u][k]);
                     }
                 }
+            if (kind == A2_OP_GRAD_A) refetch(ga);
+            else if (kind == A2_OP_GRAD_B) refetch(gb);
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -666,7 +752,7 @@ __device__ __forceinline__ uint32_t bf16_pack(float lo, float hi) {  // round to
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int WORDS, int UNROLL, int KW>
+template <int WORDS, int UNROLL, int KW, bool SLICE = false>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const EventArgs p) {
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
     __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
@@ -677,16 +763,17 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
     __nv_bfloat16* const X = static_cast<__nv_bfloat16*>(p.x);
     const __nv_bfloat16* const G = static_cast<const __nv_bfloat16*>(p.g);
     const float alpha = p.alpha, ngamma = -p.gamma;
-    const long long n_units = (long long)p.n_items * p.n_tiles;
-    const int n_it = p.n_items;
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int rem = (int)(unit % n_it);
-        const long long tile = unit / n_it;
-        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
-        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+    const UnitWalk<SLICE, kEventThreads * UNROLL> walk(p);
+    const long long v_end = walk.v_end;
+    for (long long unit = walk.first; unit < walk.end; unit += walk.step) {
+        int item_idx;
+        long long tile_v0;
+        walk.map(unit, item_idx, tile_v0);
+        const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0;
         const bool has_c = KW == 3 && it.c >= 0, has_gc = KW == 3 && it.slot_c >= 0;
-        const long long v0 = tile * (long long)(kEventThreads * UNROLL) + threadIdx.x;
+        const long long v0 = tile_v0 + threadIdx.x;
+        if (SLICE && tile_v0 + (long long)(threadIdx.x & ~31u) >= v_end) continue;
         __nv_bfloat16* const pxa = X + (long long)it.a * p.pitch;
         __nv_bfloat16* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch;
         const __nv_bfloat16* const pga = G + (long long)(has_ga ? it.slot_a : 0) * p.pitch;
@@ -701,7 +788,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const long long v = v0 + (long long)u * kEventThreads;
-            live[u] = v < p.n_vec;
+            live[u] = v < v_end;
             const long long off = v * (2 * WORDS);
 #pragma unroll
             for (int k = 0; k < WORDS; ++k) { xa[u][k] = 0u; xb[u][k] = 0u; ga[u][k] = 0u; gb[u][k] = 0u; }
@@ -720,7 +807,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
                 if (has_gb) Words<WORDS>::ld(pgb + off, gb[u]);
             }
         }
-        const int o_begin = it.op_first, o_end = it.op_first + it.op_count;
+        const int o_begin = it.op_first - p.op_base, o_end = o_begin + it.op_count;
         bool dirty = false;
         for (int o = o_begin; o < o_end; ++o) dirty |= s_kind[o] != A2_OP_MIX_A;
         constexpr int WG = A2_PLAIN_BF16_GROUP < WORDS ? A2_PLAIN_BF16_GROUP : WORDS;  // words widened and updated together
@@ -805,7 +892,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain_bf16(const
 #ifndef A2_BF16_PACKED_GROUP
 #define A2_BF16_PACKED_GROUP 2  // 32-bit words (pairs of columns) widened and updated together
 #endif
-template <int WORDS, int WG>
+template <int WORDS, int WG, bool SLICE = false>
 __global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_packed(const EventArgs p) {
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
     __shared__ float s_ca[kMaxOpsPerLaunch];
@@ -826,17 +913,16 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_packed(cons
     const __nv_bfloat16* const G = static_cast<const __nv_bfloat16*>(p.g);
     const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
     const bool before = p.msg_before_mix != 0;
-    const long long n_units = (long long)p.n_items * p.n_tiles;
-    const int n_it = p.n_items;
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int rem = (int)(unit % n_it);
-        const long long tile = unit / n_it;
-        const int skew = (int)((unsigned long long)tile % (unsigned)n_it);
-        const DevItem it = s_items[rem + skew >= n_it ? rem + skew - n_it : rem + skew];
+    const UnitWalk<SLICE, kEventThreads> walk(p);
+    for (long long unit = walk.first; unit < walk.end; unit += walk.step) {
+        int item_idx;
+        long long tile_v0;
+        walk.map(unit, item_idx, tile_v0);
+        const DevItem it = s_items[item_idx];
         const bool has_b = it.b >= 0, has_c = it.c >= 0;
         const bool has_ga = it.slot_a >= 0, has_gb = it.slot_b >= 0, has_gc = it.slot_c >= 0;
-        const long long v = tile * (long long)kEventThreads + threadIdx.x;
-        if (v >= p.n_vec) continue;
+        const long long v = tile_v0 + threadIdx.x;
+        if (v >= walk.v_end) continue;
         const long long off = v * (2 * WORDS);
         const long long ra = (long long)it.a * p.pitch + off;
         const long long rb = (long long)(has_b ? it.b : it.a) * p.pitch + off;
@@ -859,7 +945,7 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_bf16_packed(cons
         if (has_gb) Words<WORDS>::ld(G + (long long)it.slot_b * p.pitch + off, gb);
         if (has_gc) Words<WORDS>::ld(G + (long long)it.slot_c * p.pitch + off, gc);
 
-        const int o_begin = it.op_first, o_end = it.op_first + it.op_count;
+        const int o_begin = it.op_first - p.op_base, o_end = o_begin + it.op_count;
         constexpr int E = 2 * WG;  // columns taken through the operations together
 #pragma unroll
         for (int k0 = 0; k0 < WORDS; k0 += WG) {
@@ -1010,6 +1096,29 @@ __global__ void __launch_bounds__(kThreads) k_consensus_final(const double* __re
 #define A2_EVENT4_UNROLL_128 2
 #endif
 
+
+// Grid of a launch. Round robin: one wave of resident CTAs (fewer if there are fewer units). Column slices: the same
+// wave, each CTA owning `slice_vec` consecutive vectors of every row -- a multiple of 8 vectors (whole 128-byte
+// lines) and at least one warp's worth, so that narrow rows give fewer, full warps instead of many empty ones.
+struct GridShape {
+    unsigned grid;
+    int slice_vec;
+};
+inline GridShape grid_shape(bool slice, long long n_vec, long long n_units, long long wave) {
+    GridShape g{0u, 0};
+    if (!slice) {
+        g.grid = (unsigned)(wave < n_units ? wave : n_units);
+        return g;
+    }
+    long long per = (n_vec + wave - 1) / wave;
+    per = (per + 7) / 8 * 8;
+    if (per < 32) per = 32;
+    if (per > 0x7FFFFFF8LL) per = 0x7FFFFFF8LL;
+    g.slice_vec = (int)per;
+    g.grid = (unsigned)((n_vec + per - 1) / per);
+    return g;
+}
+
 template <typename T, int BYTES, int KW, int THREADS = kEventThreads, int U = EventCfg<T, BYTES>::UNROLL>
 int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr int N = Vec<T, BYTES>::N;
@@ -1021,13 +1130,15 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
+    a.op_base = L.op_base;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const int per_sm = KW == 4 ? dev.event4_ctas_per_sm[BYTES == 32 ? 1 : 0]
                                : (KW == 3 ? dev.event3_ctas_per_sm : dev.event_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
-    long long grid = (long long)dev.sm_count * per_sm;
-    if (grid > n_units) grid = n_units;
-    if (grid < 1) return 0;
-    k_apply_events<T, BYTES, U, KW, THREADS><<<(unsigned)grid, THREADS, 0, stream>>>(a);
+    const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * per_sm);
+    a.slice_vec = gs.slice_vec;
+    if (gs.grid < 1) return 0;
+    if (L.slice) k_apply_events<T, BYTES, U, KW, THREADS, true><<<gs.grid, THREADS, 0, stream>>>(a);
+    else k_apply_events<T, BYTES, U, KW, THREADS, false><<<gs.grid, THREADS, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -1043,12 +1154,14 @@ int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t str
     a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
+    a.op_base = L.op_base;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const int per_sm = (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
-    long long grid = (long long)dev.sm_count * per_sm;
-    if (grid > n_units) grid = n_units;
-    if (grid < 1) return 0;
-    k_apply_events_plain<T, BYTES, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * per_sm);
+    a.slice_vec = gs.slice_vec;
+    if (gs.grid < 1) return 0;
+    if (L.slice) k_apply_events_plain<T, BYTES, U, KW, true><<<gs.grid, kEventThreads, 0, stream>>>(a);
+    else k_apply_events_plain<T, BYTES, U, KW, false><<<gs.grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -1063,11 +1176,14 @@ int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t 
     a.n_tiles = (int)((a.n_vec + vec_per_tile - 1) / vec_per_tile);
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
+    a.op_base = L.op_base;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    long long grid = (long long)dev.sm_count * (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[1][WORDS == 8 ? 1 : 0];
-    if (grid > n_units) grid = n_units;
-    if (grid < 1) return 0;
-    k_apply_events_plain_bf16<WORDS, U, KW><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    const long long wave = (long long)dev.sm_count * (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[1][WORDS == 8 ? 1 : 0];
+    const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, wave);
+    a.slice_vec = gs.slice_vec;
+    if (gs.grid < 1) return 0;
+    if (L.slice) k_apply_events_plain_bf16<WORDS, U, KW, true><<<gs.grid, kEventThreads, 0, stream>>>(a);
+    else k_apply_events_plain_bf16<WORDS, U, KW, false><<<gs.grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
@@ -1236,11 +1352,13 @@ int launch_bf16_packed(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t
     a.n_tiles = (int)((a.n_vec + kEventThreads - 1) / kEventThreads);
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
+    a.op_base = L.op_base;
     const long long n_units = (long long)a.n_items * a.n_tiles;
-    long long grid = (long long)dev.sm_count * dev.event3_ctas_per_sm[1][WORDS == 8 ? 1 : 0];
-    if (grid > n_units) grid = n_units;
-    if (grid < 1) return 0;
-    k_apply_events_bf16_packed<WORDS, A2_BF16_PACKED_GROUP><<<(unsigned)grid, kEventThreads, 0, stream>>>(a);
+    const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * dev.event3_ctas_per_sm[1][WORDS == 8 ? 1 : 0]);
+    a.slice_vec = gs.slice_vec;
+    if (gs.grid < 1) return 0;
+    if (L.slice) k_apply_events_bf16_packed<WORDS, A2_BF16_PACKED_GROUP, true><<<gs.grid, kEventThreads, 0, stream>>>(a);
+    else k_apply_events_bf16_packed<WORDS, A2_BF16_PACKED_GROUP, false><<<gs.grid, kEventThreads, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 

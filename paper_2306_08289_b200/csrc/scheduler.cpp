@@ -37,7 +37,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     if (n < 2) { err = "need n >= 2 workers"; return A2_EINVAL; }
     if (n_grad_slots < 0 || n_events < 0) { err = "negative size"; return A2_EINVAL; }
     if (n_events > 0 && (!times || !wi || !wj || !slot)) { err = "event arrays are NULL"; return A2_EINVAL; }
-    if (flags & ~uint32_t(A2_SCHED_FUSE | A2_SCHED_RESIDENT | A2_SCHED_CHAIN)) { err = "unknown scheduling flag"; return A2_EINVAL; }
+    if (flags & ~uint32_t(A2_SCHED_FUSE | A2_SCHED_RESIDENT | A2_SCHED_CHAIN | A2_SCHED_ROW_PER_OP)) { err = "unknown scheduling flag"; return A2_EINVAL; }
     if (max_workers_per_item <= 0) max_workers_per_item = kMaxItemWorkers;
     if (max_workers_per_item < 2 || max_workers_per_item > kMaxItemWorkers) { err = "an item holds 2 to 4 workers"; return A2_EINVAL; }
     if (max_ops_per_item <= 0) max_ops_per_item = kDefaultMaxOpsPerItem;
@@ -45,6 +45,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
     const bool resident = (flags & A2_SCHED_RESIDENT) != 0;
     const bool chain = !resident && (flags & A2_SCHED_CHAIN) != 0 && max_ops_per_item >= 2;
     const bool fuse = !resident && ((flags & A2_SCHED_FUSE) != 0 || chain) && max_ops_per_item >= 2;
+    const bool row_per_op = fuse && (flags & A2_SCHED_ROW_PER_OP) != 0;  // a worker's gradient row may change inside an item
 
     a2cid2_sched* s = new (std::nothrow) a2cid2_sched();
     if (!s) { err = "out of host memory"; return A2_ENOMEM; }
@@ -92,6 +93,8 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
         struct Build {
             SchedItem it;
             int64_t head = -1, tail = -1;  // first and last operation
+            int32_t cur_row[kMaxItemWorkers] = {-1, -1, -1, -1};   // gradient row each worker's registers hold at the item's end so far
+            int64_t last_gop[kMaxItemWorkers] = {-1, -1, -1, -1};  // each worker's latest gradient operation
         };
         std::vector<Build> items;
         std::vector<SchedOp> ops;      // creation order
@@ -126,7 +129,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
         // can the held-back gradient events of worker w go into item k (which holds w)?
         auto slot_ok = [&](int64_t k, int32_t w) -> bool {
             const Pending& p = pend[(size_t)w];
-            if (p.events.empty()) return true;
+            if (p.events.empty() || row_per_op) return true;
             SchedItem& it = items[(size_t)k].it;
             const int32_t cur = slot_ref(it, local_of(it, w));
             return cur == -1 || cur == p.slot;
@@ -135,12 +138,16 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
         auto push_pending = [&](int64_t k, int32_t w) {
             Pending& p = pend[(size_t)w];
             if (p.events.empty()) return;
-            SchedItem& it = items[(size_t)k].it;
-            const int l = local_of(it, w);
-            slot_ref(it, l) = p.slot;
+            const int l = local_of(items[(size_t)k].it, w);
             const int32_t kind = l == 0 ? A2_OP_GRAD_A : (l == 1 ? A2_OP_GRAD_B : (l == 2 ? A2_OP_GRAD_C : A2_OP_GRAD_D));
             for (int64_t e : p.events) {
+                Build& bd = items[(size_t)k];
+                const int32_t row = slot[e];
+                if (bd.cur_row[l] < 0) slot_ref(bd.it, l) = row;  // the worker's first gradient row: read with the state rows
+                else if (bd.cur_row[l] != row) ops[(size_t)bd.last_gop[l]].reload = row;  // fetched once the previous one is used
+                bd.cur_row[l] = row;
                 add_op(k, SchedOp{e, kind, times[e], tcur[(size_t)w], 0.0});
+                items[(size_t)k].last_gop[l] = (int64_t)ops.size() - 1;
                 tcur[(size_t)w] = times[e];
             }
             p.events.clear();
@@ -180,7 +187,7 @@ int build_schedule(int32_t n, int32_t n_grad_slots, const double* t_last, int64_
             if (j == -1) {
                 if (fuse) {
                     Pending& p = pend[(size_t)i];
-                    if (!p.events.empty() && (p.slot != slot[e] || (int32_t)p.events.size() >= max_ops_per_item - 1)) flush(i);
+                    if (!p.events.empty() && ((!row_per_op && p.slot != slot[e]) || (int32_t)p.events.size() >= max_ops_per_item - 1)) flush(i);
                     p.slot = slot[e];
                     p.events.push_back(e);
                 } else {
@@ -324,6 +331,7 @@ void schedule_stats(const a2cid2_sched& s, int64_t b0, int64_t b1, int64_t d, in
             rows_moved += 2 * state_rows + (it.slot_a >= 0 ? 1 : 0) + (it.slot_b >= 0 ? 1 : 0) + (it.slot_c >= 0 ? 1 : 0) +
                           (it.slot_d >= 0 ? 1 : 0);
         for (int32_t o = 0; o < it.n_ops; ++o) {
+            if (s.ops[(size_t)(it.first_op + o)].reload >= 0) rows_moved += 1;  // a gradient row fetched inside the item
             const int32_t kind = s.ops[(size_t)(it.first_op + o)].kind;
             if (kind == A2_OP_COMM || kind == A2_OP_COMM_AC || kind == A2_OP_COMM_BC || kind == A2_OP_COMM_AD ||
                 kind == A2_OP_COMM_BD || kind == A2_OP_COMM_CD) { st.n_comm += 1; rows_single += momentum ? 8 : 4; }

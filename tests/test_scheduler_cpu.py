@@ -28,7 +28,8 @@ def _replay(cfg, ev, sched, params, x0, G):
 
 
 @pytest.mark.parametrize("name,d,n_events", [("cfg1", 7, 2000), ("cfg2", 5, 3000), ("cfg4", 3, 4000), ("cfg5", 3, 4000)])
-@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN])
+@pytest.mark.parametrize("flags", [0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_FUSE | B.A2_SCHED_ROW_PER_OP,
+                                   B.A2_SCHED_CHAIN | B.A2_SCHED_ROW_PER_OP])
 def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
     cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
     cfg = cfg if cfg.storage == "f32" else W.WorkloadConfig(**{**cfg.__dict__, "storage": "f32"})
@@ -54,22 +55,28 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
             assert it.batch == b and it.n_ops >= 1
             ws = set(it.workers())
             assert len(ws) == len(it.workers()) and not (ws & used)
-            assert (it.c < 0 or it.b >= 0) and (it.d < 0 or it.c >= 0) and (flags == B.A2_SCHED_CHAIN or it.c < 0)
+            assert (it.c < 0 or it.b >= 0) and (it.d < 0 or it.c >= 0) and (flags & B.A2_SCHED_CHAIN or it.c < 0)
             used |= ws
             evs, kinds = s.ops(it.first_op, it.n_ops)
             pairs = {B.A2_OP_COMM: (it.a, it.b), B.A2_OP_COMM_AC: (it.a, it.c), B.A2_OP_COMM_BC: (it.b, it.c),
                      B.A2_OP_COMM_AD: (it.a, it.d), B.A2_OP_COMM_BD: (it.b, it.d), B.A2_OP_COMM_CD: (it.c, it.d)}
             grads = {B.A2_OP_GRAD_A: (it.a, it.slot_a), B.A2_OP_GRAD_B: (it.b, it.slot_b), B.A2_OP_GRAD_C: (it.c, it.slot_c),
                      B.A2_OP_GRAD_D: (it.d, it.slot_d)}
-            for e, kd in zip(evs, kinds):
+            reloads = s.op_reloads(it.first_op, it.n_ops)
+            assert flags & B.A2_SCHED_ROW_PER_OP or np.all(reloads == -1)
+            for e, kd, rl in zip(evs, kinds, reloads):
                 if kd in pairs:
                     # the pair may be stored the other way round: the update is symmetric in its two workers
                     assert {ev.wi[e], ev.wj[e]} == set(pairs[kd]) and min(pairs[kd]) >= 0
                     touched = pairs[kd]
                 else:
-                    w, sl = grads[kd]
+                    w, sl = grads[kd]  # sl: the row the worker's gradient registers hold when the operation runs
                     assert ev.wi[e] == w and ev.wj[e] == -1 and ev.slot[e] == sl
+                    if rl >= 0:
+                        assert rl != sl
+                        grads[kd] = (w, int(rl))
                     touched = (w,)
+                assert kd not in pairs or rl == -1
                 for w in touched:
                     assert last_pos.get(w, -1) < e  # this worker's events come in stream order
                     last_pos[w] = e
@@ -82,6 +89,11 @@ def test_batches_replay_to_the_time_ordered_state(name, d, n_events, flags):
     assert st["bytes_one_by_one"] == (8 * st["n_comm"] + 5 * st["n_grad"]) * cfg.d * 4
     if flags:
         assert st["bytes_moved"] < st["bytes_one_by_one"] and s.num_items < len(ev)
+        if flags & B.A2_SCHED_ROW_PER_OP:  # never more rows than with items cut at every change of row
+            cut = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=flags & ~B.A2_SCHED_ROW_PER_OP)
+            assert st["bytes_moved"] <= cut.stats(cfg.d, 4)["bytes_moved"] and s.num_items <= cut.num_items
+            if cfg.grad_pool > 1:
+                assert st["bytes_moved"] < cut.stats(cfg.d, 4)["bytes_moved"] and s.num_items < cut.num_items
         if flags == B.A2_SCHED_CHAIN:  # chaining moves fewer rows in fewer batches than gradient fusion alone
             f = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)
             assert st["bytes_moved"] < f.stats(cfg.d, 4)["bytes_moved"] and s.num_batches < f.num_batches
@@ -217,7 +229,7 @@ def test_resident_schedule_is_one_batch_in_stream_order():
     sim.apply_stream(ev)
     assert np.array_equal(s.t_final(cfg.n), sim.t)
     with pytest.raises(B.A2Error):
-        B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=8)
+        B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=16)
 
 
 def test_fifo_stream_with_ties_replays_exactly():
@@ -260,6 +272,8 @@ def test_random_streams_property():
             else:
                 wi.append(i); wj.append(-1); sl.append(draw(st.integers(0, n_slots - 1)))
         flags = draw(st.sampled_from([0, B.A2_SCHED_FUSE, B.A2_SCHED_CHAIN, B.A2_SCHED_CHAIN]))
+        if flags and draw(st.booleans()):
+            flags |= B.A2_SCHED_ROW_PER_OP
         cap = draw(st.sampled_from([0, 2, 3, 5]))
         kw = draw(st.sampled_from([0, 2, 3, 4]))
         return (n, n_slots, times, np.array(wi, dtype=np.int32), np.array(wj, dtype=np.int32), np.array(sl, dtype=np.int32),
@@ -283,12 +297,18 @@ def test_random_streams_property():
                 it = s.item(k)
                 ws = set(it.workers())
                 assert not (ws & used) and (cap == 0 or it.n_ops <= max(cap, 1))
-                assert len(ws) <= (kw or 4) and (flags == B.A2_SCHED_CHAIN or len(ws) <= 2)
+                assert len(ws) <= (kw or 4) and (flags & B.A2_SCHED_CHAIN or len(ws) <= 2)
                 used |= ws
                 evs, kinds = s.ops(it.first_op, it.n_ops)
                 slots = {B.A2_OP_GRAD_A: it.slot_a, B.A2_OP_GRAD_B: it.slot_b, B.A2_OP_GRAD_C: it.slot_c, B.A2_OP_GRAD_D: it.slot_d}
-                for x, kd in zip(evs, kinds):  # one gradient row per worker and item
+                reloads = s.op_reloads(it.first_op, it.n_ops)
+                for x, kd, rl in zip(evs, kinds, reloads):
+                    # a gradient operation finds its row in its worker's gradient registers: the item's row for
+                    # that worker, or the one fetched after the worker's previous gradient operation
                     assert kd not in slots or sl[x] == slots[kd]
+                    if rl >= 0:
+                        assert kd in slots and flags & B.A2_SCHED_ROW_PER_OP
+                        slots[kd] = int(rl)
                 e = evs[np.argsort(times[evs], kind="stable")]
                 # inside an item a worker's own events are already in stream order
                 for w in ws:
