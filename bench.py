@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--events-per-step", type=int, default=500)
     ap.add_argument("--grad-pool", type=int, default=None,
                     help="gradient rows per worker, used round-robin by its gradient events (default: the workload's own)")
+    ap.add_argument("--launch-mode", default="auto", choices=["auto", "per-batch", "column-slices"],
+                    help="how a whole step is put on the GPU (a2cid2_set_launch_mode)")
     ap.add_argument("--no-fuse", action="store_true", help="one event per item (no gradient fusion)")
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -248,6 +250,8 @@ def main():
 
     eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
                    device=str(device))
+    eng.set_launch_mode({"auto": B.A2_LAUNCH_AUTO, "per-batch": B.A2_LAUNCH_PER_BATCH,
+                         "column-slices": B.A2_LAUNCH_COLUMN_SLICES}[args.launch_mode])
     fill_engine(eng, cfg, threads)
     # four stretches of the stream: plans resident on the device, end to end, shared-memory-resident mode,
     # and the asynchronous baseline without the momentum buffer

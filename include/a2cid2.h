@@ -252,8 +252,8 @@ int a2cid2_consensus_distance(a2cid2_t* h, double t_eval, double* out);
  *   out_device  device, one double, written by the queued work; the caller owns it
  *
  * The first call on each device looks up the device address of the fixed array (with that
- * device current) and remembers it; make that first call during start-up, outside any stream
- * capture. All calls on one device share the array: a call overwrites every entry it later
+ * device current), remembers it, and has the kernels of both storage types loaded onto the
+ * device; make that first call during start-up, outside any stream capture. All calls on one device share the array: a call overwrites every entry it later
  * reads, so nothing has to be cleared between calls, but two calls whose work overlaps on the
  * GPU (different streams, no ordering between them) race on it and give wrong sums. Calls on
  * one stream, or otherwise ordered, are safe. Errors: A2_EINVAL, A2_ERANGE, A2_ECUDA; the text

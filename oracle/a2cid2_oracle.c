@@ -35,6 +35,7 @@
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <string.h>
 
 enum { A2O_OK = 0, A2O_EINVAL = -1, A2O_EORDER = -2, A2O_ERANGE = -3 };
 
@@ -181,4 +182,56 @@ double a2o_consensus_at(int32_t n, int64_t d, int64_t ld, double eta, const doub
         }
     }
     return total;
+}
+
+/*
+ * Model of reduced-precision STORAGE (no passage of the paper: the method is stated in real numbers; this
+ * models an implementation that keeps its state in bfloat16 and writes rows back at known points). The
+ * value is rounded to IEEE binary32 and then to bfloat16 -- the upper 16 bits of that binary32 -- both to
+ * nearest, ties to even. Finite inputs only.
+ */
+double a2o_to_bf16(double v) {
+    float f = (float)v;
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Round columns [0, d) of the rows X[w], Xt[w] (w in rows[0 .. n_rows)) to bfloat16. */
+void a2o_round_rows_bf16(int64_t d, int64_t ld, double* X, double* Xt, int32_t n_rows, const int32_t* rows) {
+    for (int32_t r = 0; r < n_rows; ++r) {
+        double* x = X + (size_t)rows[r] * ld;
+        double* xt = Xt + (size_t)rows[r] * ld;
+        for (int64_t k = 0; k < d; ++k) {
+            x[k] = a2o_to_bf16(x[k]);
+            xt[k] = a2o_to_bf16(xt[k]);
+        }
+    }
+}
+
+/*
+ * a2o_run on consecutive groups of events, with the storage model applied between groups: group k is
+ * events [group_end[k-1], group_end[k]) (group_end[-1] = 0), applied in the order given by a2o_run (fp64
+ * arithmetic, unchanged); then the rows of workers[worker_ptr[k] .. worker_ptr[k+1]) are rounded to
+ * bfloat16. The time-order check of a2o_run holds inside a group; groups may overlap in time (they are
+ * the items of a schedule, which keeps every worker's own order).
+ */
+int a2o_run_groups_bf16(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double alpha_t, double gamma,
+                        double* X, double* Xt, double* tl, const double* G, int32_t n_slots, int64_t ldg,
+                        const double* times, const int32_t* wi, const int32_t* wj, const int32_t* slot,
+                        int32_t variant, int64_t n_groups, const int64_t* group_end, const int64_t* worker_ptr,
+                        const int32_t* workers) {
+    int64_t e0 = 0;
+    for (int64_t k = 0; k < n_groups; ++k) {
+        const int64_t e1 = group_end[k];
+        if (e1 < e0) return A2O_EINVAL;
+        const int rc = a2o_run(n, d, ld, eta, alpha, alpha_t, gamma, X, Xt, tl, G, n_slots, ldg, e1 - e0, times + e0,
+                               wi + e0, wj + e0, slot + e0, variant);
+        if (rc != A2O_OK) return rc;
+        a2o_round_rows_bf16(d, ld, X, Xt, (int32_t)(worker_ptr[k + 1] - worker_ptr[k]), workers + worker_ptr[k]);
+        e0 = e1;
+    }
+    return A2O_OK;
 }

@@ -1608,6 +1608,13 @@ int launch_consensus_static(const void* x, int64_t pitch, int32_t n, int64_t d, 
             void* p = nullptr;
             e = cudaGetSymbolAddress(&p, g_static_partials);
             if (e != cudaSuccess) return (int)e;
+            // With lazy module loading a kernel's code reaches the device when it is first needed. Asking for the
+            // attributes of the three kernels this entry point can launch (both storage types) loads them now, so
+            // that a later call with the other storage type brings nothing new onto the device either.
+            cudaFuncAttributes fa;
+            if ((e = cudaFuncGetAttributes(&fa, k_consensus_partial<float, 16, false>)) != cudaSuccess) return (int)e;
+            if ((e = cudaFuncGetAttributes(&fa, k_consensus_partial<__nv_bfloat16, 16, false>)) != cudaSuccess) return (int)e;
+            if ((e = cudaFuncGetAttributes(&fa, k_consensus_final)) != cudaSuccess) return (int)e;
             g_static_addr[dev] = static_cast<double*>(p);
         }
         partials = g_static_addr[dev];

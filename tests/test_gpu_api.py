@@ -72,11 +72,17 @@ def test_apply_events_equals_plan_and_reports_stats():
     cfg = _small()
     ev = W.config_events(cfg)
     outs = []
-    for mode in ("apply", "plan", "plan_chunks"):
+    for mode in ("apply", "apply_per_batch", "apply_slices", "plan", "plan_chunks"):
         eng, _ = P.make_small(cfg)
-        if mode == "apply":
+        if mode.startswith("apply"):
+            eng.set_launch_mode({"apply": B.A2_LAUNCH_AUTO, "apply_per_batch": B.A2_LAUNCH_PER_BATCH,
+                                 "apply_slices": B.A2_LAUNCH_COLUMN_SLICES}[mode])
             st = eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE, want_stats=True)
-            assert st["n_events"] == len(ev) and st["n_launches"] >= st["n_batches"] > 0
+            assert st["n_events"] == len(ev) and st["n_batches"] > 0 and st["n_launches"] > 0
+            if mode == "apply_per_batch":
+                assert st["n_launches"] >= st["n_batches"]
+            if mode == "apply_slices":  # a launch holds the items of several batches
+                assert st["n_launches"] < st["n_batches"]
             assert st["bytes_moved"] < st["bytes_one_by_one"] and st["descriptor_bytes"] > 0
         else:
             p = eng.plan(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE)

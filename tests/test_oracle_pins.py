@@ -597,6 +597,45 @@ def test_bf16_rounding_of_the_storage_model():
     assert s.X[0, 0] == 1.0 + 2.0 ** -9 and s.X[1, 1] == 1.0 and s.Xt[1, 1] == 1.0
 
 
+def test_c_storage_model_rounds_like_the_hand_checked_one_and_groups_equal_the_loop():
+    """The C checker's own bfloat16 rounding (used when a whole schedule is run with the storage modelled):
+    the hand-worked values above, and bit-equality with the NumPy routine on random, tiny and tie values.
+    Running groups of events with a rounding after each equals apply() + round_rows() group by group."""
+    from oracle.sim import lib, round_to_bf16
+
+    f = lib().a2o_to_bf16
+    assert f(1.0 + 2.0 ** -8) == 1.0 and f(1.0 + 3 * 2.0 ** -8) == 1.0 + 2.0 ** -6          # ties to even
+    assert f(1.0 + 2.0 ** -8 + 2.0 ** -20) == 1.0 + 2.0 ** -7 and f(-0.5) == -0.5 and f(0.0) == 0.0
+    rng = np.random.default_rng(11)
+    v = np.concatenate([rng.standard_normal(4000) * 0.02, rng.standard_normal(500) * 1e-30,
+                        (1.0 + np.arange(64) * 2.0 ** -8) * 0.0123, -(1.0 + np.arange(64) * 2.0 ** -8)])
+    assert np.array_equal(np.array([f(float(a)) for a in v]), round_to_bf16(v))
+    cfg = W.CONFIGS["cfg5"].scaled(d=37, n_events=600)
+    _, x0 = W.x0_matrix(cfg)
+    _, G = W.grad_matrix(cfg)
+    ev = W.config_events(cfg)
+    par = spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
+    # groups: runs of 1..5 consecutive events; after each, the rows of the workers it touched are rounded
+    ends = np.unique(np.concatenate([np.cumsum(rng.integers(1, 6, size=400)), [len(ev)]]))
+    ends = ends[ends <= len(ev)]
+    loop = OracleSim(x0, *par, cfg.gamma, grads=G)
+    ptr, flat, e0 = [0], [], 0
+    for e1 in ends:
+        c = ev.slice(e0, e1)
+        w = sorted(set(c.wi.tolist()) | set(int(j) for j in c.wj if j >= 0))
+        loop.apply_stream(c)
+        loop.round_rows(w)
+        flat += w
+        ptr.append(len(flat))
+        e0 = e1
+    once = OracleSim(x0, *par, cfg.gamma, grads=G)
+    once.apply_groups_bf16(ev.times, ev.wi, ev.wj, ev.slot, ends, ptr, flat)
+    assert np.array_equal(once.X, loop.X) and np.array_equal(once.Xt, loop.Xt) and np.array_equal(once.t, loop.t)
+    plain = OracleSim(x0, *par, cfg.gamma, grads=G)
+    plain.apply_stream(ev)
+    assert not np.array_equal(once.X, plain.X)  # the rounding did take place
+
+
 def test_what_bf16_storage_alone_costs():
     """Why the 2e-2 bar of bf16-storage runs is applied norm-wise: a run that does all arithmetic in
     fp64 and only rounds the rows of an event's workers to bf16 when they are stored already differs

@@ -5,9 +5,12 @@ already owns the device, or they sit in a loop that cannot afford the device-wid
 allocation may cause. For them the library offers the consensus distance with its scratch in a
 fixed array inside the library instead of in allocated memory. This test calls it through the C
 ABI twice in a row, on different data and sizes, and compares each result with the handle-based
-a2cid2_consensus_distance on the same rows, within the tolerance the other consensus tests use.
-The second call uses fewer partial sums than the first, so anything the first call left in the
-shared array would show up as a wrong sum.
+a2cid2_consensus_distance on the same rows and with the CPU checker's reduction of the same rows
+(a fault shared by the two device entry points would pass the first comparison alone), within the
+tolerance the other consensus tests use. The second call uses fewer partial sums than the first, so
+anything the first call left in the shared array would show up as a wrong sum; and the free device
+memory is read before and after that second call, since the point of the entry point is that it
+takes none.
 
 The file is named so that pytest collects it last; it needs nothing from the other tests and
 passes on its own in a fresh process as well as after them.
@@ -15,7 +18,9 @@ passes on its own in a fresh process as well as after them.
 import numpy as np
 import pytest
 
+from oracle.sim import OracleSim
 from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import workload as W
 
 pytestmark = pytest.mark.gpu
 
@@ -41,17 +46,23 @@ def test_static_scratch_matches_allocating_entry_point_twice(storage):
     for k, (n, d) in enumerate([(12, 300_007), (5, 4_099)]):  # many partials, then few
         rows = (rng.standard_normal((n, d)) * (k + 1.0) + 0.5).astype(np.float32)
         if storage == "bf16":
-            from paper_2306_08289_b200 import workload as W
-
             rows = W.f32_to_bf16_bits(rows)
         eng, want = _reference(n, d, storage, rows)
+        wide = W.bf16_bits_to_f32(rows).astype(np.float64) if storage == "bf16" else rows.astype(np.float64)
+        checker = OracleSim(wide, 0.0, 0.5, 0.5, 0.0).consensus()
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.consensus_distance_static(eng.x.data_ptr(), n, d, eng.pitch, code, stream, out[k:].data_ptr())
         torch.cuda.synchronize()
+        free_after = torch.cuda.mem_get_info()[0]
+        if k == 1:  # the first call on a device may load the kernels; later calls take nothing
+            assert free_after == free_before, (free_before, free_after)
         got = float(out[k].item())
-        results.append((got, want))
+        results.append((got, want, checker))
         eng.close()
-    for got, want in results:
+    for got, want, checker in results:
         assert want > 0 and abs(got - want) <= REL_TOL * want, (got, want)
+        assert abs(got - checker) <= REL_TOL * checker, (got, checker)
 
 
 def test_static_scratch_rejects_what_it_cannot_hold():
