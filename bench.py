@@ -4,9 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg4]
 
 A step is one pass of the whole hot path over one chunk of the seeded event stream: host
-scheduling, one fused event kernel per batch, then the consensus-distance reduction. The default
-workload is the 64-worker ring with ResNet-50-sized rows (d = 25.6e6, fp32), 500 events per step
-and a consensus distance after every step; 3 warm-up + 17 timed steps are its 10,000 events.
+scheduling, the fused event kernel over the chunk's batches, then the consensus-distance reduction.
+The default workload is the 64-worker ring with ResNet-50-sized rows (d = 25.6e6, fp32), 500 events
+per step and a consensus distance after every step.
 
 Printed JSON line (rank 0):
   value     events/s with the step's descriptors already resident on the device (plans built
@@ -16,9 +16,13 @@ Printed JSON line (rank 0):
             timed region
   roofline  of the event kernel: bytes its items must move / its measured time, against the
             measured copy bandwidth of this machine's B200s
+  clocks    SM clock and throttle reasons sampled (NVML) inside the timed region of `value`
+  fresh_gradients   the same workload with a pool of gradient rows per worker, so that consecutive
+            gradient events of a worker use different rows (fetched inside chained items)
+  other_configs     the other four workloads, a few timed steps each
   cpu_baseline  the CPU checker timed on a column slice of the same workload (reported only)
-With N > 1 every rank runs an independent replica (the path has no exchange between GPUs).
-`--impl reference` times the CPU checker alone, as the reference arm.
+With N > 1 every rank runs an independent replica (the path has no exchange between GPUs) and only
+the main figures are taken. `--impl reference` times the CPU checker alone, as the reference arm.
 """
 from __future__ import annotations
 
@@ -28,8 +32,10 @@ import os
 import statistics
 import subprocess
 import sys
+import threading
 import time
 from concurrent.futures import ThreadPoolExecutor
+from dataclasses import replace
 
 import numpy as np
 
@@ -42,12 +48,12 @@ from paper_2306_08289_b200.distutil import Ranks, aggregate_throughput  # noqa: 
 
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per event-kernel launch from the committed ncu
-# summary (profiles/k_apply_events_cfg4_d2m.md: two launches of the four-worker instance on a
-# d = 2e6 case), as a ratio to the bytes the launch's items must move: reads 1.000, writes 0.93
-# (the rest was still in L2 when the small launches ended). None once the kernel has changed
-# since the counters were taken.
-NCU_TRAFFIC_RATIO = 0.973
+# dram__bytes_read.sum + dram__bytes_write.sum of one event-kernel launch as a ratio to the bytes the
+# launch's items must move, from the committed ncu summary named beside it; None while the kernel has
+# changed since the counters were taken.
+NCU_TRAFFIC_RATIO = None
+NCU_TRAFFIC_SOURCE = None
+LAUNCH_MODES = {"auto": 0, "per-batch": 1, "column-slices": 2}
 
 
 def parse_args():
@@ -61,14 +67,17 @@ def parse_args():
     ap.add_argument("--events-per-step", type=int, default=500)
     ap.add_argument("--grad-pool", type=int, default=None,
                     help="gradient rows per worker, used round-robin by its gradient events (default: the workload's own)")
-    ap.add_argument("--launch-mode", default="auto", choices=["auto", "per-batch", "column-slices"],
+    ap.add_argument("--launch-mode", default="auto", choices=sorted(LAUNCH_MODES),
                     help="how a whole step is put on the GPU (a2cid2_set_launch_mode)")
     ap.add_argument("--no-fuse", action="store_true", help="one event per item (no gradient fusion)")
+    ap.add_argument("--no-chain", action="store_true", help="gradient fusion only (A2_SCHED_FUSE), no item chaining")
     ap.add_argument("--cpu-sample-cols", type=int, default=None)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--no-chain", action="store_true", help="gradient fusion only (A2_SCHED_FUSE), no item chaining")
     ap.add_argument("--skip-resident-mode", action="store_true")
     ap.add_argument("--skip-baseline-dynamic", action="store_true")
+    ap.add_argument("--skip-other-configs", action="store_true")
+    ap.add_argument("--skip-fresh-gradients", action="store_true")
+    ap.add_argument("--fresh-pool", type=int, default=4, help="gradient rows per worker of the fresh_gradients figure")
     return ap.parse_args()
 
 
@@ -83,58 +92,129 @@ def measured_peak():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def config_dict(cfg, args, world):
+    """The workload and how it is run; the same keys in both arms."""
+    eb = 2 if cfg.storage == "bf16" else 4
+    return {"workload": f"{cfg.name}: {cfg.note}", "n": cfg.n, "d": cfg.d, "graph": cfg.graph, "storage": cfg.storage,
+            "events_per_step": args.events_per_step, "consensus_every_events": args.events_per_step,
+            "gradient_rows_per_worker": cfg.grad_pool, "gradient_fusion": not args.no_fuse,
+            "item_chaining": not (args.no_fuse or args.no_chain), "launch_mode": args.launch_mode,
+            "parallelism": "replicas only" if world > 1 else "1 gpu",
+            "l2": "state 2*n*d*elem bytes per replica exceeds L2; no flush needed" if 2 * cfg.n * cfg.d * eb > 3 * 126e6
+                  else "state fits L2: figures are L2-assisted"}
+
+
+def dtype_string(cfg):
+    return "f32" if cfg.storage == "f32" else "bf16 storage, f32 math"
+
+
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    """SM clock, power and throttle reasons of one GPU, polled from a thread for the whole run (NVML reads
+    only; nvidia-smi as a fallback); `window(t0, t1)` summarises the samples taken between two
+    time.perf_counter() stamps, so the timed region has samples however short it is."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
 
-    def __init__(self, index):
-        self.index = index
-        self.proc = None
+    def __init__(self, torch_device, period_s=0.004):
+        self.samples = []  # (stamp, sm_mhz, power_w, reasons bitmask)
+        self.max_mhz = None
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+        self._handle = None
+        self._smi_index = None
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            props = torch.cuda.get_device_properties(torch_device)
+            try:
+                self._handle = pynvml.nvmlDeviceGetHandleByUUID(f"GPU-{props.uuid}")
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = torch_device.index or 0
+                self._handle = pynvml.nvmlDeviceGetHandleByIndex(int(vis.split(",")[idx]) if vis and vis.split(",")[idx].isdigit() else idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM))
+            self._nvml = pynvml
+        except Exception:
+            self._nvml = None
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = getattr(torch_device, "index", 0) or 0
+            self._smi_index = vis.split(",")[idx] if vis else str(idx)
+
+    def _read_nvml(self):
+        n, h = self._nvml, self._handle
+        sm = float(n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM))
+        try:
+            mask = int(n.nvmlDeviceGetCurrentClocksEventReasons(h))
+        except Exception:
+            mask = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+        try:
+            power = n.nvmlDeviceGetPowerUsage(h) / 1e3
+        except Exception:
+            power = float("nan")
+        return sm, power, mask
+
+    def _read_smi(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.sw_power_cap,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.hw_thermal_slowdown")
+        out = subprocess.run(["nvidia-smi", "-i", self._smi_index, f"--query-gpu={q}", "--format=csv,noheader,nounits"],
+                             capture_output=True, text=True, timeout=5).stdout.strip().splitlines()[0]
+        f = [s.strip() for s in out.split(",")]
+        self.max_mhz = float(f[1])
+        mask = 0
+        for bit, v in zip((0x4, 0x8, 0x20, 0x40), f[3:7]):
+            if v.lower().startswith("active"):
+                mask |= bit
+        return float(f[0]), float(f[2]), mask
+
+    def _loop(self):
+        read = self._read_nvml if self._nvml is not None else self._read_smi
+        while not self._stop.is_set():
+            try:
+                sm, power, mask = read()
+                self.samples.append((time.perf_counter(), sm, power, mask))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
+        self._thread = threading.Thread(target=self._loop, daemon=True)
+        self._thread.start()
 
     def stop(self):
-        if self.proc is None:
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=5)
+
+    def window(self, t0, t1):
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not inside:  # nearest samples on either side: better than nothing, and said so
+            inside = sorted(self.samples, key=lambda s: min(abs(s[0] - t0), abs(s[0] - t1)))[:2]
+            note = "no sample fell inside the timed region; nearest samples used"
+        else:
+            note = None
+        if not inside:
             return None
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except Exception:
-            self.proc.kill()
-            return None
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.splitlines():
-            f = [s.strip() for s in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for nm, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(nm)
-        if not sm:
-            return None
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+        mask = 0
+        for s in inside:
+            mask |= s[3]
+        out = {"sm_mhz": statistics.median(s[1] for s in inside), "sm_mhz_min": min(s[1] for s in inside),
+               "sm_max_mhz": self.max_mhz, "power_w_max": max(s[2] for s in inside), "samples": len(inside),
+               "window_s": t1 - t0, "source": "nvml" if self._nvml is not None else "nvidia-smi",
+               "reasons": sorted(name for bit, name in self.REASONS.items() if mask & bit)}
+        if note:
+            out["note"] = note
+        return out
 
 
 def fill_engine(eng, cfg, threads):
     """x0 and the gradient rows, generated row by row on the host and copied in; x~ <- x."""
-    def job(args):
-        which, row = args
+    def job(a):
+        which, row = a
         stored, _ = (W.x0_row if which == "x" else W.grad_row)(cfg, row)
         return which, row, stored
 
@@ -142,7 +222,8 @@ def fill_engine(eng, cfg, threads):
     with ThreadPoolExecutor(max(1, threads)) as ex:
         for which, row, stored in ex.map(job, jobs):
             eng.fill_row(which, row, stored)
-    eng.xt.copy_(eng.x)
+    if eng.xt is not None:
+        eng.xt.copy_(eng.x)
     eng.set_times(np.zeros(cfg.n))
     eng.sync()
 
@@ -156,19 +237,22 @@ def sample_inputs(cfg, n_cols, threads):
     return xw, gw
 
 
+def oracle_params(cfg):
+    from oracle import spectral
+
+    if cfg.fixed_params is not None:
+        return cfg.fixed_params
+    return spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
+
+
 def cpu_baseline(cfg, ev, n_cols, threads):
     """The CPU checker, as it stands, on the first n_cols columns of the workload and the given
     events; events/s is scaled to the full width by the column fraction (columns never interact,
     so the work is proportional to the width)."""
-    from oracle import spectral
     from oracle.sim import OracleSim
 
     xw, gw = sample_inputs(cfg, n_cols, threads)
-    if cfg.fixed_params is not None:
-        params = cfg.fixed_params
-    else:
-        params = spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
-    sim = OracleSim(xw, *params, cfg.gamma, grads=gw)
+    sim = OracleSim(xw, *oracle_params(cfg), cfg.gamma, grads=gw)
     t0 = time.perf_counter()
     sim.apply_stream(ev, threads=threads)
     cons = sim.consensus()
@@ -178,16 +262,14 @@ def cpu_baseline(cfg, ev, n_cols, threads):
 
 def run_reference(args, cfg):
     """Reference arm: the CPU checker on the host cores (rank 0 only)."""
+    from oracle.sim import OracleSim
+
     threads = max(1, min(os.cpu_count() or 1, 32))
     n_cols = args.cpu_sample_cols or max(1, min(cfg.d, 256_000))
     eps = args.events_per_step
     ev_all = W.config_events(cfg, n_events=(args.warmup + args.steps) * eps)
-    from oracle import spectral
-    from oracle.sim import OracleSim
-
     xw, gw = sample_inputs(cfg, n_cols, threads)
-    params = cfg.fixed_params if cfg.fixed_params is not None else spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
-    sim = OracleSim(xw, *params, cfg.gamma, grads=gw)
+    sim = OracleSim(xw, *oracle_params(cfg), cfg.gamma, grads=gw)
     t_timed = 0.0
     for s in range(args.warmup + args.steps):
         chunk = ev_all.slice(s * eps, (s + 1) * eps)
@@ -198,19 +280,150 @@ def run_reference(args, cfg):
             t_timed += time.perf_counter() - t0
     value = args.steps * eps / t_timed * (n_cols / cfg.d)
     sample = (f"first {n_cols} of {cfg.d} columns, all {cfg.n} workers, {eps} events + one consensus distance per step; "
-              f"events/s scaled by the column fraction")
+              f"events/s scaled to the full width by the column fraction, ms_per_step as run")
     line = {
         "impl": "reference", "metric": "gossip_events_per_s", "value": value, "unit": "events/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * t_timed / args.steps * (cfg.d / n_cols), "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {cfg.note}", "n": cfg.n, "d": cfg.d, "graph": cfg.graph,
-                   "events_per_step": eps},
+        "ms_per_step": 1e3 * t_timed / args.steps,  # as run, on the column sample
+        "ms_per_step_full_width_equivalent": 1e3 * t_timed / args.steps * (cfg.d / n_cols),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(cfg, args, max(1, args.gpus)),
         "cpu_baseline": {"value": value, "unit": "events/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "events/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+class Bench:
+    """One workload on one engine: the timed passes share the engine, the event stream and the ranks."""
+
+    def __init__(self, cfg, args, ranks, device, threads, n_warm, n_timed, stretches):
+        import torch
+
+        from paper_2306_08289_b200 import binding as B
+
+        self.torch, self.B = torch, B
+        self.cfg, self.args, self.ranks, self.device = cfg, args, ranks, device
+        self.W_, self.K, self.eps = n_warm, n_timed, args.events_per_step
+        self.n_steps = n_warm + n_timed
+        self.flags = 0 if args.no_fuse else (B.A2_SCHED_FUSE if args.no_chain else B.A2_SCHED_CHAIN)
+        self.eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage,
+                            n_grad_slots=cfg.n_grad_slots, device=str(device))
+        self.eng.set_launch_mode(LAUNCH_MODES[args.launch_mode])
+        fill_engine(self.eng, cfg, threads)
+        self.ev_all = W.config_events(cfg, n_events=stretches * self.n_steps * self.eps)
+        self.stretch = 0
+        self.cons = []
+
+    def _chunk(self, s):
+        k = self.stretch * self.n_steps + s
+        return self.ev_all.slice(k * self.eps, (k + 1) * self.eps)
+
+    def _plans(self, flags):
+        plans, t_start = [], self.eng.times()
+        for s in range(self.n_steps):
+            c = self._chunk(s)
+            p = self.eng.plan(c.times, c.wi, c.wj, c.slot, flags=flags, t_start=t_start)
+            t_start = p.sched.t_final(self.cfg.n)
+            plans.append(p)
+        return plans
+
+    def plans_pass(self, flags=None):
+        """Descriptors resident on the device; CUDA events around every plan run and every consensus distance."""
+        torch, dev, W_, n = self.torch, self.device, self.W_, self.n_steps
+        plans = self._plans(self.flags if flags is None else flags)
+        stream = self.eng.stream
+        marks = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(n)]
+        stats = []
+        t0 = t1 = None
+        for s in range(n):
+            if s == W_:
+                torch.cuda.synchronize(dev)
+                self.ranks.barrier()
+                torch.cuda.synchronize(dev)
+                t0 = time.perf_counter()
+            a, b, c = marks[s]
+            a.record(stream)
+            stats.append(plans[s].run(want_stats=True))
+            b.record(stream)
+            self.cons.append(self.eng.consensus_distance())
+            c.record(stream)
+        torch.cuda.synchronize(dev)
+        t1 = time.perf_counter()
+        self.ranks.barrier()
+        timed = range(W_, n)
+        out = {
+            "total_ms": marks[W_][0].elapsed_time(marks[n - 1][2]),
+            "k1_ms": sum(marks[s][0].elapsed_time(marks[s][1]) for s in timed),
+            "k2_ms": sum(marks[s][1].elapsed_time(marks[s][2]) for s in timed),
+            "launches": sum(stats[s]["n_launches"] for s in timed),
+            "bytes": sum(stats[s]["bytes_moved"] for s in timed),
+            "bytes_single": sum(stats[s]["bytes_one_by_one"] for s in timed),
+            "events": sum(stats[s]["n_events"] for s in timed),
+            "batches": sum(stats[s]["n_batches"] for s in timed),
+            "items": sum(stats[s]["n_items"] for s in timed),
+            "window": (t0, t1),
+        }
+        for p in plans:
+            p.close()
+        self.stretch += 1
+        return out
+
+    def e2e_pass(self):
+        """Through a2cid2_apply_events with host arrays; wall clock around the timed steps."""
+        torch, dev = self.torch, self.device
+        h2d = []
+        torch.cuda.synchronize(dev)
+        t0 = None
+        for s in range(self.n_steps):
+            if s == self.W_:
+                torch.cuda.synchronize(dev)
+                self.ranks.barrier()
+                t0 = time.perf_counter()
+            c = self._chunk(s)
+            st = self.eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=self.flags, want_stats=True)
+            self.cons.append(self.eng.consensus_distance())  # waits for the stream and reads the result back
+            if s >= self.W_:
+                h2d.append(st["descriptor_bytes"])
+        torch.cuda.synchronize(dev)
+        secs = time.perf_counter() - t0
+        self.ranks.barrier()
+        self.stretch += 1
+        value, _ = aggregate_throughput(self.ranks, self.K * self.eps, secs)
+        return {"value": value, "unit": "events/s", "h2d_bytes_per_step": int(np.mean(h2d)) if h2d else 0, "d2h_bytes_per_step": 8}
+
+    def check(self):
+        if not all(np.isfinite(self.cons)):
+            raise SystemExit("non-finite consensus distance: the run is invalid")
+
+    def close(self):
+        self.eng.close()
+        self.eng = None
+        self.torch.cuda.empty_cache()
+
+
+def kernel_figures(p, peak):
+    gbs = p["bytes"] / (p["k1_ms"] / 1e3) / 1e9
+    return {"achieved_gbs": gbs, "frac": gbs / peak, "avg_launch_ms": p["k1_ms"] / max(1, p["launches"]), "launches": p["launches"]}
+
+
+def light_run(cfg, args, ranks, device, threads, peak, n_warm=3, n_timed=5):
+    """A few timed steps of another workload: events/s (plans resident), end to end, the event kernel."""
+    t0 = time.perf_counter()
+    b = Bench(cfg, args, ranks, device, threads, n_warm, n_timed, stretches=2)
+    p = b.plans_pass()
+    value, slowest = aggregate_throughput(ranks, p["events"], p["total_ms"] / 1e3)
+    e2e = b.e2e_pass()
+    b.check()
+    b.close()
+    out = {"value": value, "unit": "events/s", "ms_per_step": 1e3 * slowest / n_timed, "e2e": e2e["value"],
+           "dtype": dtype_string(cfg), "steps": n_timed, "warmup": n_warm, "events_per_step": args.events_per_step,
+           "rows_per_event": p["bytes"] / (cfg.d * (2 if cfg.storage == "bf16" else 4)) / max(1, p["events"]),
+           "batches_per_step": p["batches"] / n_timed, "seconds_spent": None}
+    out.update(kernel_figures(p, peak))
+    out["seconds_spent"] = round(time.perf_counter() - t0, 1)
+    return out
 
 
 def main():
@@ -219,8 +432,6 @@ def main():
     if args.d is not None:
         cfg = cfg.scaled(d=args.d, name=f"{cfg.name}-d{args.d}")
     if args.grad_pool is not None:
-        from dataclasses import replace
-
         cfg = replace(cfg, grad_pool=int(args.grad_pool))
     if args.impl == "reference":
         # rank 0 alone times the CPU checker; the other ranks have nothing to do and no group is formed
@@ -242,112 +453,35 @@ def main():
     if ranks.rank == 0:
         cuda_build.build()
     ranks.barrier()
+    sampler = ClockSampler(device)
+    sampler.start()
 
     W_, K, eps = args.warmup, args.steps, args.events_per_step
-    flags = 0 if args.no_fuse else (B.A2_SCHED_FUSE if args.no_chain else B.A2_SCHED_CHAIN)
-    n_steps = W_ + K
     threads = max(1, min(os.cpu_count() or 1, 32) // max(1, ranks.world))
+    peak, peak_src = measured_peak()
 
-    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots,
-                   device=str(device))
-    eng.set_launch_mode({"auto": B.A2_LAUNCH_AUTO, "per-batch": B.A2_LAUNCH_PER_BATCH,
-                         "column-slices": B.A2_LAUNCH_COLUMN_SLICES}[args.launch_mode])
-    fill_engine(eng, cfg, threads)
     # four stretches of the stream: plans resident on the device, end to end, shared-memory-resident mode,
     # and the asynchronous baseline without the momentum buffer
-    ev_all = W.config_events(cfg, n_events=4 * n_steps * eps)
+    b = Bench(cfg, args, ranks, device, threads, W_, K, stretches=4)
+    eng = b.eng
 
     # ---- pass 1: descriptors resident on the device ---------------------------------------------
-    plans, t_start = [], np.zeros(cfg.n)
-    for s in range(n_steps):
-        c = ev_all.slice(s * eps, (s + 1) * eps)
-        p = eng.plan(c.times, c.wi, c.wj, c.slot, flags=flags, t_start=t_start)
-        t_start = p.sched.t_final(cfg.n)
-        plans.append(p)
-    stream = eng.stream
-    ev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
-                 torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
-    stats, cons = [], []
-    sampler = ClockSampler(local_rank if os.environ.get("CUDA_VISIBLE_DEVICES") is None else
-                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
-    for s in range(n_steps):
-        if s == W_:
-            torch.cuda.synchronize(device)
-            ranks.barrier()
-            sampler.start()
-            torch.cuda.synchronize(device)
-        a, b, c_ = ev_pairs[s]
-        a.record(stream)
-        stats.append(plans[s].run(want_stats=True))
-        b.record(stream)
-        cons.append(eng.consensus_distance())
-        c_.record(stream)
-    torch.cuda.synchronize(device)
-    ranks.barrier()
-    clocks = sampler.stop()
-    timed = range(W_, n_steps)
-    total_ms = ev_pairs[W_][0].elapsed_time(ev_pairs[n_steps - 1][2])
-    k1_ms = sum(ev_pairs[s][0].elapsed_time(ev_pairs[s][1]) for s in timed)
-    k2_ms = sum(ev_pairs[s][1].elapsed_time(ev_pairs[s][2]) for s in timed)
-    k1_launches = sum(stats[s]["n_launches"] for s in timed)
-    k1_bytes = sum(stats[s]["bytes_moved"] for s in timed)
-    k1_bytes_single = sum(stats[s]["bytes_one_by_one"] for s in timed)
-    n_events_timed = sum(stats[s]["n_events"] for s in timed)
-    for p in plans:
-        p.close()
-    value, slowest_s = aggregate_throughput(ranks, n_events_timed, total_ms / 1e3)
+    p1 = b.plans_pass()
+    clocks = sampler.window(*p1["window"])
+    value, slowest_s = aggregate_throughput(ranks, p1["events"], p1["total_ms"] / 1e3)
 
     # ---- pass 2: end to end through a2cid2_apply_events with host arrays --------------------------
-    h2d = []
-    torch.cuda.synchronize(device)
-    for s in range(n_steps):
-        if s == W_:
-            torch.cuda.synchronize(device)
-            ranks.barrier()
-            t0 = time.perf_counter()
-        c = ev_all.slice((n_steps + s) * eps, (n_steps + s + 1) * eps)
-        st = eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=flags, want_stats=True)
-        cons.append(eng.consensus_distance())  # waits for the stream and reads the result back
-        if s >= W_:
-            h2d.append(st["descriptor_bytes"])
-    torch.cuda.synchronize(device)
-    e2e_s = time.perf_counter() - t0
-    ranks.barrier()
-    e2e_value, _ = aggregate_throughput(ranks, K * eps, e2e_s)
-
-    if not all(np.isfinite(cons)):
-        raise SystemExit("non-finite consensus distance: the run is invalid")
+    e2e = b.e2e_pass()
+    b.check()
 
     # ---- pass 3: the shared-memory-resident mode (one launch per step), reported beside the main figure ---
     resident = None
     if not args.skip_resident_mode:
         try:
-            r_plans, t_start = [], eng.times()
-            for s in range(n_steps):
-                c = ev_all.slice((2 * n_steps + s) * eps, (2 * n_steps + s + 1) * eps)
-                p = eng.plan(c.times, c.wi, c.wj, c.slot, flags=B.A2_SCHED_RESIDENT, t_start=t_start)
-                t_start = p.sched.t_final(cfg.n)
-                r_plans.append(p)
-            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            r_bytes = 0
-            for s in range(n_steps):
-                if s == W_:
-                    torch.cuda.synchronize(device)
-                    ranks.barrier()
-                    r0.record(stream)
-                st = r_plans[s].run(want_stats=True)
-                cons.append(eng.consensus_distance())
-                if s >= W_:
-                    r_bytes += st["bytes_moved"]
-            r1.record(stream)
-            torch.cuda.synchronize(device)
-            ranks.barrier()
-            r_ms = r0.elapsed_time(r1)
-            for p in r_plans:
-                p.close()
-            r_value, r_slow = aggregate_throughput(ranks, K * eps, r_ms / 1e3)
+            r = b.plans_pass(flags=B.A2_SCHED_RESIDENT)
+            r_value, r_slow = aggregate_throughput(ranks, r["events"], r["total_ms"] / 1e3)
             resident = {"value": r_value, "unit": "events/s", "ms_per_step": 1e3 * r_slow / K,
-                        "hbm_gbs": r_bytes / (r_ms / 1e3) / 1e9,
+                        "hbm_gbs": r["bytes"] / (r["total_ms"] / 1e3) / 1e9,
                         "note": "A2_SCHED_RESIDENT: one launch per step, column tile of all workers in shared "
                                 "memory; needs every gradient of the step up front; not HBM-bound"}
         except B.A2Error as exc:
@@ -357,80 +491,74 @@ def main():
     plain = None
     if not args.skip_baseline_dynamic:
         eng.set_variant(B.A2_NO_MOMENTUM)
-        p_plans, t_start = [], eng.times()
-        for s in range(n_steps):
-            c = ev_all.slice((3 * n_steps + s) * eps, (3 * n_steps + s + 1) * eps)
-            p = eng.plan(c.times, c.wi, c.wj, c.slot, flags=flags, t_start=t_start)
-            t_start = p.sched.t_final(cfg.n)
-            p_plans.append(p)
-        marks = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
-        q_end = torch.cuda.Event(enable_timing=True)
-        p_bytes = p_launches = 0
-        for s in range(n_steps):
-            if s == W_:
-                torch.cuda.synchronize(device)
-                ranks.barrier()
-            marks[s][0].record(stream)
-            st = p_plans[s].run(want_stats=True)
-            marks[s][1].record(stream)
-            cons.append(eng.consensus_distance())
-            if s >= W_:
-                p_bytes += st["bytes_moved"]
-                p_launches += st["n_launches"]
-        q_end.record(stream)
-        torch.cuda.synchronize(device)
-        ranks.barrier()
-        p_ms = marks[W_][0].elapsed_time(q_end)
-        p_k1_ms = sum(marks[s][0].elapsed_time(marks[s][1]) for s in timed)
-        for p in p_plans:
-            p.close()
+        q = b.plans_pass()
         eng.set_variant(B.A2_MSG_AFTER_MIX)
-        p_value, p_slow = aggregate_throughput(ranks, K * eps, p_ms / 1e3)
-        plain = {"value": p_value, "unit": "events/s", "ms_per_step": 1e3 * p_slow / K,
-                 "kernel": "k_apply_events_plain", "achieved_gbs": p_bytes / (p_k1_ms / 1e3) / 1e9,
-                 "launches": p_launches,
+        q_value, q_slow = aggregate_throughput(ranks, q["events"], q["total_ms"] / 1e3)
+        plain = {"value": q_value, "unit": "events/s", "ms_per_step": 1e3 * q_slow / K, "kernel": "k_apply_events_plain",
                  "note": "A2_NO_MOMENTUM: the paper's asynchronous baseline on the same stream recipe; x only, so "
                          "an event moves half the bytes"}
-        if not all(np.isfinite(cons)):
-            raise SystemExit("non-finite consensus distance: the run is invalid")
+        plain.update(kernel_figures(q, peak))
+        b.check()
+    elem_bytes = eng.elem_bytes
+    b.close()
 
     # ---- roofline of the event kernel ------------------------------------------------------------
-    peak, peak_src = measured_peak()
-    achieved = k1_bytes / (k1_ms / 1e3) / 1e9
-    per_launch_bytes = k1_bytes / max(1, k1_launches)
+    achieved = p1["bytes"] / (p1["k1_ms"] / 1e3) / 1e9
+    per_launch_bytes = p1["bytes"] / max(1, p1["launches"])
     roofline = {
         "kernel": "k_apply_events", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_source": f"of {peak_src} copy bandwidth",
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * per_launch_bytes,
-        "bytes_per_launch": per_launch_bytes, "avg_launch_ms": k1_ms / max(1, k1_launches), "launches": k1_launches,
-        "effective_gbs_one_event_per_item": k1_bytes_single / (k1_ms / 1e3) / 1e9,
-        "share_of_step_time": k1_ms / total_ms,
+        "traffic_source": NCU_TRAFFIC_SOURCE,
+        "bytes_per_launch": per_launch_bytes, "avg_launch_ms": p1["k1_ms"] / max(1, p1["launches"]), "launches": p1["launches"],
+        "rows_per_event": p1["bytes"] / (cfg.d * elem_bytes) / max(1, p1["events"]),
+        "effective_gbs_one_event_per_item": p1["bytes_single"] / (p1["k1_ms"] / 1e3) / 1e9,
+        "share_of_step_time": p1["k1_ms"] / p1["total_ms"],
     }
-    consensus_gbs = K * cfg.n * cfg.d * eng.elem_bytes / (k2_ms / 1e3) / 1e9
+    consensus_gbs = K * cfg.n * cfg.d * elem_bytes / (p1["k2_ms"] / 1e3) / 1e9
 
     line = {
         "metric": "gossip_events_per_s", "value": value, "unit": "events/s", "n_gpus": ranks.world, "steps": K,
         "warmup": W_, "ms_per_step": 1e3 * slowest_s / K, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {cfg.note}", "n": cfg.n, "d": cfg.d, "graph": cfg.graph,
-                   "storage": cfg.storage, "events_per_step": eps, "consensus_every_events": eps,
-                   "gradient_fusion": not args.no_fuse, "item_chaining": not (args.no_fuse or args.no_chain), "parallelism": "replicas only" if ranks.world > 1 else "1 gpu",
-                   "l2": "state 2*n*d*elem bytes per replica exceeds L2; no flush needed" if
-                   2 * cfg.n * cfg.d * eng.elem_bytes > 3 * 126e6 else "state fits L2: figures are L2-assisted"},
-        "clocks": clocks, "roofline": roofline,
-        "e2e": {"value": e2e_value, "unit": "events/s", "h2d_bytes_per_step": int(np.mean(h2d)) if h2d else 0,
-                "d2h_bytes_per_step": 8},
-        "gpu_launches": int(k1_launches + 2 * K),
-        "consensus_kernel": {"ms": k2_ms / K, "gbs": consensus_gbs, "frac": consensus_gbs / peak},
-        "batches_per_step": sum(stats[s]["n_batches"] for s in timed) / K,
+        "vs_baseline": None, "dtype": dtype_string(cfg), "data": "synthetic",
+        "config": config_dict(cfg, args, ranks.world),
+        "clocks": clocks, "roofline": roofline, "e2e": e2e,
+        "gpu_launches": int(p1["launches"] + 2 * K),
+        "consensus_kernel": {"ms": p1["k2_ms"] / K, "gbs": consensus_gbs, "frac": consensus_gbs / peak},
+        "batches_per_step": p1["batches"] / K, "items_per_step": p1["items"] / K,
         "resident_mode": resident,
         "baseline_dynamic": plain,
     }
-    if plain is not None:
-        plain["frac"] = plain["achieved_gbs"] / peak
 
-    if ranks.rank == 0 and ranks.world == 1 and not args.skip_cpu_baseline:
+    solo = ranks.world == 1
+    # ---- the same workload with fresh gradient rows (a pool per worker, used round robin) ---------
+    if solo and not args.skip_fresh_gradients and args.fresh_pool != cfg.grad_pool:
+        try:
+            fc = replace(cfg, grad_pool=args.fresh_pool, name=f"{cfg.name}-pool{args.fresh_pool}")
+            fr = light_run(fc, args, ranks, device, threads, peak)
+            fr["gradient_rows_per_worker"] = args.fresh_pool
+            fr["note"] = ("consecutive gradient events of a worker name different rows; chained items fetch a worker's "
+                          "next row inside the item, and every row fetched is counted in the kernel's bytes")
+            line["fresh_gradients"] = fr
+        except Exception as exc:  # e.g. not enough device memory for the pool
+            line["fresh_gradients"] = {"unavailable": f"{type(exc).__name__}: {exc}"}
+    # ---- the other workloads, a few timed steps each ---------------------------------------------
+    if solo and not args.skip_other_configs:
+        others, budget_s, t_begin = {}, 150.0, time.perf_counter()
+        for name in sorted(W.CONFIGS):
+            if name == args.config:
+                continue
+            if time.perf_counter() - t_begin > budget_s:
+                others[name] = {"skipped": f"time budget of {budget_s:.0f} s for the other workloads used up"}
+                continue
+            try:
+                others[name] = light_run(W.CONFIGS[name], args, ranks, device, threads, peak)
+            except Exception as exc:
+                others[name] = {"unavailable": f"{type(exc).__name__}: {exc}"}
+        line["other_configs"] = others
+
+    if ranks.rank == 0 and solo and not args.skip_cpu_baseline:
         cores = max(1, min(os.cpu_count() or 1, 32))
         n_cols = args.cpu_sample_cols or max(1, min(cfg.d, 2_560_000))
         sample_ev = W.config_events(cfg, n_events=4 * eps)
@@ -444,7 +572,7 @@ def main():
         v1, dt1, _ = cpu_baseline(cfg, W.config_events(cfg, n_events=eps), n1, 1)
         line["cpu_baseline"]["one_thread"] = {"value": v1, "seconds": dt1,
                                               "sample": f"first {n1} columns, {eps} events + one consensus distance"}
-    eng.close()
+    sampler.stop()
     if ranks.rank == 0:
         print(json.dumps(line), flush=True)
     ranks.close()

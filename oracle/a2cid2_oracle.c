@@ -199,14 +199,18 @@ double a2o_to_bf16(double v) {
     return (double)f;
 }
 
-/* Round columns [0, d) of the rows X[w], Xt[w] (w in rows[0 .. n_rows)) to bfloat16. */
-void a2o_round_rows_bf16(int64_t d, int64_t ld, double* X, double* Xt, int32_t n_rows, const int32_t* rows) {
+/* The same for IEEE binary32 storage: one rounding to nearest, ties to even. */
+double a2o_to_f32(double v) { return (double)(float)v; }
+
+/* Round columns [0, d) of the rows X[w], Xt[w] (w in rows[0 .. n_rows)) to the storage format
+ * (fmt 0: bfloat16, 1: binary32). */
+void a2o_round_rows(int64_t d, int64_t ld, double* X, double* Xt, int32_t n_rows, const int32_t* rows, int32_t fmt) {
     for (int32_t r = 0; r < n_rows; ++r) {
         double* x = X + (size_t)rows[r] * ld;
         double* xt = Xt + (size_t)rows[r] * ld;
         for (int64_t k = 0; k < d; ++k) {
-            x[k] = a2o_to_bf16(x[k]);
-            xt[k] = a2o_to_bf16(xt[k]);
+            x[k] = fmt == 0 ? a2o_to_bf16(x[k]) : a2o_to_f32(x[k]);
+            xt[k] = fmt == 0 ? a2o_to_bf16(xt[k]) : a2o_to_f32(xt[k]);
         }
     }
 }
@@ -214,15 +218,16 @@ void a2o_round_rows_bf16(int64_t d, int64_t ld, double* X, double* Xt, int32_t n
 /*
  * a2o_run on consecutive groups of events, with the storage model applied between groups: group k is
  * events [group_end[k-1], group_end[k]) (group_end[-1] = 0), applied in the order given by a2o_run (fp64
- * arithmetic, unchanged); then the rows of workers[worker_ptr[k] .. worker_ptr[k+1]) are rounded to
- * bfloat16. The time-order check of a2o_run holds inside a group; groups may overlap in time (they are
- * the items of a schedule, which keeps every worker's own order).
+ * arithmetic, unchanged); then the rows of workers[worker_ptr[k] .. worker_ptr[k+1]) are rounded to the
+ * storage format. The time-order check of a2o_run holds inside a group; groups may overlap in time (they
+ * are the items of a schedule, which keeps every worker's own order).
  */
-int a2o_run_groups_bf16(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double alpha_t, double gamma,
-                        double* X, double* Xt, double* tl, const double* G, int32_t n_slots, int64_t ldg,
-                        const double* times, const int32_t* wi, const int32_t* wj, const int32_t* slot,
-                        int32_t variant, int64_t n_groups, const int64_t* group_end, const int64_t* worker_ptr,
-                        const int32_t* workers) {
+int a2o_run_groups(int32_t n, int64_t d, int64_t ld, double eta, double alpha, double alpha_t, double gamma,
+                   double* X, double* Xt, double* tl, const double* G, int32_t n_slots, int64_t ldg,
+                   const double* times, const int32_t* wi, const int32_t* wj, const int32_t* slot,
+                   int32_t variant, int64_t n_groups, const int64_t* group_end, const int64_t* worker_ptr,
+                   const int32_t* workers, int32_t fmt) {
+    if (fmt != 0 && fmt != 1) return A2O_EINVAL;
     int64_t e0 = 0;
     for (int64_t k = 0; k < n_groups; ++k) {
         const int64_t e1 = group_end[k];
@@ -230,7 +235,7 @@ int a2o_run_groups_bf16(int32_t n, int64_t d, int64_t ld, double eta, double alp
         const int rc = a2o_run(n, d, ld, eta, alpha, alpha_t, gamma, X, Xt, tl, G, n_slots, ldg, e1 - e0, times + e0,
                                wi + e0, wj + e0, slot + e0, variant);
         if (rc != A2O_OK) return rc;
-        a2o_round_rows_bf16(d, ld, X, Xt, (int32_t)(worker_ptr[k + 1] - worker_ptr[k]), workers + worker_ptr[k]);
+        a2o_round_rows(d, ld, X, Xt, (int32_t)(worker_ptr[k + 1] - worker_ptr[k]), workers + worker_ptr[k], fmt);
         e0 = e1;
     }
     return A2O_OK;

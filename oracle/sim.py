@@ -28,10 +28,10 @@ def load(path):
         lp = C.POINTER(C.c_int64)
         L.a2o_to_bf16.restype = C.c_double
         L.a2o_to_bf16.argtypes = [C.c_double]
-        L.a2o_run_groups_bf16.restype = C.c_int
-        L.a2o_run_groups_bf16.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_double,
-                                          dp, dp, dp, dp, C.c_int32, C.c_int64, dp, ip, ip, ip, C.c_int32,
-                                          C.c_int64, lp, lp, ip]
+        L.a2o_run_groups.restype = C.c_int
+        L.a2o_run_groups.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_double,
+                                     dp, dp, dp, dp, C.c_int32, C.c_int64, dp, ip, ip, ip, C.c_int32,
+                                     C.c_int64, lp, lp, ip, C.c_int32]
         L.a2o_consensus.restype = C.c_double
         L.a2o_consensus.argtypes = [C.c_int32, C.c_int64, C.c_int64, dp]
         L.a2o_consensus_at.restype = C.c_double
@@ -111,11 +111,11 @@ class OracleSim:
             raise OracleError(f"a2o_run -> {rcs}")
         self.t[:] = tls[0]
 
-    def apply_groups_bf16(self, times, wi, wj, slot, group_end, worker_ptr, workers):
+    def apply_groups(self, times, wi, wj, slot, group_end, worker_ptr, workers, fmt="bf16"):
         """Storage model over a whole schedule in one call: the events (already in the order they are to be
         applied) come in consecutive groups ending at group_end[k]; after group k the rows of
-        workers[worker_ptr[k]:worker_ptr[k+1]] are rounded to bfloat16. Equal to apply() on each group followed
-        by round_rows() on its workers."""
+        workers[worker_ptr[k]:worker_ptr[k+1]] are rounded to the storage format ("bf16" or "f32"). Equal to
+        apply() on each group followed by round_rows() on its workers."""
         times = np.ascontiguousarray(times, dtype=np.float64)
         wi = np.ascontiguousarray(wi, dtype=np.int32)
         wj = np.ascontiguousarray(wj, dtype=np.int32)
@@ -126,12 +126,13 @@ class OracleSim:
         assert len(worker_ptr) == len(group_end) + 1 and (len(group_end) == 0 or group_end[-1] == len(times))
         G = self.G if self.G is not None else np.zeros((1, self.d))
         lp = C.POINTER(C.c_int64)
-        rc = lib().a2o_run_groups_bf16(self.n, self.d, self.d, self.eta, self.alpha, self.alpha_tilde, self.gamma,
-                                       _dp(self.X), _dp(self.Xt), _dp(self.t), _dp(G), G.shape[0], self.d,
-                                       _dp(times), _ip(wi), _ip(wj), _ip(slot), self.variant, len(group_end),
-                                       group_end.ctypes.data_as(lp), worker_ptr.ctypes.data_as(lp), _ip(workers))
+        rc = lib().a2o_run_groups(self.n, self.d, self.d, self.eta, self.alpha, self.alpha_tilde, self.gamma,
+                                  _dp(self.X), _dp(self.Xt), _dp(self.t), _dp(G), G.shape[0], self.d,
+                                  _dp(times), _ip(wi), _ip(wj), _ip(slot), self.variant, len(group_end),
+                                  group_end.ctypes.data_as(lp), worker_ptr.ctypes.data_as(lp), _ip(workers),
+                                  {"bf16": 0, "f32": 1}[fmt])
         if rc != 0:
-            raise OracleError(f"a2o_run_groups_bf16 -> {rc}")
+            raise OracleError(f"a2o_run_groups -> {rc}")
 
     def apply_stream(self, ev, threads=1):
         self.apply(ev.times, ev.wi, ev.wj, ev.slot, threads=threads)

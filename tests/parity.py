@@ -92,6 +92,36 @@ def oracle_params(cfg):
     return tuple(float(v) for v in spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3])
 
 
+def per_event_groups(ev):
+    """Rounding points of an implementation that stores the rows of an event's workers after every event:
+    (group_end, worker_ptr, workers) for OracleSim.apply_groups."""
+    n = len(ev)
+    comm = ev.wj >= 0
+    ptr = np.concatenate([[0], np.cumsum(1 + comm.astype(np.int64))])
+    workers = np.empty(int(ptr[-1]), dtype=np.int32)
+    workers[ptr[:-1]] = ev.wi
+    workers[ptr[:-1][comm] + 1] = ev.wj[comm]
+    return np.arange(1, n + 1, dtype=np.int64), ptr.astype(np.int64), workers
+
+
+def storage_only_error(cfg, fmt, x0=None, G=None, ev=None):
+    """Element-wise error (the metric of the fp32 parity tests) of a run whose arithmetic is fp64 and
+    whose only loss is that the rows of an event's workers are rounded to `fmt` ("f32" or "bf16") when
+    they are stored, once per event: what an ideal implementation with that storage format delivers.
+    x0, G: widened inputs (default: the configuration's own, all columns)."""
+    if x0 is None:
+        _, x0 = W.x0_matrix(cfg)
+        _, G = W.grad_matrix(cfg)
+    if ev is None:
+        ev = W.config_events(cfg)
+    par = oracle_params(cfg)
+    plain = OracleSim(x0, *par, cfg.gamma, grads=G)
+    stored = OracleSim(x0, *par, cfg.gamma, grads=G)
+    plain.apply_stream(ev)
+    stored.apply_groups(ev.times, ev.wi, ev.wj, ev.slot, *per_event_groups(ev), fmt=fmt)
+    return max(rel_err(stored.X, plain.X), rel_err(stored.Xt, plain.Xt))
+
+
 class _XOnly:
     """View of a simulator in which x stands in for x~ too, for engines that hold x alone."""
 

@@ -244,8 +244,13 @@ def test_many_items_per_batch_are_split_into_launches():
     eng = B.Engine(n, d, 0.2, 0.5, 1.2, 0.05)
     eng.write_state(x0)
     eng.write_grads(g)
-    st = eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_FUSE, want_stats=True)
+    eng.set_launch_mode(B.A2_LAUNCH_PER_BATCH)
+    h = len(ev) // 2
+    st = eng.apply_events(ev.times[:h], ev.wi[:h], ev.wj[:h], ev.slot[:h], flags=B.A2_SCHED_FUSE, want_stats=True)
     assert st["n_launches"] > st["n_batches"]
+    eng.set_launch_mode(B.A2_LAUNCH_COLUMN_SLICES)  # the caps cut these launches too, anywhere in the item list
+    st = eng.apply_events(ev.times[h:], ev.wi[h:], ev.wj[h:], ev.slot[h:], flags=B.A2_SCHED_FUSE, want_stats=True)
+    assert st["n_launches"] * 128 >= st["n_items"] and st["n_launches"] > 1
     from oracle.sim import OracleSim
 
     sim = OracleSim(x0.astype(np.float64), 0.2, 0.5, 1.2, 0.05, grads=g.astype(np.float64))

@@ -1,0 +1,288 @@
+"""Every element of the state, at the full sizes of the workloads, against the CPU checker.
+
+The engine runs the workload's whole event stream the way the benchmark does (steps of 500 events,
+chained schedule, every step run whole in the library's default launch mode, a consensus distance after
+every step). The state is kept at a few check points (device copies) and at the end. The checker then
+goes through the same stream on ALL columns, a chunk of columns at a time on all host cores -- columns never
+interact (every step of Algorithm 1 is element-wise over the parameter dimension), so the checker on a
+range of columns is that range of the full run -- and every element of x and x~ at every check point is
+compared with it:
+
+  fp32 rows   max |gpu - ref| / max(|ref|, rms) <= 1e-5, rms = root mean square of the reference row
+              over the chunk's columns (8192 columns of the same distribution: within a percent of the
+              whole row's). Beside it, on every eighth chunk, the same figure for an IDEAL fp32-storage
+              implementation: the checker's fp64 arithmetic with the rows of an event's workers rounded
+              to binary32 after every event. Where that ideal run is itself above 0.5e-5 -- the bar is
+              within a factor two of what the storage format delivers on the stream -- the engine is
+              held to twice the ideal figure instead, and the report says whether 1e-5 was met;
+  bf16 rows   row-wise 2-norm error <= 2e-2 against the plain fp64 run (made on every second chunk, the
+              norm taken over those columns), and every
+              element against the fp64 run with the storage modelled (rows rounded to bf16 where the
+              schedule's items write them back) in bf16 units in the last place, with the histogram of
+              those distances (tests/parity.py states where the bounds come from).
+
+The consensus distance the engine reported after every step is compared with the checker's, summed over
+the chunks (fp32 rows). The checker's share is bounded in time: no new chunk is started after BUDGET_S
+seconds per workload, the chunks are taken in an order that spreads any prefix evenly over the row, and
+the coverage is printed; on the 16-core hosts of this pool all chunks fit.
+"""
+import os
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from oracle.sim import OracleSim
+from paper_2306_08289_b200 import binding as B
+from paper_2306_08289_b200 import workload as W
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+CHUNK_COLS = 8192
+EVENTS_PER_STEP = 500
+BUDGET_S = 200.0
+
+
+def _threads():
+    return max(1, min(32, os.cpu_count() or 1))
+
+
+def _fill_and_keep(eng, cfg):
+    """x0 and the gradient rows in the storage precision, kept on the host and copied to the engine."""
+    dt = np.uint16 if cfg.storage == "bf16" else np.float32
+    x0 = np.empty((cfg.n, cfg.d), dtype=dt)
+    g = np.empty((cfg.n_grad_slots, cfg.d), dtype=dt)
+
+    def job(a):
+        which, row = a
+        stored, _ = (W.x0_row if which == "x" else W.grad_row)(cfg, row)
+        (x0 if which == "x" else g)[row] = stored
+        return which, row
+
+    jobs = [("x", i) for i in range(cfg.n)] + [("g", i) for i in range(cfg.n_grad_slots)]
+    with ThreadPoolExecutor(_threads()) as ex:
+        for which, row in ex.map(job, jobs):
+            eng.fill_row(which, row, (x0 if which == "x" else g)[row])
+    eng.xt.copy_(eng.x)
+    eng.set_times(np.zeros(cfg.n))
+    eng.sync()
+    return x0, g
+
+
+def _step_groups(ev, sched):
+    """The events of a schedule in the order its items apply them (time order inside an item), the end of
+    every item's run of events, and the item's workers: the storage model's rounding points."""
+    t, wi, wj, sl, ends, ptr, flat = [], [], [], [], [], [0], []
+    for k in range(sched.num_items):
+        it = sched.item(k)
+        e, _ = sched.ops(it.first_op, it.n_ops)
+        e = e[np.argsort(ev.times[e], kind="stable")]
+        t.append(ev.times[e]); wi.append(ev.wi[e]); wj.append(ev.wj[e]); sl.append(ev.slot[e])
+        ends.append((ends[-1] if ends else 0) + len(e))
+        flat += it.workers()
+        ptr.append(len(flat))
+    cat = np.concatenate
+    return cat(t), cat(wi), cat(wj), cat(sl), np.array(ends, dtype=np.int64), np.array(ptr, dtype=np.int64), np.array(flat, dtype=np.int32)
+
+
+def _run_engine(eng, cfg, ev, check_steps):
+    """The whole stream in steps; returns per-step consensus distances, device copies of (x, x~) after the
+    steps in check_steps, the per-step event slices and (bf16) the per-step storage-model groups."""
+    n_steps = (len(ev) + EVENTS_PER_STEP - 1) // EVENTS_PER_STEP
+    cons, snaps, slices, groups = [], {}, [], []
+    t_start = np.zeros(cfg.n)
+    for s in range(n_steps):
+        c = ev.slice(s * EVENTS_PER_STEP, (s + 1) * EVENTS_PER_STEP)
+        plan = eng.plan(c.times, c.wi, c.wj, c.slot, flags=B.A2_SCHED_CHAIN, t_start=t_start)
+        t_start = plan.sched.t_final(cfg.n)
+        plan.run()  # whole: the launch mode the library picks, as the benchmark times it
+        if cfg.storage == "bf16":
+            groups.append(_step_groups(c, plan.sched))
+        plan.close()
+        cons.append(eng.consensus_distance())
+        slices.append(c)
+        if s in check_steps:
+            snaps[s] = (eng.x.clone(), eng.xt.clone())
+    return cons, snaps, slices, groups
+
+
+class _Worst:
+    """Running worst figures over chunks (updated from several threads)."""
+
+    def __init__(self, n, check_steps):
+        self.lock = threading.Lock()
+        self.elem = {s: 0.0 for s in check_steps}
+        self.ideal = {s: 0.0 for s in check_steps}  # fp32 rows: an ideal fp32-storage run on a share of the chunks
+        self.ulps = {s: {"n": 0, "eq": 0, "le1": 0, "le2": 0, "gt2": 0, "max": 0.0} for s in check_steps}
+        self.num = {s: np.zeros((2, n)) for s in check_steps}  # row-wise sums of (gpu - ref)^2 for x and x~
+        self.den = {s: np.zeros((2, n)) for s in check_steps}
+
+    def merge(self, s, elem=None, ulps=None, num=None, den=None, ideal=None):
+        with self.lock:
+            if elem is not None:
+                self.elem[s] = max(self.elem[s], elem)
+            if ideal is not None:
+                self.ideal[s] = max(self.ideal[s], ideal)
+            if ulps is not None:
+                h = self.ulps[s]
+                for k in ("n", "eq", "le1", "le2", "gt2"):
+                    h[k] += ulps[k]
+                h["max"] = max(h["max"], ulps["max"])
+            if num is not None:
+                self.num[s] += num
+                self.den[s] += den
+
+
+def _compare_chunk(torch, worst, s, snap, c0, c1, plain, stored, storage):
+    dev = snap[0].device
+    n = (plain or stored).n
+    out_num, out_den = np.zeros((2, n)), np.zeros((2, n))
+    for which in (0, 1):
+        gpu = snap[which][:, c0:c1].to(torch.float64)
+        if plain is not None:
+            ref = torch.from_numpy(plain.X if which == 0 else plain.Xt).to(dev)
+            diff = (gpu - ref).abs()
+            if storage == "f32":
+                rms = ref.pow(2).mean(dim=1, keepdim=True).sqrt()
+                worst.merge(s, elem=float((diff / torch.maximum(ref.abs(), rms)).max().item()))
+            else:
+                out_num[which] = diff.pow(2).sum(dim=1).cpu().numpy()
+                out_den[which] = ref.pow(2).sum(dim=1).cpu().numpy()
+        if stored is not None:
+            st = torch.from_numpy(stored.X if which == 0 else stored.Xt).to(dev)
+            rms = st.pow(2).mean(dim=1, keepdim=True).sqrt()
+            mag = torch.maximum(st.abs(), rms)
+            u = (gpu - st).abs() / torch.exp2(torch.floor(torch.log2(mag)) - 7.0)
+            worst.merge(s, ulps={"n": u.numel(), "eq": int((u == 0).sum().item()), "le1": int((u <= 1).sum().item()),
+                                 "le2": int((u <= 2).sum().item()), "gt2": int((u > 2).sum().item()),
+                                 "max": float(u.max().item())})
+    if storage != "f32" and plain is not None:
+        worst.merge(s, num=out_num, den=out_den)
+
+
+IDEAL_EVERY = 8  # fp32 rows: the ideal fp32-storage run is made on every eighth chunk
+PLAIN_EVERY_BF16 = 2  # bf16 rows: the plain fp64 run (row norms, consensus distances) on every second chunk
+
+
+def _check_full_width(cfg, check_events):
+    import torch
+
+    torch.cuda.set_device(0)
+    eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots)
+    x0, g = _fill_and_keep(eng, cfg)
+    ev = W.config_events(cfg)
+    n_steps = (len(ev) + EVENTS_PER_STEP - 1) // EVENTS_PER_STEP
+    check_steps = sorted({min(n_steps, (e + EVENTS_PER_STEP - 1) // EVENTS_PER_STEP) - 1 for e in check_events} | {n_steps - 1})
+    t0 = time.perf_counter()
+    cons_gpu, snaps, slices, groups = _run_engine(eng, cfg, ev, set(check_steps))
+    t_final = eng.times()
+    eng.close()
+    t_gpu = time.perf_counter() - t0
+
+    params = P.oracle_params(cfg)
+    per_event = [P.per_event_groups(c) for c in slices]
+    starts = list(range(0, cfg.d, CHUNK_COLS))
+    worst = _Worst(cfg.n, check_steps)
+    cons_ref = np.zeros(n_steps)
+    cons_lock = threading.Lock()
+    plain_cols = [0]  # columns on which the plain fp64 run was made
+
+    def job(c0, k):
+        c1 = min(cfg.d, c0 + CHUNK_COLS)
+        xw, gw = P.widen(x0[:, c0:c1], cfg.storage), P.widen(g[:, c0:c1], cfg.storage)
+        stored = OracleSim(xw, *params, cfg.gamma, grads=gw) if cfg.storage == "bf16" else None
+        # bf16 rows: the plain run (for the row norms and the consensus distances) on every second chunk taken
+        plain = OracleSim(xw, *params, cfg.gamma, grads=gw) if stored is None or order.index(k) % PLAIN_EVERY_BF16 == 0 else None
+        ideal = None
+        if cfg.storage == "f32" and order.index(k) % IDEAL_EVERY == 0:
+            ideal = OracleSim(xw, *params, cfg.gamma, grads=gw)
+        cons = np.zeros(n_steps)
+        for s in range(n_steps):
+            c = slices[s]
+            if plain is not None:
+                plain.apply_stream(c)
+                cons[s] = plain.consensus()
+            if stored is not None:
+                stored.apply_groups(*groups[s])
+            if ideal is not None:
+                ideal.apply_groups(c.times, c.wi, c.wj, c.slot, *per_event[s], fmt="f32")
+            if s in snaps:
+                _compare_chunk(torch, worst, s, snaps[s], c0, c1, plain, stored, cfg.storage)
+                if ideal is not None:
+                    worst.merge(s, ideal=max(P.rel_err(ideal.X, plain.X), P.rel_err(ideal.Xt, plain.Xt)))
+        assert np.array_equal((plain or stored).t, t_final)
+        with cons_lock:
+            cons_ref[:] += cons
+            if plain is not None:
+                plain_cols[0] += c1 - c0
+        return c1 - c0
+
+    # Chunks are taken in an order whose every prefix is spread evenly over the row (first and last chunk,
+    # then a golden-ratio stride through the rest), and no new chunk is started once the time budget is
+    # used up: a slow host checks fewer whole chunks, still from all over the row.
+    order = sorted(range(len(starts)), key=lambda k: (k not in (0, len(starts) - 1), (k * 0.6180339887498949) % 1.0))
+    T = _threads()
+    t0 = time.perf_counter()
+
+    def guarded(k):
+        if time.perf_counter() - t0 > BUDGET_S:
+            return 0
+        return job(starts[k], k)
+
+    with ThreadPoolExecutor(T) as ex:
+        done_cols = sum(ex.map(guarded, order))
+    t_cpu = time.perf_counter() - t0
+    full = done_cols == cfg.d
+
+    report = {"workload": cfg.name, "columns_checked": done_cols, "of": cfg.d, "check_points_after_events":
+              [min(len(ev), (s + 1) * EVENTS_PER_STEP) for s in check_steps], "gpu_s": round(t_gpu, 1), "checker_s": round(t_cpu, 1)}
+    ok = True
+    for s in check_steps:
+        if cfg.storage == "f32":
+            bound = P.TOL["f32"] if worst.ideal[s] <= 0.5 * P.TOL["f32"] else 2.0 * worst.ideal[s]
+            report[f"after_step_{s}"] = {"max_rel_err": worst.elem[s], "ideal_fp32_storage": worst.ideal[s], "bound": bound,
+                                         "1e-5_met": worst.elem[s] <= P.TOL["f32"]}
+            ok = ok and worst.elem[s] <= bound
+        else:
+            h = worst.ulps[s]
+            norm = float(np.sqrt(worst.num[s] / np.maximum(worst.den[s], 1e-300)).max())
+            report[f"after_step_{s}"] = {"ulps_max": h["max"], "exact": h["eq"] / h["n"], "within_1": h["le1"] / h["n"],
+                                         "within_2": h["le2"] / h["n"], "beyond_2": h["gt2"] / h["n"], "row_norm_err": norm}
+            ok = ok and h["max"] <= P.BF16_ULP_BOUND and h["eq"] / h["n"] >= P.BF16_MIN_EXACT and h["le1"] / h["n"] >= P.BF16_MIN_WITHIN_1
+            ok = ok and norm <= P.TOL["bf16"]  # over the columns on which the plain run was made
+    report["columns_with_plain_run"] = plain_cols[0]
+    if plain_cols[0] == cfg.d:  # the engine's own reduction after every step, against the checker's state
+        tol = 1e-4 if cfg.storage == "f32" else 5e-2
+        rel = np.abs(np.array(cons_gpu) - cons_ref) / cons_ref
+        report["consensus_rel_err_max"] = float(rel.max())
+        ok = ok and rel.max() <= tol
+    print("FULLWIDTH", report)
+    assert ok, "see the FULLWIDTH line above"
+    return report
+
+
+@pytest.mark.parametrize("name,check_events", [
+    ("cfg2", (25_000,)),
+    ("cfg3", ()),
+    ("cfg4", (500, 5_000)),  # two of its consensus points, and the end
+    ("cfg5", ()),
+])
+def test_every_element_at_full_size(name, check_events):
+    _check_full_width(W.CONFIGS[name], check_events)
+
+
+def test_static_gradient_rows_on_the_complete_graph_workload():
+    """The 16-worker complete-graph workload with ONE gradient row per worker for the whole run (a gradient
+    event of worker i always uses row i). Adding the same gamma g to a value on the binary32 grid rounds the
+    same way every time, so the error of ANY fp32-storage implementation grows linearly with the number of
+    gradient events here: the ideal fp32-storage run already misses 1e-5 on this stream, and the engine is
+    held to twice the ideal figure (it stores a row once per item, so no more often than once per event; the
+    factor covers the maximum being taken over eight times more elements)."""
+    cfg = replace(W.CONFIGS["cfg2"], grad_pool=1, name="cfg2-static-rows")
+    rep = _check_full_width(cfg, ())
+    last = rep[max(k for k in rep if k.startswith("after_step_"))]
+    assert last["ideal_fp32_storage"] > 1e-5  # the bar is out of reach of the storage format here, not of the kernel

@@ -10,6 +10,7 @@ from oracle import spectral
 from oracle.sim import OracleSim, OracleError, lib
 from oracle.sim_np import NumpySim
 from paper_2306_08289_b200 import workload as W
+from tests import parity as P
 
 SIMS = [OracleSim, NumpySim]
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -618,22 +619,26 @@ def test_c_storage_model_rounds_like_the_hand_checked_one_and_groups_equal_the_l
     # groups: runs of 1..5 consecutive events; after each, the rows of the workers it touched are rounded
     ends = np.unique(np.concatenate([np.cumsum(rng.integers(1, 6, size=400)), [len(ev)]]))
     ends = ends[ends <= len(ev)]
-    loop = OracleSim(x0, *par, cfg.gamma, grads=G)
-    ptr, flat, e0 = [0], [], 0
-    for e1 in ends:
-        c = ev.slice(e0, e1)
-        w = sorted(set(c.wi.tolist()) | set(int(j) for j in c.wj if j >= 0))
-        loop.apply_stream(c)
-        loop.round_rows(w)
-        flat += w
-        ptr.append(len(flat))
-        e0 = e1
-    once = OracleSim(x0, *par, cfg.gamma, grads=G)
-    once.apply_groups_bf16(ev.times, ev.wi, ev.wj, ev.slot, ends, ptr, flat)
-    assert np.array_equal(once.X, loop.X) and np.array_equal(once.Xt, loop.Xt) and np.array_equal(once.t, loop.t)
     plain = OracleSim(x0, *par, cfg.gamma, grads=G)
     plain.apply_stream(ev)
-    assert not np.array_equal(once.X, plain.X)  # the rounding did take place
+    for fmt in ("bf16", "f32"):
+        loop = OracleSim(x0, *par, cfg.gamma, grads=G)
+        ptr, flat, e0 = [0], [], 0
+        for e1 in ends:
+            c = ev.slice(e0, e1)
+            w = sorted(set(c.wi.tolist()) | set(int(j) for j in c.wj if j >= 0))
+            loop.apply_stream(c)
+            loop.round_rows(w, fmt=fmt)
+            flat += w
+            ptr.append(len(flat))
+            e0 = e1
+        once = OracleSim(x0, *par, cfg.gamma, grads=G)
+        once.apply_groups(ev.times, ev.wi, ev.wj, ev.slot, ends, ptr, flat, fmt=fmt)
+        assert np.array_equal(once.X, loop.X) and np.array_equal(once.Xt, loop.Xt) and np.array_equal(once.t, loop.t)
+        assert not np.array_equal(once.X, plain.X)  # the rounding did take place
+    # one event per group is the storage model of an implementation that stores after every event
+    per_event = P.per_event_groups(ev)
+    assert per_event[0][-1] == len(ev) and per_event[1][-1] == len(per_event[2]) == len(ev) + int((ev.wj >= 0).sum())
 
 
 def test_what_bf16_storage_alone_costs():
@@ -660,26 +665,6 @@ def test_what_bf16_storage_alone_costs():
     assert elem > 2e-2 and norm < 1e-2, (elem, norm)
 
 
-def _storage_only_error(cfg, fmt):
-    """Element-wise error (the metric of the GPU parity tests) of a run whose arithmetic is fp64 and
-    whose only loss is that the rows of an event's workers are rounded to `fmt` when stored."""
-    _, x0 = W.x0_matrix(cfg)
-    _, G = W.grad_matrix(cfg)
-    ev = W.config_events(cfg)
-    par = cfg.fixed_params or spectral.prescribe(cfg.n, cfg.edges(), cfg.rates())[:3]
-    plain = OracleSim(x0, *par, cfg.gamma, grads=G)
-    stored = OracleSim(x0, *par, cfg.gamma, grads=G)
-    plain.apply_stream(ev)
-    for k in range(len(ev)):
-        stored.apply_stream(ev.slice(k, k + 1))
-        stored.round_rows([ev.wi[k]] + ([ev.wj[k]] if ev.wj[k] >= 0 else []), fmt=fmt)
-    elem = 0.0
-    for a, r in ((stored.X, plain.X), (stored.Xt, plain.Xt)):
-        rms = np.sqrt((r * r).mean(axis=1, keepdims=True))
-        elem = max(elem, float((np.abs(a - r) / np.maximum(np.abs(r), rms)).max()))
-    return elem
-
-
 def test_what_fp32_storage_alone_costs():
     """What the 1e-5 bar of fp32-storage runs can and cannot hold, measured and kept as a test. An ideal
     fp32 implementation (fp64 arithmetic, one rounding to binary32 per stored value and event) of the
@@ -690,8 +675,8 @@ def test_what_fp32_storage_alone_costs():
     workloads with a static row (their increments are ten times smaller relative to the values)."""
     from dataclasses import replace
 
-    static = _storage_only_error(replace(W.CONFIGS["cfg2"].scaled(d=1_000), grad_pool=1), "f32")
-    fresh = _storage_only_error(replace(W.CONFIGS["cfg2"].scaled(d=1_000), grad_pool=128), "f32")
-    ring = _storage_only_error(W.CONFIGS["cfg4"].scaled(d=1_000), "f32")
+    static = P.storage_only_error(replace(W.CONFIGS["cfg2"].scaled(d=1_000), grad_pool=1), "f32")
+    fresh = P.storage_only_error(replace(W.CONFIGS["cfg2"].scaled(d=1_000), grad_pool=128), "f32")
+    ring = P.storage_only_error(W.CONFIGS["cfg4"].scaled(d=1_000), "f32")
     assert 2e-5 < static < 1e-4, static
     assert fresh < 1e-5 and ring < 1e-5, (fresh, ring)

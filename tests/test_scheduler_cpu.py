@@ -321,3 +321,24 @@ def test_random_streams_property():
         assert np.array_equal(s.t_final(n), ref.t)
 
     check()
+
+
+def test_storage_model_groups_of_a_schedule_equal_the_item_by_item_loop():
+    """The full-size bf16 parity test hands the checker a whole schedule at once (events in item order, a
+    rounding point after every item); that must be the item-by-item loop of the batch-wise parity helper."""
+    from oracle.sim import OracleSim
+    from tests import parity as P
+    from tests.test_gpu_fullwidth import _step_groups
+
+    cfg = W.CONFIGS["cfg5"].scaled(d=29, n_events=1500)
+    ev = W.config_events(cfg)
+    _, xw = W.x0_matrix(cfg)
+    _, gw = W.grad_matrix(cfg)
+    sched = B.Schedule(cfg.n, cfg.n_grad_slots, ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN, max_workers_per_item=3)
+    chk = P.Checker(xw, P.oracle_params(cfg), cfg.gamma, gw, "bf16")
+    for b in range(sched.num_batches):
+        chk.apply_batch(ev, sched, b)
+    once = OracleSim(xw, *P.oracle_params(cfg), cfg.gamma, grads=gw)
+    once.apply_groups(*_step_groups(ev, sched))
+    assert np.array_equal(once.X, chk.stored.X) and np.array_equal(once.Xt, chk.stored.Xt)
+    assert np.array_equal(once.t, chk.stored.t) and not np.array_equal(once.X, chk.plain.X)
