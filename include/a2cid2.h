@@ -123,7 +123,9 @@ enum {
 
 /* How a whole event stream (a2cid2_apply_events, a whole a2cid2_plan_run) is put on the GPU. */
 enum {
-    A2_LAUNCH_AUTO = 0,          /* the library chooses (column slices)                                  */
+    A2_LAUNCH_AUTO = 0,          /* the library chooses per schedule: column slices when a batch moves less than
+                                    1 GiB on average (short launches, where launch gaps and tails weigh), else
+                                    one launch per batch                                                     */
     A2_LAUNCH_PER_BATCH = 1,     /* one kernel launch per batch of worker-disjoint items; the CTAs of a launch
                                     share out its (item, column tile) units round robin                      */
     A2_LAUNCH_COLUMN_SLICES = 2  /* launches that hold the items of several consecutive batches: every CTA owns a

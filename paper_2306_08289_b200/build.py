@@ -1,4 +1,9 @@
-"""Compile the CUDA library for sm_100a into paper_2306_08289_b200/liba2cid2.so (in-tree)."""
+"""Compile the CUDA library for sm_100a into paper_2306_08289_b200/liba2cid2.so (in-tree).
+
+Extra nvcc flags for experiments may be given in the environment variable A2CID2_NVCC_FLAGS, e.g.
+"-DA2_EVENT_THREADS=512" (threads per CTA of the event kernel) or "-DA2_TUNING_KNOBS=1" (a build whose
+launch shapes can be overridden from the environment, see csrc/a2cid2_internal.h). The default build has
+no such flags and reads no tuning variable at run time."""
 from __future__ import annotations
 
 import os

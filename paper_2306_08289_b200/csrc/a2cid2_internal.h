@@ -2,12 +2,31 @@
 #pragma once
 
 #include <cstdint>
+#include <cstdlib>
 #include <string>
 #include <vector>
 
 #include "a2cid2.h"
 
 namespace a2 {
+
+// ---- tuning knobs ---------------------------------------------------------------------------
+// The launch shapes (CTAs per SM, vector width, workers per item) are fixed by measurement. A build with
+// -DA2_TUNING_KNOBS=1 lets the environment override them for sweeps (A2CID2_EVENT_CTAS_PER_SM,
+// A2CID2_EVENT3_CTAS_PER_SM, A2CID2_EVENT4_CTAS_PER_SM, A2CID2_PLAIN_CTAS_PER_SM, A2CID2_PLAIN3_CTAS_PER_SM: resident
+// CTAs per SM of the kernel instances; A2CID2_FORCE_128BIT, A2CID2_EVENT4_128BIT: 128-bit accesses;
+// A2CID2_ITEM_WORKERS: most workers per chained item). The default build reads none of them.
+#ifndef A2_TUNING_KNOBS
+#define A2_TUNING_KNOBS 0
+#endif
+inline const char* tuning_env(const char* name) {
+#if A2_TUNING_KNOBS
+    return std::getenv(name);
+#else
+    (void)name;
+    return nullptr;
+#endif
+}
 
 // ---- error text ---------------------------------------------------------------------------
 void set_thread_error(const std::string& msg);
@@ -113,6 +132,7 @@ struct EventLaunch {
     int32_t max_workers;  // most workers any item of the launch holds (2, 3 or 4): selects the kernel instance
     int32_t op_base = 0;  // index, in the plan, of the launch's first operation
     bool slice = false;   // column-slice launch: the items may span several batches, each CTA owns a range of columns
+    bool has_reloads = false;  // some operation of the launch fetches a gradient row in the middle of its item
 };
 
 struct DeviceInfo {

@@ -33,6 +33,7 @@ struct LaunchRange {
     int64_t item0, item1;  // items of the plan covered by this launch
     int64_t op0, op1;
     int workers = 2;  // most workers any item of the launch holds
+    bool reloads = false;  // some operation fetches a gradient row in the middle of its item
 };
 
 // Grow-only pinned + device buffer pair used to ship the descriptors of one apply_events call.
@@ -89,6 +90,7 @@ struct Packed {
     std::vector<LaunchRange> launches;
     std::vector<int64_t> batch_launch_first;  // launches of batch b: [first[b], first[b+1])
     std::vector<LaunchRange> slice_launches;  // the whole schedule as column-slice launches (items of several batches each)
+    bool auto_slices = false;                 // what A2_LAUNCH_AUTO picks for a whole run of this schedule
     // resident mode
     bool resident = false;
     int32_t cache_rows = 0;
@@ -164,6 +166,7 @@ void make_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launches, st
                 L.workers = std::max(L.workers, si.d >= 0 ? 4 : (si.c >= 0 ? 3 : 2));
                 L.item1 += 1;
             }
+            for (int64_t o = L.op0; o < L.op1 && !L.reloads; ++o) L.reloads = s.ops[(size_t)o].reload >= 0;
             launches.push_back(L);
             i = L.item1;
         }
@@ -185,12 +188,15 @@ void make_slice_launches(const a2cid2_sched& s, std::vector<LaunchRange>& launch
             L.workers = std::max(L.workers, si.d >= 0 ? 4 : (si.c >= 0 ? 3 : 2));
             L.item1 += 1;
         }
+        for (int64_t o = L.op0; o < L.op1 && !L.reloads; ++o) L.reloads = s.ops[(size_t)o].reload >= 0;
         launches.push_back(L);
         i = L.item1;
     }
 }
 
 size_t align16(size_t v) { return (v + 15) & ~size_t(15); }
+
+constexpr int64_t kAutoSliceBatchBytes = int64_t(1) << 30;  // 1 GiB per batch: about 160 microseconds of HBM traffic
 
 // Decide how the schedule is launched and lay its descriptors out. Resident schedules need the
 // population to fit shared memory.
@@ -203,6 +209,17 @@ int plan_layout(a2cid2* h, const a2cid2_sched& s, Packed& pk) {
     if (!pk.resident) {
         make_launches(s, pk.launches, pk.batch_launch_first);
         make_slice_launches(s, pk.slice_launches);
+        // A2_LAUNCH_AUTO: column slices where a batch is short work for the whole GPU -- its launch would last
+        // tens of microseconds, so launch gaps and the tail of every launch weigh (measured: 1.1x to 1.7x the
+        // events per second on the 16- and 4-worker workloads) -- and one launch per batch where a batch moves
+        // gigabytes (there the two modes are within a percent, and round-robin units keep all CTAs on the same
+        // few rows, which the no-momentum kernels on bf16 rows reward with 7 %).
+        const int64_t nb = (int64_t)s.batch_first.size() - 1;
+        if (nb > 0) {
+            a2cid2_stats st{};
+            a2::schedule_stats(s, 0, nb, h->d, (int32_t)elem_bytes(h->dtype), h->variant != A2_NO_MOMENTUM, &st);
+            pk.auto_slices = st.bytes_moved / nb < kAutoSliceBatchBytes;
+        }
     } else {
         pk.cache_rows = a2::resident_cache_rows(h->n, h->n_slots);
         if (pk.cache_rows <= 0)
@@ -267,10 +284,11 @@ uint32_t engine_flags(const a2cid2* h, uint32_t flags) {
 
 // Column-slice launches serve a schedule that is run whole (any batch boundary inside a launch is then harmless);
 // a range of batches is run with one launch per batch.
-bool uses_slices(const a2cid2* h, const a2cid2_sched& s, int64_t b0, int64_t b1) {
+bool uses_slices(const a2cid2* h, const a2cid2_sched& s, const Packed& pk, int64_t b0, int64_t b1) {
     const int64_t nb = (int64_t)s.batch_first.size() - 1;
     if ((s.flags & A2_SCHED_RESIDENT) || b0 != 0 || b1 != nb) return false;
-    return h->launch_mode != A2_LAUNCH_PER_BATCH;
+    if (h->launch_mode == A2_LAUNCH_AUTO) return pk.auto_slices;
+    return h->launch_mode == A2_LAUNCH_COLUMN_SLICES;
 }
 
 // Queue the kernels of batches [b0, b1) of a schedule whose blob sits at `dev`.
@@ -296,7 +314,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;
     }
-    const std::vector<LaunchRange>& list = uses_slices(h, s, b0, b1) ? pk.slice_launches : pk.launches;
+    const std::vector<LaunchRange>& list = uses_slices(h, s, pk, b0, b1) ? pk.slice_launches : pk.launches;
     const bool slices = &list == &pk.slice_launches;
     const int64_t l0 = slices ? 0 : pk.batch_launch_first[(size_t)b0];
     const int64_t l1 = slices ? (int64_t)list.size() : pk.batch_launch_first[(size_t)b1];
@@ -317,6 +335,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.max_workers = R.workers;
         L.op_base = (int32_t)R.op0;
         L.slice = slices;
+        L.has_reloads = R.reloads;
         const int rc = a2::launch_events(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
@@ -352,7 +371,7 @@ int ensure_plan_graph(a2cid2* h, a2cid2_plan* p) {
 // Launches a whole run of the plan takes under the handle's launch mode.
 int64_t whole_run_launches(const a2cid2* h, const a2cid2_plan* p) {
     const int64_t nb = (int64_t)p->sched->batch_first.size() - 1;
-    return uses_slices(h, *p->sched, 0, nb) ? (int64_t)p->pk.slice_launches.size() : (int64_t)p->pk.launches.size();
+    return uses_slices(h, *p->sched, p->pk, 0, nb) ? (int64_t)p->pk.slice_launches.size() : (int64_t)p->pk.launches.size();
 }
 
 int run_plan_graph(a2cid2* h, a2cid2_plan* p) {
@@ -370,7 +389,7 @@ void fill_stats(const a2cid2* h, const a2cid2_sched& s, const Packed& pk, int64_
         st->n_launches = b1 > b0 ? 2 : 0;
         st->bytes_moved = b1 > b0 ? ((int64_t)4 * h->n + (int64_t)pk.g_rows.size()) * h->d * eb : 0;
     } else {
-        st->n_launches = uses_slices(h, s, b0, b1) ? (int64_t)pk.slice_launches.size()
+        st->n_launches = uses_slices(h, s, pk, b0, b1) ? (int64_t)pk.slice_launches.size()
                                                    : pk.batch_launch_first[(size_t)b1] - pk.batch_launch_first[(size_t)b0];
     }
 }
@@ -423,7 +442,7 @@ int a2cid2_create(int32_t n, int64_t d, double eta, double alpha, double alpha_t
     if (!h) return fail(nullptr, A2_ENOMEM, "out of host memory");
     h->n = n; h->d = d; h->eta = eta; h->alpha = alpha; h->alpha_tilde = alpha_tilde; h->gamma = gamma;
     h->dtype = storage_dtype;
-    if (const char* v = std::getenv("A2CID2_ITEM_WORKERS")) {  // tuning override
+    if (const char* v = a2::tuning_env("A2CID2_ITEM_WORKERS")) {  // tuning override
         const int k = std::atoi(v);
         if (k >= 2 && k <= a2::kMaxItemWorkers) h->item_workers = k;
     }

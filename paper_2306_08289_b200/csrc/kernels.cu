@@ -69,6 +69,9 @@ __device__ __forceinline__ void st_u32x8(void* p, const uint32_t (&w)[8]) {
                  : "memory");
 }
 
+// Hint: bring the 128-byte line that holds p into L2 (no register, nothing to wait for).
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 template <int WORDS> struct Words;
 template <> struct Words<4> {
     static __device__ __forceinline__ void ld(const void* p, uint32_t (&w)[4]) { ld_u32x4(p, w); }
@@ -326,6 +329,7 @@ struct EventArgs {
     int msg_before_mix;
     int op_base;      // index, in the plan, of the launch's first operation (DevItem::op_first counts from the plan's)
     int slice_vec;    // column-slice launches: vectors of a row owned by one CTA (a multiple of 4); else 0
+    int has_reloads;  // some operation of the launch fetches a gradient row in the middle of its item
 };
 
 // How a launch walks its (item, column tile) units.
@@ -500,6 +504,21 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
                                                 : (A2_F32X2_BF16 != 0);
         const bool before = p.msg_before_mix != 0;
         const int o_first = it.op_first - p.op_base;
+        // Gradient rows that operations of this item fetch in the middle of the item (fresh gradients, Sec. 3.2) are
+        // asked into L2 now, while the unit's own loads are in flight: the fetch then finds its line in L2 instead
+        // of paying the DRAM and address-translation latency between two operations of the same worker. A hint
+        // only: no register, nothing to wait for. (Asking the NEXT unit's rows into L2 the same way was measured
+        // and dropped: no gain on any workload.)
+        if (sizeof(T) == 4 && p.has_reloads) {  // (bf16 rows: items never change a worker's gradient row)
+            for (int o = o_first; o < o_first + it.op_count; ++o) {
+                const int rl = s_reload[o];
+                if (rl >= 0) {
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u)
+                        if (live[u]) prefetch_l2(G + (long long)rl * p.pitch + (v0 + (long long)u * THREADS) * N);
+                }
+            }
+        }
         for (int o = o_first; o < o_first + it.op_count; ++o) {
             const int kind = s_kind[o];
             const float ca = s_ca[o];
@@ -668,6 +687,16 @@ __global__ void __launch_bounds__(kEventThreads) k_apply_events_plain(const Even
         }
         bool dirty = false;
         const int o_first = it.op_first - p.op_base;
+        if (p.has_reloads) {  // rows fetched in the middle of the item: asked into L2 now (see k_apply_events)
+            for (int o = o_first; o < o_first + it.op_count; ++o) {
+                const int rl = s_reload[o];
+                if (rl >= 0) {
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u)
+                        if (live[u]) prefetch_l2(G + (long long)rl * p.pitch + (v0 + (long long)u * kEventThreads) * N);
+                }
+            }
+        }
         for (int o = o_first; o < o_first + it.op_count; ++o) {
             const int kind = s_kind[o];
             if (kind == A2_OP_MIX_A) continue;
@@ -1131,6 +1160,7 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     a.op_base = L.op_base;
+    a.has_reloads = L.has_reloads ? 1 : 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const int per_sm = KW == 4 ? dev.event4_ctas_per_sm[BYTES == 32 ? 1 : 0]
                                : (KW == 3 ? dev.event3_ctas_per_sm : dev.event_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
@@ -1155,6 +1185,7 @@ int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t str
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
     a.op_base = L.op_base;
+    a.has_reloads = L.has_reloads ? 1 : 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const int per_sm = (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[L.dtype == A2_BF16 ? 1 : 0][BYTES == 32 ? 1 : 0];
     const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * per_sm);
@@ -1177,6 +1208,7 @@ int launch_plain_bf16(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t 
     a.eta = 0.0; a.alpha = L.alpha; a.alpha_tilde = 0.f; a.gamma = L.gamma;
     a.msg_before_mix = 0;
     a.op_base = L.op_base;
+    a.has_reloads = L.has_reloads ? 1 : 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const long long wave = (long long)dev.sm_count * (KW == 3 ? dev.plain3_ctas_per_sm : dev.plain_ctas_per_sm)[1][WORDS == 8 ? 1 : 0];
     const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, wave);
@@ -1219,7 +1251,7 @@ cudaError_t plain_occupancy(int* out) {
 // need every row start on a 32-byte boundary.
 bool rows_32B_aligned(const void* a, const void* b, const void* c, int64_t pitch, int32_t dtype) {
     if (dtype == A2_BF16) return false;
-    static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+    static const bool force_narrow = a2::tuning_env("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
     if (force_narrow) return false;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c);
     const int64_t pitch_bytes = pitch * (dtype == A2_BF16 ? 2 : 4);
@@ -1273,7 +1305,7 @@ int query_device(DeviceInfo* info) {
                                                           A2_EVENT4_THREADS, 0);
         if (e != cudaSuccess) return (int)e;
         info->event4_ctas_per_sm[1] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
-        if (const char* v = std::getenv("A2CID2_EVENT4_CTAS_PER_SM")) {  // tuning override
+        if (const char* v = a2::tuning_env("A2CID2_EVENT4_CTAS_PER_SM")) {  // tuning override
             const int k = std::atoi(v);
             if (k > 0) info->event4_ctas_per_sm[0] = info->event4_ctas_per_sm[1] = k;
         }
@@ -1315,26 +1347,26 @@ int query_device(DeviceInfo* info) {
         // bf16 rows of 25.6e6 columns, 256-bit accesses, chained schedule: 2 CTAs/SM 5.37 TB/s, 3: 6.36, 4: 5.12
         info->plain3_ctas_per_sm[1][1] = occ > 3 ? 3 : (occ > 0 ? occ : 1);
     }
-    if (const char* v = std::getenv("A2CID2_PLAIN_CTAS_PER_SM")) {  // tuning override, as for the event kernel
+    if (const char* v = a2::tuning_env("A2CID2_PLAIN_CTAS_PER_SM")) {  // tuning override, as for the event kernel
         const int k = std::atoi(v);
         if (k > 0)
             for (auto& row : info->plain_ctas_per_sm)
                 for (int& c : row) c = k;
     }
-    if (const char* v = std::getenv("A2CID2_PLAIN3_CTAS_PER_SM")) {  // the same for the three-worker instances
+    if (const char* v = a2::tuning_env("A2CID2_PLAIN3_CTAS_PER_SM")) {  // the same for the three-worker instances
         const int k = std::atoi(v);
         if (k > 0)
             for (auto& row : info->plain3_ctas_per_sm)
                 for (int& c : row) c = k;
     }
     info->consensus_ctas_per_sm = 8;  // capacity of the partial-sum scratch, CTAs per SM
-    if (const char* v = std::getenv("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
+    if (const char* v = a2::tuning_env("A2CID2_EVENT_CTAS_PER_SM")) {  // tuning override: resident CTAs per SM of the event kernel
         const int k = std::atoi(v);
         if (k > 0)
             for (auto& row : info->event_ctas_per_sm)
                 for (int& c : row) c = k;
     }
-    if (const char* v = std::getenv("A2CID2_EVENT3_CTAS_PER_SM")) {  // the same for the three-worker instances
+    if (const char* v = a2::tuning_env("A2CID2_EVENT3_CTAS_PER_SM")) {  // the same for the three-worker instances
         const int k = std::atoi(v);
         if (k > 0)
             for (auto& row : info->event3_ctas_per_sm)
@@ -1353,6 +1385,7 @@ int launch_bf16_packed(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t
     a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
     a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
     a.op_base = L.op_base;
+    a.has_reloads = L.has_reloads ? 1 : 0;
     const long long n_units = (long long)a.n_items * a.n_tiles;
     const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * dev.event3_ctas_per_sm[1][WORDS == 8 ? 1 : 0]);
     a.slice_vec = gs.slice_vec;
@@ -1368,7 +1401,7 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.variant == A2_NO_MOMENTUM) {
         const bool wide_x = rows_32B_aligned(L.x, nullptr, L.g, L.pitch, L.dtype);
         if (L.dtype == A2_BF16) {
-            static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+            static const bool force_narrow = a2::tuning_env("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
             const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.g);
             const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;
             if (L.max_workers >= 3)
@@ -1381,13 +1414,13 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
     if (L.max_workers >= 4 && L.dtype != A2_BF16) {
-        static const bool narrow4 = std::getenv("A2CID2_EVENT4_128BIT") != nullptr;  // tuning override
+        static const bool narrow4 = a2::tuning_env("A2CID2_EVENT4_128BIT") != nullptr;  // tuning override
         if (wide && !narrow4) return launch_events_t<float, 32, 4, A2_EVENT4_THREADS, 1>(L, dev, stream);
         return launch_events_t<float, 16, 4, kEventThreads, A2_EVENT4_UNROLL_128>(L, dev, stream);
     }
     if (L.max_workers >= 3) {
         if (L.dtype == A2_BF16) {
-            static const bool force_narrow = std::getenv("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
+            static const bool force_narrow = a2::tuning_env("A2CID2_FORCE_128BIT") != nullptr;  // tuning override
             const uintptr_t bits = reinterpret_cast<uintptr_t>(L.x) | reinterpret_cast<uintptr_t>(L.xt) |
                                    reinterpret_cast<uintptr_t>(L.g);
             const bool wide_bf16 = !force_narrow && bits % 32 == 0 && (L.pitch * 2) % 32 == 0;

@@ -15,7 +15,7 @@ compared with it:
               to binary32 after every event. Where that ideal run is itself above 0.5e-5 -- the bar is
               within a factor two of what the storage format delivers on the stream -- the engine is
               held to twice the ideal figure instead, and the report says whether 1e-5 was met;
-  bf16 rows   row-wise 2-norm error <= 2e-2 against the plain fp64 run (made on every second chunk, the
+  bf16 rows   row-wise 2-norm error <= 2e-2 against the plain fp64 run (made on every fourth chunk, the
               norm taken over those columns), and every
               element against the fp64 run with the storage modelled (rows rounded to bf16 where the
               schedule's items write them back) in bf16 units in the last place, with the histogram of
@@ -44,7 +44,7 @@ pytestmark = pytest.mark.gpu
 
 CHUNK_COLS = 8192
 EVENTS_PER_STEP = 500
-BUDGET_S = 200.0
+BUDGET_S = 180.0
 
 
 def _threads():
@@ -165,7 +165,7 @@ def _compare_chunk(torch, worst, s, snap, c0, c1, plain, stored, storage):
 
 
 IDEAL_EVERY = 8  # fp32 rows: the ideal fp32-storage run is made on every eighth chunk
-PLAIN_EVERY_BF16 = 2  # bf16 rows: the plain fp64 run (row norms, consensus distances) on every second chunk
+PLAIN_EVERY_BF16 = 4  # bf16 rows: the plain fp64 run (row norms) on every fourth chunk taken
 
 
 def _check_full_width(cfg, check_events):
@@ -195,7 +195,7 @@ def _check_full_width(cfg, check_events):
         c1 = min(cfg.d, c0 + CHUNK_COLS)
         xw, gw = P.widen(x0[:, c0:c1], cfg.storage), P.widen(g[:, c0:c1], cfg.storage)
         stored = OracleSim(xw, *params, cfg.gamma, grads=gw) if cfg.storage == "bf16" else None
-        # bf16 rows: the plain run (for the row norms and the consensus distances) on every second chunk taken
+        # bf16 rows: the plain run (for the row norms) on a share of the chunks taken
         plain = OracleSim(xw, *params, cfg.gamma, grads=gw) if stored is None or order.index(k) % PLAIN_EVERY_BF16 == 0 else None
         ideal = None
         if cfg.storage == "f32" and order.index(k) % IDEAL_EVERY == 0:
