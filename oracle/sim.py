@@ -145,20 +145,23 @@ class OracleSim:
         self.X, self.Xt = self.flushed(t_flush)
         self.t[:] = t_flush
 
-    def round_rows(self, workers, fmt="bf16"):
+    def round_rows(self, workers, fmt="bf16", which=("x", "xt")):
         """Model of reduced-precision *storage*: the rows of these workers are rounded to the storage
         format (bfloat16, or IEEE binary32 with fmt="f32"; both to nearest even), as happens whenever
         an implementation that keeps its state in that format writes them back. The arithmetic
-        between two stores stays fp64."""
+        between two stores stays fp64. `which` restricts the rounding to x or to x~ (to see which
+        of the two buffers' roundings an error comes from)."""
         w = np.unique(np.asarray(workers, dtype=np.int64))
         if fmt == "bf16":
-            self.X[w] = round_to_bf16(self.X[w])
-            self.Xt[w] = round_to_bf16(self.Xt[w])
+            rnd = round_to_bf16
         elif fmt == "f32":
-            self.X[w] = self.X[w].astype(np.float32).astype(np.float64)
-            self.Xt[w] = self.Xt[w].astype(np.float32).astype(np.float64)
+            rnd = lambda a: a.astype(np.float32).astype(np.float64)  # noqa: E731
         else:
             raise ValueError(fmt)
+        if "x" in which:
+            self.X[w] = rnd(self.X[w])
+        if "xt" in which:
+            self.Xt[w] = rnd(self.Xt[w])
 
     def consensus(self, t_eval=None):
         if t_eval is None:

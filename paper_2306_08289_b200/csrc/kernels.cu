@@ -1,12 +1,15 @@
 // Device kernels for sm_100a.
 //
-//   event kernel      one launch per batch of worker-disjoint items. A work unit is (item, column
-//                     tile); a persistent grid strides over the units. For a unit the item's rows
-//                     (x, x~ of its two or three workers and the gradient rows it needs) are read
-//                     once with 256- or 128-bit loads, the item's operations are applied in
-//                     registers in event order, and the state rows are written once. HBM-bound
-//                     streaming work. Separate instances for two- and three-worker items, for bf16
-//                     rows kept packed in registers, and for the dynamic without x~.
+//   event kernel      a launch holds the items of one batch of worker-disjoint items (CTAs share out
+//                     its (item, column tile) units round robin) or of several consecutive batches
+//                     (column slices: every CTA owns a range of columns and walks all items in
+//                     order). For a unit the item's rows (x, x~ of its two to four workers and the
+//                     gradient rows it starts with) are read once with 256- or 128-bit loads, the
+//                     item's operations are applied in registers in event order -- a gradient
+//                     operation may fetch its worker's next gradient row -- and the state rows are
+//                     written once. HBM-bound streaming work. Separate instances for two-, three- and
+//                     four-worker items (the last with its rows as native 64-bit register pairs), for
+//                     bf16 rows kept packed in registers, and for the dynamic without x~.
 //   consensus kernel  per column: sum_i (x_i - xbar)^2 from shifted sums, fp64 across columns,
 //                     warp shuffle + block reduce, per-block partials, fixed-order final sum.
 //
@@ -207,10 +210,9 @@ struct GradK {  // per-operation constants of a gradient event, both lanes equal
     f32x2 c, nc, ngamma;
     __device__ __forceinline__ GradK(float c_, float ngamma_) : c(pk2(c_, c_)), nc(pk2(-c_, -c_)), ngamma(pk2(ngamma_, ngamma_)) {}
 };
+// The two updates on a native pair (one 64-bit register holding two fp32 columns).
 template <bool ONE_ROUNDING>
-__device__ __forceinline__ void grad_pair(float& x0, float& x1, float& xt0, float& xt1, const GradK& K, float g0, float g1) {
-    f32x2 x = pk2(x0, x1), xt = pk2(xt0, xt1);
-    const f32x2 g = pk2(g0, g1);
+__device__ __forceinline__ void grad_pair2(f32x2& x, f32x2& xt, const GradK& K, f32x2 g) {
     const f32x2 dlt = sub2(x, xt);
     if (!ONE_ROUNDING) {
         x = fma2(K.ngamma, g, fma2(K.nc, dlt, x));
@@ -220,6 +222,11 @@ __device__ __forceinline__ void grad_pair(float& x0, float& x1, float& xt0, floa
         x = add2(x, fma2(K.nc, dlt, tg));
         xt = add2(xt, fma2(K.c, dlt, tg));
     }
+}
+template <bool ONE_ROUNDING>
+__device__ __forceinline__ void grad_pair(float& x0, float& x1, float& xt0, float& xt1, const GradK& K, float g0, float g1) {
+    f32x2 x = pk2(x0, x1), xt = pk2(xt0, xt1);
+    grad_pair2<ONE_ROUNDING>(x, xt, K, pk2(g0, g1));
     upk2(x, x0, x1);
     upk2(xt, xt0, xt1);
 }
@@ -230,9 +237,7 @@ struct CommK {  // per-operation constants of a communication event
         : nca(pk2(-ca, -ca)), ncb(pk2(-cb, -cb)), alpha(pk2(a, a)), nalpha(pk2(-a, -a)), alpha_t(pk2(at, at)), nalpha_t(pk2(-at, -at)) {}
 };
 template <bool COMPENSATED>
-__device__ __forceinline__ void comm_pair(float& xa0, float& xa1, float& xta0, float& xta1, float& xb0, float& xb1,
-                                          float& xtb0, float& xtb1, const CommK& K, bool msg_before_mix) {
-    f32x2 xa = pk2(xa0, xa1), xta = pk2(xta0, xta1), xb = pk2(xb0, xb1), xtb = pk2(xtb0, xtb1);
+__device__ __forceinline__ void comm_pair2(f32x2& xa, f32x2& xta, f32x2& xb, f32x2& xtb, const CommK& K, bool msg_before_mix) {
     const f32x2 ua = mul2(K.nca, sub2(xa, xta));
     const f32x2 ub = mul2(K.ncb, sub2(xb, xtb));
     if (!COMPENSATED) {
@@ -264,6 +269,12 @@ __device__ __forceinline__ void comm_pair(float& xa0, float& xa1, float& xta0, f
         xb = add2(xb, fma2(K.alpha, m, fma2(K.alpha, m_lo, ub)));
         xtb = sub2(xtb, fma2(K.nalpha_t, m, fma2(K.nalpha_t, m_lo, ub)));  // + (alpha~ m + alpha~ m_lo - ub)
     }
+}
+template <bool COMPENSATED>
+__device__ __forceinline__ void comm_pair(float& xa0, float& xa1, float& xta0, float& xta1, float& xb0, float& xb1,
+                                          float& xtb0, float& xtb1, const CommK& K, bool msg_before_mix) {
+    f32x2 xa = pk2(xa0, xa1), xta = pk2(xta0, xta1), xb = pk2(xb0, xb1), xtb = pk2(xtb0, xtb1);
+    comm_pair2<COMPENSATED>(xa, xta, xb, xtb, K, msg_before_mix);
     upk2(xa, xa0, xa1);
     upk2(xta, xta0, xta1);
     upk2(xb, xb0, xb1);
@@ -606,6 +617,179 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
                         V::store(pxtd + off, xtd[u]);
                     }
                 }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Four-worker items on fp32 rows with the rows held as NATIVE PAIRS: a row's 32 bytes arrive as four 64-bit
+// registers (ld.global.cs.v4.b64), every operation is one of sm_100's packed fp32 instructions on such a register
+// (add/sub/mul/fma.rn.f32x2: two IEEE results each, rounded like the scalar forms), and the row leaves as four
+// 64-bit registers. k_apply_events reaches the same instructions from scalar registers through mov.b64 packs and
+// unpacks around every operation; ncu showed those moves issuing about as many ALU instructions as there are
+// packed FMA-pipe instructions, on a kernel that is short of issue slots (an item serves ten events, an SM holds
+// only twelve of its warps). Per element the arithmetic, and so every bit of the result, is that of k_apply_events.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ld_pairs(const float* p, f32x2 (&v)[4]) {
+    asm volatile("ld.global.cs.v4.b64 {%0,%1,%2,%3}, [%4];" : "=l"(v[0]), "=l"(v[1]), "=l"(v[2]), "=l"(v[3]) : "l"(p));
+}
+__device__ __forceinline__ void st_pairs(float* p, const f32x2 (&v)[4]) {
+    asm volatile("st.global.cs.v4.b64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(v[0]), "l"(v[1]), "l"(v[2]), "l"(v[3]) : "memory");
+}
+
+template <int KW, int THREADS, bool SLICE>
+__global__ void __launch_bounds__(THREADS) k_apply_events_pairs(const EventArgs p) {
+    constexpr int N = 8, NP = 4;  // fp32 columns and native pairs per 256-bit vector
+    __shared__ DevItem s_items[kMaxItemsPerLaunch];
+    __shared__ float s_ca[kMaxOpsPerLaunch];
+    __shared__ float s_cb[kMaxOpsPerLaunch];
+    __shared__ unsigned char s_kind[kMaxOpsPerLaunch];
+    __shared__ int s_reload[kMaxOpsPerLaunch];
+
+    for (int i = threadIdx.x; i < p.n_items; i += THREADS) s_items[i] = p.items[i];
+    for (int o = threadIdx.x; o < p.n_ops; o += THREADS) {
+        const DevOp op = p.ops[o];
+        s_kind[o] = (unsigned char)op.kind;
+        s_reload[o] = op.reload;
+        const bool comm = op.kind == A2_OP_COMM || op.kind == A2_OP_COMM_AC || op.kind == A2_OP_COMM_BC ||
+                          op.kind == A2_OP_COMM_AD || op.kind == A2_OP_COMM_BD || op.kind == A2_OP_COMM_CD;
+        s_ca[o] = (float)mix_coeff(p.eta, op.t - op.t_prev_a);
+        s_cb[o] = comm ? (float)mix_coeff(p.eta, op.t - op.t_prev_b) : 0.f;
+    }
+    __syncthreads();
+
+    float* const X = static_cast<float*>(p.x);
+    float* const Xt = static_cast<float*>(p.xt);
+    const float* const G = static_cast<const float*>(p.g);
+    const float alpha = p.alpha, alpha_t = p.alpha_tilde, ngamma = -p.gamma;
+    const bool before = p.msg_before_mix != 0;
+
+    const UnitWalk<SLICE, THREADS> walk(p);
+    const long long v_end = walk.v_end;
+    const int n_it = p.n_items;
+    // (item, tile) of the round-robin walk advanced incrementally, as in k_apply_events
+    int rem = (int)(blockIdx.x % (unsigned)n_it);
+    long long tile = blockIdx.x / (unsigned)n_it;
+    int skew = (int)((unsigned long long)tile % (unsigned)n_it);
+    const int step_rem = (int)(gridDim.x % (unsigned)n_it);
+    const long long step_tile = gridDim.x / (unsigned)n_it;
+    const int step_skew = (int)((unsigned long long)step_tile % (unsigned)n_it);
+    for (long long unit = walk.first; unit < walk.end; unit += walk.step, rem += step_rem, tile += step_tile, skew += step_skew) {
+        int item_idx;
+        long long tile_v0;
+        if (SLICE) {
+            walk.map(unit, item_idx, tile_v0);
+        } else {
+            if (rem >= n_it) { rem -= n_it; tile += 1; skew += 1; }
+            if (skew >= n_it) skew -= n_it;
+            item_idx = rem + skew >= n_it ? rem + skew - n_it : rem + skew;
+            tile_v0 = tile * (long long)THREADS;
+        }
+        const DevItem it = s_items[item_idx];
+        const long long v = tile_v0 + threadIdx.x;
+        if (v >= v_end) continue;  // this thread's vector lies past the row (or past the slice)
+        const long long off = v * N;
+        const bool has_b = it.b >= 0, has_c = KW >= 3 && it.c >= 0, has_d = KW >= 4 && it.d >= 0;
+
+        float* const pxa = X + (long long)it.a * p.pitch + off;
+        float* const pxta = Xt + (long long)it.a * p.pitch + off;
+        float* const pxb = X + (long long)(has_b ? it.b : it.a) * p.pitch + off;
+        float* const pxtb = Xt + (long long)(has_b ? it.b : it.a) * p.pitch + off;
+        float* const pxc = X + (long long)(has_c ? it.c : it.a) * p.pitch + off;
+        float* const pxtc = Xt + (long long)(has_c ? it.c : it.a) * p.pitch + off;
+        float* const pxd = X + (long long)(has_d ? it.d : it.a) * p.pitch + off;
+        float* const pxtd = Xt + (long long)(has_d ? it.d : it.a) * p.pitch + off;
+
+        constexpr int PC = KW >= 3 ? NP : 1, PD = KW >= 4 ? NP : 1;
+        f32x2 xa[NP], xta[NP], xb[NP], xtb[NP], ga[NP], gb[NP], xc[PC], xtc[PC], gc[PC], xd[PD], xtd[PD], gd[PD];
+        ld_pairs(pxa, xa);
+        ld_pairs(pxta, xta);
+        if (has_b) {
+            ld_pairs(pxb, xb);
+            ld_pairs(pxtb, xtb);
+        }
+        if (it.slot_a >= 0) ld_pairs(G + (long long)it.slot_a * p.pitch + off, ga);
+        if (it.slot_b >= 0) ld_pairs(G + (long long)it.slot_b * p.pitch + off, gb);
+        if constexpr (KW >= 3) {
+            if (has_c) {
+                ld_pairs(pxc, xc);
+                ld_pairs(pxtc, xtc);
+            }
+            if (it.slot_c >= 0) ld_pairs(G + (long long)it.slot_c * p.pitch + off, gc);
+        }
+        if constexpr (KW >= 4) {
+            if (has_d) {
+                ld_pairs(pxd, xd);
+                ld_pairs(pxtd, xtd);
+            }
+            if (it.slot_d >= 0) ld_pairs(G + (long long)it.slot_d * p.pitch + off, gd);
+        }
+
+        const int o_first = it.op_first - p.op_base;
+        if (p.has_reloads) {  // rows fetched in the middle of the item: asked into L2 now (see k_apply_events)
+            for (int o = o_first; o < o_first + it.op_count; ++o) {
+                const int rl = s_reload[o];
+                if (rl >= 0) prefetch_l2(G + (long long)rl * p.pitch + off);
+            }
+        }
+        for (int o = o_first; o < o_first + it.op_count; ++o) {
+            const int kind = s_kind[o];
+            const float ca = s_ca[o];
+            auto grad = [&](f32x2 (&x)[NP], f32x2 (&xt)[NP], f32x2 (&g)[NP]) {
+                const GradK K(ca, ngamma);
+#pragma unroll
+                for (int k = 0; k < NP; ++k) grad_pair2<true>(x[k], xt[k], K, g[k]);
+                const int rl = s_reload[o];  // the worker's next gradient row, when it is another one
+                if (rl >= 0) ld_pairs(G + (long long)rl * p.pitch + off, g);
+            };
+            auto comm = [&](f32x2 (&xp)[NP], f32x2 (&xtp)[NP], f32x2 (&xq)[NP], f32x2 (&xtq)[NP]) {
+                const CommK K(ca, s_cb[o], alpha, alpha_t);
+#pragma unroll
+                for (int k = 0; k < NP; ++k) comm_pair2<true>(xp[k], xtp[k], xq[k], xtq[k], K, before);
+            };
+            if (kind == A2_OP_GRAD_A) {
+                grad(xa, xta, ga);
+            } else if (kind == A2_OP_GRAD_B) {
+                grad(xb, xtb, gb);
+            } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
+                const GradK K(ca, ngamma);
+#pragma unroll
+                for (int k = 0; k < NP; ++k) grad_pair2<true>(xa[k], xta[k], K, pk2(0.f, 0.f));
+            } else if (kind == A2_OP_COMM) {
+                comm(xa, xta, xb, xtb);
+            } else if constexpr (KW >= 3) {
+                if (kind == A2_OP_GRAD_C) {
+                    grad(xc, xtc, gc);
+                } else if (kind == A2_OP_COMM_AC) {
+                    comm(xa, xta, xc, xtc);
+                } else if (kind == A2_OP_COMM_BC) {
+                    comm(xb, xtb, xc, xtc);
+                } else if constexpr (KW >= 4) {
+                    if (kind == A2_OP_GRAD_D) grad(xd, xtd, gd);
+                    else if (kind == A2_OP_COMM_AD) comm(xa, xta, xd, xtd);
+                    else if (kind == A2_OP_COMM_BD) comm(xb, xtb, xd, xtd);
+                    else comm(xc, xtc, xd, xtd);
+                }
+            }
+        }
+
+        st_pairs(pxa, xa);
+        st_pairs(pxta, xta);
+        if (has_b) {
+            st_pairs(pxb, xb);
+            st_pairs(pxtb, xtb);
+        }
+        if constexpr (KW >= 3) {
+            if (has_c) {
+                st_pairs(pxc, xc);
+                st_pairs(pxtc, xtc);
+            }
+        }
+        if constexpr (KW >= 4) {
+            if (has_d) {
+                st_pairs(pxd, xd);
+                st_pairs(pxtd, xtd);
             }
         }
     }
@@ -1172,6 +1356,26 @@ int launch_events_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t st
     return (int)cudaGetLastError();
 }
 
+int launch_events_pairs4(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
+    constexpr int THREADS = A2_EVENT4_THREADS;
+    EventArgs a;
+    a.x = L.x; a.xt = L.xt; a.g = L.g; a.pitch = L.pitch;
+    a.n_vec = (L.d + 7) / 8;
+    a.items = L.items; a.ops = L.ops; a.n_items = L.n_items; a.n_ops = L.n_ops;
+    a.n_tiles = (int)((a.n_vec + THREADS - 1) / THREADS);
+    a.eta = L.eta; a.alpha = L.alpha; a.alpha_tilde = L.alpha_tilde; a.gamma = L.gamma;
+    a.msg_before_mix = L.variant == A2_MSG_BEFORE_MIX;
+    a.op_base = L.op_base;
+    a.has_reloads = L.has_reloads ? 1 : 0;
+    const long long n_units = (long long)a.n_items * a.n_tiles;
+    const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * dev.event4_ctas_per_sm[1]);
+    a.slice_vec = gs.slice_vec;
+    if (gs.grid < 1) return 0;
+    if (L.slice) k_apply_events_pairs<4, THREADS, true><<<gs.grid, THREADS, 0, stream>>>(a);
+    else k_apply_events_pairs<4, THREADS, false><<<gs.grid, THREADS, 0, stream>>>(a);
+    return (int)cudaGetLastError();
+}
+
 template <typename T, int BYTES, int KW>
 int launch_plain_t(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr int U = PlainCfg<BYTES>::UNROLL;
@@ -1301,7 +1505,7 @@ int query_device(DeviceInfo* info) {
             &occ, k_apply_events<float, 16, A2_EVENT4_UNROLL_128, 4, kEventThreads>, kEventThreads, 0);
         if (e != cudaSuccess) return (int)e;
         info->event4_ctas_per_sm[0] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events<float, 32, 1, 4, A2_EVENT4_THREADS>,
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_apply_events_pairs<4, A2_EVENT4_THREADS, false>,
                                                           A2_EVENT4_THREADS, 0);
         if (e != cudaSuccess) return (int)e;
         info->event4_ctas_per_sm[1] = occ > 2 ? 2 : (occ > 0 ? occ : 1);
@@ -1415,7 +1619,7 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
     if (L.max_workers >= 4 && L.dtype != A2_BF16) {
         static const bool narrow4 = a2::tuning_env("A2CID2_EVENT4_128BIT") != nullptr;  // tuning override
-        if (wide && !narrow4) return launch_events_t<float, 32, 4, A2_EVENT4_THREADS, 1>(L, dev, stream);
+        if (wide && !narrow4) return launch_events_pairs4(L, dev, stream);
         return launch_events_t<float, 16, 4, kEventThreads, A2_EVENT4_UNROLL_128>(L, dev, stream);
     }
     if (L.max_workers >= 3) {
