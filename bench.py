@@ -51,8 +51,10 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one event-kernel launch as a ratio to the bytes the
 # launch's items must move, from the committed ncu summary named beside it; None while the kernel has
 # changed since the counters were taken.
-NCU_TRAFFIC_RATIO = None
-NCU_TRAFFIC_SOURCE = None
+NCU_TRAFFIC_RATIO = 0.986
+NCU_TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of three whole-step launches of the four-worker instance "
+                      "on a d = 2e6 case of cfg4 (15.04 GB against 15.25 GB the items move: profiles/k_apply_events_cfg4_d2m.md), "
+                      "scaled to this launch by its bytes; not a counter of this run")
 LAUNCH_MODES = {"auto": 0, "per-batch": 1, "column-slices": 2}
 
 
