@@ -323,3 +323,33 @@ def test_closed_loop_quadratic_matches_the_checker_and_shows_the_speed_up():
         res[acc] = g["trace"]
     assert res[True][-1][2] < res[False][-1][2]      # consensus distance
     assert res[False][-1][1] < res[False][0][1]      # and the mean does approach the minimiser
+
+
+@pytest.mark.parametrize("storage,momentum", [("f32", True), ("bf16", True), ("f32", False), ("bf16", False)])
+@pytest.mark.parametrize("d", [1, 9, 2_049, 50_003])
+def test_launch_modes_give_the_same_bits(storage, momentum, d):
+    """One launch per batch, column slices (a launch spans batches; every CTA walks all items over columns of
+    its own) and the library's own choice: the same state bit for bit, for every storage type and both
+    dynamics, from a single column to slices with a ragged last tile; and that state is the checker's."""
+    cfg = W.WorkloadConfig(name=f"modes{d}", n=12, graph="ring", d=d, storage=storage, n_events=900, x0_std=1.0,
+                           g_std=0.3, gamma=0.05, edge_rate=1.0, fixed_params=(0.4, 0.5, 1.7), grad_pool=3, seed=91)
+    ev = W.config_events(cfg)
+    states = []
+    for mode in (B.A2_LAUNCH_PER_BATCH, B.A2_LAUNCH_COLUMN_SLICES, B.A2_LAUNCH_AUTO):
+        eng, chk = P.make_small(cfg, momentum=momentum)
+        eng.set_launch_mode(mode)
+        for lo in range(0, len(ev), 300):  # several calls, so that launches start from stored state
+            c = ev.slice(lo, lo + 300)
+            st = eng.apply_events(c.times, c.wi, c.wj, c.slot, flags=B.A2_SCHED_CHAIN, want_stats=True)
+            if mode == B.A2_LAUNCH_COLUMN_SLICES:
+                assert st["n_launches"] < st["n_batches"]
+        states.append(eng.read_state())
+        eng.close()
+    for o in states[1:]:
+        assert all(u is None and v is None or np.array_equal(u, v) for u, v in zip(states[0], o))
+    if storage == "f32":
+        eng, chk = P.make_small(cfg, momentum=momentum)
+        chk.plain.apply_stream(ev)
+        x, xt, t = states[0]
+        chk.compare(P.widen(x, "f32"), None if xt is None else P.widen(xt, "f32"), t, where=f"launch modes, d={d}")
+        eng.close()
