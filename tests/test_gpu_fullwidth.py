@@ -275,6 +275,14 @@ def test_every_element_at_full_size(name, check_events):
     _check_full_width(W.CONFIGS[name], check_events)
 
 
+def test_every_element_with_fresh_gradient_rows_inside_four_worker_items():
+    """The 64-worker ring at full width with a pool of four gradient rows per worker, so that consecutive gradient
+    events of a worker name different rows and the chained four-worker items fetch rows in the middle of an item
+    (the paper's gradients are fresh draws at every step, Sec. 3.2). The first 4,000 events of the stream."""
+    cfg = replace(W.CONFIGS["cfg4"], grad_pool=4, n_events=4_000, name="cfg4-pool4")
+    _check_full_width(cfg, ())
+
+
 def test_static_gradient_rows_on_the_complete_graph_workload():
     """The 16-worker complete-graph workload with ONE gradient row per worker for the whole run (a gradient
     event of worker i always uses row i). Adding the same gamma g to a value on the binary32 grid rounds the
