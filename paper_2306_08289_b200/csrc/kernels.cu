@@ -638,6 +638,9 @@ __device__ __forceinline__ void st_pairs(float* p, const f32x2 (&v)[4]) {
     asm volatile("st.global.cs.v4.b64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(v[0]), "l"(v[1]), "l"(v[2]), "l"(v[3]) : "memory");
 }
 
+// (Launch bounds without a minimum CTA count on purpose: ptxas then settles at 156-158 registers and two CTAs of
+// 192 threads fit an SM. With an explicit minimum of one it takes more than 170, one CTA fits, and the kernel
+// loses a third of its speed; with the registers capped at 128 for sixteen warps it gains nothing.)
 template <int KW, int THREADS, bool SLICE>
 __global__ void __launch_bounds__(THREADS) k_apply_events_pairs(const EventArgs p) {
     constexpr int N = 8, NP = 4;  // fp32 columns and native pairs per 256-bit vector
