@@ -37,6 +37,15 @@ def test_every_declared_symbol_is_exported_and_bound():
     assert B.lib().a2cid2_version().startswith(b"a2cid2")
 
 
+def test_enumerators_of_the_header_are_those_of_the_binding():
+    src = open(os.path.join(ROOT, "include", "a2cid2.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    found = {k: int(v.rstrip("u")) for k, v in re.findall(r"\b(A2_[A-Z0-9_]+)\s*=\s*(-?\d+u?)", src)}
+    assert len(found) >= 30
+    for name, value in found.items():
+        assert getattr(B, name) == value, name
+
+
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
 def test_graph_quantities_agree_with_checker(name):
     c = W.CONFIGS[name]
@@ -90,6 +99,9 @@ def test_create_validates_without_a_device():
     for v in (B.A2_MSG_BEFORE_MIX, B.A2_NO_MOMENTUM, B.A2_MSG_AFTER_MIX):
         assert L.a2cid2_set_variant(h, v) == B.A2_OK
     assert L.a2cid2_set_variant(h, 3) == B.A2_EINVAL and L.a2cid2_set_variant(h, -1) == B.A2_EINVAL
+    for m in (B.A2_LAUNCH_PER_BATCH, B.A2_LAUNCH_COLUMN_SLICES, B.A2_LAUNCH_AUTO):
+        assert L.a2cid2_set_launch_mode(h, m) == B.A2_OK
+    assert L.a2cid2_set_launch_mode(h, 3) == B.A2_EINVAL and b"launch mode" in L.a2cid2_last_error(h)
     # binding without an x~ buffer is refused unless the variant has no momentum (checked before any device call)
     dummy = C.c_void_p(4096)
     assert L.a2cid2_bind(h, dummy, None, None, 0, 16, None) == B.A2_EINVAL
