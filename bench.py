@@ -517,6 +517,10 @@ def main():
         "rows_per_event": p1["bytes"] / (cfg.d * elem_bytes) / max(1, p1["events"]),
         "effective_gbs_one_event_per_item": p1["bytes_single"] / (p1["k1_ms"] / 1e3) / 1e9,
         "share_of_step_time": p1["k1_ms"] / p1["total_ms"],
+        "note": "HBM is the roofline every instance of the event kernel is measured against; the four-worker instance on "
+                "static gradient rows (ten events on 20 rows per item) is held back by instruction issue and latency "
+                "before DRAM and follows the SM clock, with a gradient row per gradient event (fresh_gradients) it sits "
+                "at the copy bandwidth",
     }
     consensus_gbs = K * cfg.n * cfg.d * elem_bytes / (p1["k2_ms"] / 1e3) / 1e9
 
