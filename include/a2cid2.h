@@ -136,6 +136,23 @@ enum {
                                     CTA ever waits for another. The results are the same bits in all modes.  */
 };
 
+/* How often x is rounded to its storage precision (fp32 rows). */
+enum {
+    A2_ROUND_PER_EVENT = 0, /* every event rounds every value it updates once (the default). This is what an
+                               fp32-storage implementation that applies events one by one does, and all
+                               schedules and launch modes then give the same bits.                           */
+    A2_ROUND_PER_STORE = 1  /* inside an item x is carried as a two-word value (what its roundings have lost
+                               is kept beside it) and rounded once, when the item stores the row. Why: at an
+                               averaging alpha~ multiplies the rounding errors x has collected into x~
+                               (Eq. (dynamic), dM term: x~ moves by alpha~ (x_i - x_j)), so where alpha~ is
+                               several times alpha (7.26 against 0.5 on the 64-worker ring) the error of x~ is
+                               a random walk of amplified half-ulps of x, and an item that serves ten events
+                               can spare nine of ten roundings. Costs about 12 % of the events per second of
+                               chained schedules; results then depend on the schedule in the last bits.
+                               fp32 rows with the momentum buffer, on 32-byte boundaries, batched schedules
+                               (not A2_SCHED_RESIDENT).                                                      */
+};
+
 /* One item of a batch: all the work done on one worker (b = c = d = -1) or on two to four workers. */
 typedef struct a2cid2_item_info {
     int32_t a, b;           /* worker rows; b = -1 for a gradient-only item                    */
@@ -181,6 +198,10 @@ int a2cid2_set_variant(a2cid2_t* h, int32_t variant);
 /* Select how whole streams are launched (A2_LAUNCH_*; default A2_LAUNCH_AUTO). A range of a plan's batches
  * (a2cid2_plan_run with a first batch or a count) is always run with one launch per batch. */
 int a2cid2_set_launch_mode(a2cid2_t* h, int32_t mode);
+
+/* Select A2_ROUND_PER_EVENT (default) or A2_ROUND_PER_STORE for later events. A2_EINVAL for bf16 storage; a call
+ * that applies events fails with A2_ESTATE, before any launch, if the bound rows do not allow the mode. */
+int a2cid2_set_rounding(a2cid2_t* h, int32_t mode);
 
 /* Lend the device buffers: x and x_tilde are [n, row_pitch_elems], grads is
  * [n_grad_slots, row_pitch_elems] (may be NULL with n_grad_slots = 0 if no gradient event is

@@ -26,6 +26,7 @@ A2_OP_GRAD_A, A2_OP_GRAD_B, A2_OP_COMM, A2_OP_MIX_A, A2_OP_GRAD_C, A2_OP_COMM_AC
 A2_OP_GRAD_D, A2_OP_COMM_AD, A2_OP_COMM_BD, A2_OP_COMM_CD = 7, 8, 9, 10
 A2_MSG_AFTER_MIX, A2_MSG_BEFORE_MIX, A2_NO_MOMENTUM = 0, 1, 2
 A2_LAUNCH_AUTO, A2_LAUNCH_PER_BATCH, A2_LAUNCH_COLUMN_SLICES = 0, 1, 2
+A2_ROUND_PER_EVENT, A2_ROUND_PER_STORE = 0, 1
 
 ERROR_NAMES = {A2_EINVAL: "A2_EINVAL", A2_EORDER: "A2_EORDER", A2_ERANGE: "A2_ERANGE", A2_ENOMEM: "A2_ENOMEM",
                A2_ECUDA: "A2_ECUDA", A2_ESTATE: "A2_ESTATE"}
@@ -66,6 +67,7 @@ SIGNATURES = {
     "a2cid2_create": (C.c_int, [C.c_int32, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int32, C.POINTER(_vp)]),
     "a2cid2_set_variant": (C.c_int, [_vp, C.c_int32]),
     "a2cid2_set_launch_mode": (C.c_int, [_vp, C.c_int32]),
+    "a2cid2_set_rounding": (C.c_int, [_vp, C.c_int32]),
     "a2cid2_bind": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp]),
     "a2cid2_write_state": (C.c_int, [_vp, _vp, _vp, _dp]),
     "a2cid2_write_grads": (C.c_int, [_vp, C.c_int32, C.c_int32, _vp]),
@@ -328,6 +330,9 @@ class Engine:
 
     def set_launch_mode(self, mode):
         _check(lib().a2cid2_set_launch_mode(self._h, mode), self._h)
+
+    def set_rounding(self, mode):
+        _check(lib().a2cid2_set_rounding(self._h, mode), self._h)
 
     def write_state(self, x, x_tilde=None, t=None):
         x = np.ascontiguousarray(x, dtype=self.np_dtype)

@@ -133,6 +133,7 @@ struct EventLaunch {
     int32_t op_base = 0;  // index, in the plan, of the launch's first operation
     bool slice = false;   // column-slice launch: the items may span several batches, each CTA owns a range of columns
     bool has_reloads = false;  // some operation of the launch fetches a gradient row in the middle of its item
+    bool round_per_store = false;  // A2_ROUND_PER_STORE: x carried as a two-word value inside an item
 };
 
 struct DeviceInfo {
@@ -148,6 +149,7 @@ struct DeviceInfo {
 // Launchers (kernels.cu). All return a cudaError_t cast to int (0 = success).
 int query_device(DeviceInfo* info);
 int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream);
+bool rows_allow_256bit(const void* x, const void* xt, const void* g, int64_t pitch, int32_t dtype);
 // Consensus distance. dt (device, n doubles) is NULL for the stored state; partials is device
 // scratch of n_partials doubles; out is a device double.
 int consensus_grid(const DeviceInfo& dev);

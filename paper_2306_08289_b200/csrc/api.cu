@@ -57,6 +57,7 @@ struct a2cid2 {
     int32_t variant = A2_MSG_AFTER_MIX;
     int32_t item_workers = a2::kMaxItemWorkers;  // most workers A2_SCHED_CHAIN puts into one item (before the kernels' limits)
     int32_t launch_mode = A2_LAUNCH_AUTO;
+    int32_t rounding = A2_ROUND_PER_EVENT;
     // borrowed buffers
     void* x = nullptr;
     void* xt = nullptr;
@@ -301,6 +302,8 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
     if (pk.resident) {
         if (h->variant == A2_NO_MOMENTUM)
             return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT is not available for the A2_NO_MOMENTUM variant");
+        if (h->rounding == A2_ROUND_PER_STORE)
+            return fail(h, A2_EINVAL, "A2_SCHED_RESIDENT rounds every value at every event: not available with A2_ROUND_PER_STORE");
         a2::ResidentLaunch L;
         L.x = h->x; L.xt = h->xt; L.g = h->g; L.pitch = h->pitch; L.d = h->d;
         L.n = h->n; L.dtype = h->dtype; L.variant = h->variant; L.eta = h->eta;
@@ -313,6 +316,12 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         const int rc = a2::launch_resident(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "resident kernel launch");
         return A2_OK;
+    }
+    const bool per_store = h->rounding == A2_ROUND_PER_STORE;
+    if (per_store) {  // before anything is launched
+        if (h->variant == A2_NO_MOMENTUM) return fail(h, A2_ESTATE, "A2_ROUND_PER_STORE has no meaning for the A2_NO_MOMENTUM variant");
+        if (!a2::rows_allow_256bit(h->x, h->xt, h->g, h->pitch, h->dtype))
+            return fail(h, A2_ESTATE, "A2_ROUND_PER_STORE needs x, x_tilde and the gradient buffer on 32-byte boundaries and a row pitch that is a multiple of 32 bytes");
     }
     const std::vector<LaunchRange>& list = uses_slices(h, s, pk, b0, b1) ? pk.slice_launches : pk.launches;
     const bool slices = &list == &pk.slice_launches;
@@ -336,6 +345,7 @@ int queue_batches(a2cid2* h, const a2cid2_sched& s, const Packed& pk, void* dev,
         L.op_base = (int32_t)R.op0;
         L.slice = slices;
         L.has_reloads = R.reloads;
+        L.round_per_store = per_store;
         const int rc = a2::launch_events(L, h->dev, stream);
         if (rc != 0) return fail_cuda(h, (cudaError_t)rc, "event kernel launch");
     }
@@ -468,6 +478,16 @@ int a2cid2_set_launch_mode(a2cid2_t* h, int32_t mode) {
         return fail(h, A2_EINVAL, "unknown launch mode");
     h->launch_mode = mode;
     h->bind_epoch += 1;  // recorded plan graphs hold the launches of the previous mode
+    return A2_OK;
+}
+
+int a2cid2_set_rounding(a2cid2_t* h, int32_t mode) {
+    if (!h) return fail(nullptr, A2_EINVAL, "handle is NULL");
+    if (mode != A2_ROUND_PER_EVENT && mode != A2_ROUND_PER_STORE) return fail(h, A2_EINVAL, "unknown rounding mode");
+    if (mode == A2_ROUND_PER_STORE && h->dtype != A2_F32)
+        return fail(h, A2_EINVAL, "A2_ROUND_PER_STORE is for fp32 rows (bf16 rows are rounded to eight bits at every store anyway)");
+    h->rounding = mode;
+    h->bind_epoch += 1;  // recorded plan graphs hold the kernels of the previous mode
     return A2_OK;
 }
 

@@ -622,6 +622,52 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
     }
 }
 
+// The two updates with x carried as an unevaluated sum x + xl inside an item (xl: what the roundings of x have lost
+// so far; it starts at zero when the row is loaded and is added back, with one rounding, when the row is stored).
+template <bool XLO>
+__device__ __forceinline__ void grad_pair_x(f32x2& x, f32x2& xl, f32x2& xt, const GradK& K, f32x2 g) {
+    f32x2 dlt = sub2(x, xt);
+    if (XLO) dlt = add2(dlt, xl);
+    const f32x2 tg = mul2(K.ngamma, g);
+    const f32x2 inc = fma2(K.nc, dlt, tg);
+    const f32x2 s = add2(x, inc);
+    if (XLO) xl = add2(xl, sub2(inc, sub2(s, x)));  // inc - (s - x): what the addition lost
+    x = s;
+    xt = add2(xt, fma2(K.c, dlt, tg));
+}
+template <bool XLO>
+__device__ __forceinline__ void comm_pair_x(f32x2& xa, f32x2& xla, f32x2& xta, f32x2& xb, f32x2& xlb, f32x2& xtb, const CommK& K,
+                                            bool msg_before_mix) {
+    f32x2 da = sub2(xa, xta), db = sub2(xb, xtb);
+    if (XLO) { da = add2(da, xla); db = add2(db, xlb); }
+    const f32x2 ua = mul2(K.nca, da);
+    const f32x2 ub = mul2(K.ncb, db);
+    const f32x2 raw = sub2(xa, xb);
+    f32x2 bv = sub2(raw, xa);
+    f32x2 av = sub2(raw, bv);
+    f32x2 e_raw = sub2(sub2(xa, av), add2(xb, bv));
+    if (XLO) e_raw = add2(e_raw, sub2(xla, xlb));
+    f32x2 m = raw, m_lo = e_raw;
+    if (!msg_before_mix) {
+        const f32x2 du = sub2(ua, ub);
+        m = add2(raw, du);
+        bv = sub2(m, raw);
+        av = sub2(m, bv);
+        m_lo = add2(e_raw, add2(sub2(raw, av), sub2(du, bv)));
+    }
+    const f32x2 ia = fma2(K.nalpha, m, fma2(K.nalpha, m_lo, ua));
+    const f32x2 ib = fma2(K.alpha, m, fma2(K.alpha, m_lo, ub));
+    const f32x2 sa = add2(xa, ia), sb = add2(xb, ib);
+    if (XLO) {
+        xla = add2(xla, sub2(ia, sub2(sa, xa)));
+        xlb = add2(xlb, sub2(ib, sub2(sb, xb)));
+    }
+    xa = sa;
+    xb = sb;
+    xta = sub2(xta, fma2(K.alpha_t, m, fma2(K.alpha_t, m_lo, ua)));
+    xtb = sub2(xtb, fma2(K.nalpha_t, m, fma2(K.nalpha_t, m_lo, ub)));
+}
+
 // ---------------------------------------------------------------------------------------------
 // Four-worker items on fp32 rows with the rows held as NATIVE PAIRS: a row's 32 bytes arrive as four 64-bit
 // registers (ld.global.cs.v4.b64), every operation is one of sm_100's packed fp32 instructions on such a register
@@ -641,7 +687,9 @@ __device__ __forceinline__ void st_pairs(float* p, const f32x2 (&v)[4]) {
 // (Launch bounds without a minimum CTA count on purpose: ptxas then settles at 156-158 registers and two CTAs of
 // 192 threads fit an SM. With an explicit minimum of one it takes more than 170, one CTA fits, and the kernel
 // loses a third of its speed; with the registers capped at 128 for sixteen warps it gains nothing.)
-template <int KW, int THREADS, bool SLICE>
+// XLO: x is carried as the two-word value x + xl inside an item and rounded once, when the row is stored
+// (A2_ROUND_PER_STORE); otherwise every event rounds x like every other value (A2_ROUND_PER_EVENT).
+template <int KW, int THREADS, bool SLICE, bool XLO = false>
 __global__ void __launch_bounds__(THREADS) k_apply_events_pairs(const EventArgs p) {
     constexpr int N = 8, NP = 4;  // fp32 columns and native pairs per 256-bit vector
     __shared__ DevItem s_items[kMaxItemsPerLaunch];
@@ -706,6 +754,16 @@ __global__ void __launch_bounds__(THREADS) k_apply_events_pairs(const EventArgs 
 
         constexpr int PC = KW >= 3 ? NP : 1, PD = KW >= 4 ? NP : 1;
         f32x2 xa[NP], xta[NP], xb[NP], xtb[NP], ga[NP], gb[NP], xc[PC], xtc[PC], gc[PC], xd[PD], xtd[PD], gd[PD];
+        constexpr int LA = XLO ? NP : 1, LC = XLO ? PC : 1, LD = XLO ? PD : 1;
+        f32x2 xla[LA], xlb[LA], xlc[LC], xld[LD];
+        if (XLO) {
+#pragma unroll
+            for (int k = 0; k < LA; ++k) { xla[k] = 0ull; xlb[k] = 0ull; }
+#pragma unroll
+            for (int k = 0; k < LC; ++k) xlc[k] = 0ull;
+#pragma unroll
+            for (int k = 0; k < LD; ++k) xld[k] = 0ull;
+        }
         ld_pairs(pxa, xa);
         ld_pairs(pxta, xta);
         if (has_b) {
@@ -739,41 +797,52 @@ __global__ void __launch_bounds__(THREADS) k_apply_events_pairs(const EventArgs 
         for (int o = o_first; o < o_first + it.op_count; ++o) {
             const int kind = s_kind[o];
             const float ca = s_ca[o];
-            auto grad = [&](f32x2 (&x)[NP], f32x2 (&xt)[NP], f32x2 (&g)[NP]) {
+            auto grad = [&](f32x2 (&x)[NP], f32x2* xl, f32x2 (&xt)[NP], f32x2 (&g)[NP]) {
                 const GradK K(ca, ngamma);
 #pragma unroll
-                for (int k = 0; k < NP; ++k) grad_pair2<true>(x[k], xt[k], K, g[k]);
+                for (int k = 0; k < NP; ++k) grad_pair_x<XLO>(x[k], xl[XLO ? k : 0], xt[k], K, g[k]);
                 const int rl = s_reload[o];  // the worker's next gradient row, when it is another one
                 if (rl >= 0) ld_pairs(G + (long long)rl * p.pitch + off, g);
             };
-            auto comm = [&](f32x2 (&xp)[NP], f32x2 (&xtp)[NP], f32x2 (&xq)[NP], f32x2 (&xtq)[NP]) {
+            auto comm = [&](f32x2 (&xp)[NP], f32x2* xlp, f32x2 (&xtp)[NP], f32x2 (&xq)[NP], f32x2* xlq, f32x2 (&xtq)[NP]) {
                 const CommK K(ca, s_cb[o], alpha, alpha_t);
 #pragma unroll
-                for (int k = 0; k < NP; ++k) comm_pair2<true>(xp[k], xtp[k], xq[k], xtq[k], K, before);
+                for (int k = 0; k < NP; ++k)
+                    comm_pair_x<XLO>(xp[k], xlp[XLO ? k : 0], xtp[k], xq[k], xlq[XLO ? k : 0], xtq[k], K, before);
             };
             if (kind == A2_OP_GRAD_A) {
-                grad(xa, xta, ga);
+                grad(xa, xla, xta, ga);
             } else if (kind == A2_OP_GRAD_B) {
-                grad(xb, xtb, gb);
+                grad(xb, xlb, xtb, gb);
             } else if (kind == A2_OP_MIX_A) {  // mixing alone: a gradient event with a zero gradient
                 const GradK K(ca, ngamma);
 #pragma unroll
-                for (int k = 0; k < NP; ++k) grad_pair2<true>(xa[k], xta[k], K, pk2(0.f, 0.f));
+                for (int k = 0; k < NP; ++k) grad_pair_x<XLO>(xa[k], xla[XLO ? k : 0], xta[k], K, pk2(0.f, 0.f));
             } else if (kind == A2_OP_COMM) {
-                comm(xa, xta, xb, xtb);
+                comm(xa, xla, xta, xb, xlb, xtb);
             } else if constexpr (KW >= 3) {
                 if (kind == A2_OP_GRAD_C) {
-                    grad(xc, xtc, gc);
+                    grad(xc, xlc, xtc, gc);
                 } else if (kind == A2_OP_COMM_AC) {
-                    comm(xa, xta, xc, xtc);
+                    comm(xa, xla, xta, xc, xlc, xtc);
                 } else if (kind == A2_OP_COMM_BC) {
-                    comm(xb, xtb, xc, xtc);
+                    comm(xb, xlb, xtb, xc, xlc, xtc);
                 } else if constexpr (KW >= 4) {
-                    if (kind == A2_OP_GRAD_D) grad(xd, xtd, gd);
-                    else if (kind == A2_OP_COMM_AD) comm(xa, xta, xd, xtd);
-                    else if (kind == A2_OP_COMM_BD) comm(xb, xtb, xd, xtd);
-                    else comm(xc, xtc, xd, xtd);
+                    if (kind == A2_OP_GRAD_D) grad(xd, xld, xtd, gd);
+                    else if (kind == A2_OP_COMM_AD) comm(xa, xla, xta, xd, xld, xtd);
+                    else if (kind == A2_OP_COMM_BD) comm(xb, xlb, xtb, xd, xld, xtd);
+                    else comm(xc, xlc, xtc, xd, xld, xtd);
                 }
+            }
+        }
+
+        if (XLO) {  // the row as stored: one rounding of x + xl
+#pragma unroll
+            for (int k = 0; k < NP; ++k) {
+                xa[k] = add2(xa[k], xla[k]);
+                if (has_b) xb[k] = add2(xb[k], xlb[k]);
+                if (KW >= 3 && has_c) xc[k] = add2(xc[k], xlc[XLO && KW >= 3 ? k : 0]);
+                if (KW >= 4 && has_d) xd[k] = add2(xd[k], xld[XLO && KW >= 4 ? k : 0]);
             }
         }
 
@@ -1374,8 +1443,13 @@ int launch_events_pairs4(const EventLaunch& L, const DeviceInfo& dev, cudaStream
     const GridShape gs = grid_shape(L.slice, a.n_vec, n_units, (long long)dev.sm_count * dev.event4_ctas_per_sm[1]);
     a.slice_vec = gs.slice_vec;
     if (gs.grid < 1) return 0;
-    if (L.slice) k_apply_events_pairs<4, THREADS, true><<<gs.grid, THREADS, 0, stream>>>(a);
-    else k_apply_events_pairs<4, THREADS, false><<<gs.grid, THREADS, 0, stream>>>(a);
+    if (L.round_per_store) {
+        if (L.slice) k_apply_events_pairs<4, THREADS, true, true><<<gs.grid, THREADS, 0, stream>>>(a);
+        else k_apply_events_pairs<4, THREADS, false, true><<<gs.grid, THREADS, 0, stream>>>(a);
+    } else {
+        if (L.slice) k_apply_events_pairs<4, THREADS, true><<<gs.grid, THREADS, 0, stream>>>(a);
+        else k_apply_events_pairs<4, THREADS, false><<<gs.grid, THREADS, 0, stream>>>(a);
+    }
     return (int)cudaGetLastError();
 }
 
@@ -1602,6 +1676,11 @@ int launch_bf16_packed(const EventLaunch& L, const DeviceInfo& dev, cudaStream_t
     return (int)cudaGetLastError();
 }
 
+// Rows on 32-byte boundaries (what the 256-bit kernels, and with them A2_ROUND_PER_STORE, need).
+bool rows_allow_256bit(const void* x, const void* xt, const void* g, int64_t pitch, int32_t dtype) {
+    return rows_32B_aligned(x, xt, g, pitch, dtype);
+}
+
 int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
     if (L.n_items <= 0) return 0;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -1620,6 +1699,10 @@ int launch_events(const EventLaunch& L, const DeviceInfo& dev, void* stream_) {
         return wide_x ? launch_plain_t<float, 32, 2>(L, dev, stream) : launch_plain_t<float, 16, 2>(L, dev, stream);
     }
     const bool wide = rows_32B_aligned(L.x, L.xt, L.g, L.pitch, L.dtype);
+    if (L.round_per_store) {  // one kernel serves every item width in this mode; the caller has checked the rest
+        if (!wide || L.dtype == A2_BF16) return (int)cudaErrorInvalidValue;
+        return launch_events_pairs4(L, dev, stream);
+    }
     if (L.max_workers >= 4 && L.dtype != A2_BF16) {
         static const bool narrow4 = a2::tuning_env("A2CID2_EVENT4_128BIT") != nullptr;  // tuning override
         if (wide && !narrow4) return launch_events_pairs4(L, dev, stream);

@@ -102,6 +102,14 @@ def test_create_validates_without_a_device():
     for m in (B.A2_LAUNCH_PER_BATCH, B.A2_LAUNCH_COLUMN_SLICES, B.A2_LAUNCH_AUTO):
         assert L.a2cid2_set_launch_mode(h, m) == B.A2_OK
     assert L.a2cid2_set_launch_mode(h, 3) == B.A2_EINVAL and b"launch mode" in L.a2cid2_last_error(h)
+    # this handle stores bf16 rows: rounding x once per store instead of once per event is an fp32 matter
+    assert L.a2cid2_set_rounding(h, B.A2_ROUND_PER_EVENT) == B.A2_OK
+    assert L.a2cid2_set_rounding(h, B.A2_ROUND_PER_STORE) == B.A2_EINVAL and b"fp32" in L.a2cid2_last_error(h)
+    assert L.a2cid2_set_rounding(h, 2) == B.A2_EINVAL
+    f = C.c_void_p()
+    assert L.a2cid2_create(4, 10, 0.1, 0.5, 0.5, 0.1, B.A2_F32, C.byref(f)) == B.A2_OK
+    assert L.a2cid2_set_rounding(f, B.A2_ROUND_PER_STORE) == B.A2_OK
+    L.a2cid2_destroy(f)
     # binding without an x~ buffer is refused unless the variant has no momentum (checked before any device call)
     dummy = C.c_void_p(4096)
     assert L.a2cid2_bind(h, dummy, None, None, 0, 16, None) == B.A2_EINVAL

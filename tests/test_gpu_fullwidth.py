@@ -168,11 +168,12 @@ IDEAL_EVERY = 8  # fp32 rows: the ideal fp32-storage run is made on every eighth
 PLAIN_EVERY_BF16 = 4  # bf16 rows: the plain fp64 run (row norms) on every fourth chunk taken
 
 
-def _check_full_width(cfg, check_events):
+def _check_full_width(cfg, check_events, rounding=B.A2_ROUND_PER_EVENT):
     import torch
 
     torch.cuda.set_device(0)
     eng = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, storage=cfg.storage, n_grad_slots=cfg.n_grad_slots)
+    eng.set_rounding(rounding)
     x0, g = _fill_and_keep(eng, cfg)
     ev = W.config_events(cfg)
     n_steps = (len(ev) + EVENTS_PER_STEP - 1) // EVENTS_PER_STEP
@@ -281,6 +282,15 @@ def test_every_element_with_fresh_gradient_rows_inside_four_worker_items():
     (the paper's gradients are fresh draws at every step, Sec. 3.2). The first 4,000 events of the stream."""
     cfg = replace(W.CONFIGS["cfg4"], grad_pool=4, n_events=4_000, name="cfg4-pool4")
     _check_full_width(cfg, ())
+
+
+def test_every_element_of_the_64_worker_ring_with_x_rounded_once_per_store():
+    """A2_ROUND_PER_STORE on the workload whose default run ends 5 % above 1e-5 on its worst element (alpha~ =
+    7.26 amplifies the rounding errors of x): with x rounded once per store instead of once per event every one
+    of the 3.3e9 elements is within 1e-5 at the end of the run, below what rounding at every event can deliver."""
+    rep = _check_full_width(replace(W.CONFIGS["cfg4"], name="cfg4-round-per-store"), (), rounding=B.A2_ROUND_PER_STORE)
+    last = rep[max(k for k in rep if k.startswith("after_step_"))]
+    assert last["max_rel_err"] <= P.TOL["f32"] and last["max_rel_err"] < last["ideal_fp32_storage"]
 
 
 def test_static_gradient_rows_on_the_complete_graph_workload():

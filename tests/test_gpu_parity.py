@@ -353,3 +353,73 @@ def test_launch_modes_give_the_same_bits(storage, momentum, d):
         x, xt, t = states[0]
         chk.compare(P.widen(x, "f32"), None if xt is None else P.widen(xt, "f32"), t, where=f"launch modes, d={d}")
         eng.close()
+
+
+@pytest.mark.parametrize("name,d,n_events", [("cfg4", 4_097, 4000), ("cfg3", 6_150, 3000), ("cfg2", 20_011, 3000)])
+def test_round_per_store_parity_every_batch(name, d, n_events):
+    """A2_ROUND_PER_STORE: inside an item x is carried as a two-word value and rounded once, when the row is
+    stored. Parity with the checker after every batch under the chained schedule; the end state differs from the
+    default mode's in the last bits only, and on the 64-worker ring it is closer to the checker."""
+    cfg = W.CONFIGS[name].scaled(d=d, n_events=n_events)
+    ev = W.config_events(cfg)
+    eng, chk = P.make_small(cfg)
+    eng.set_rounding(B.A2_ROUND_PER_STORE)
+    worst, nb = P.run_batches_and_check(eng, chk, ev, B.A2_SCHED_CHAIN)
+    per_store = eng.read_state()
+    eng.close()
+    base, _ = P.make_small(cfg)
+    base.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)
+    per_event = base.read_state()
+    base.close()
+    assert np.array_equal(per_store[2], per_event[2])
+    # both are within 1e-5 of the checker, hence within 2e-5 of each other; and they are not the same bits
+    assert P.rel_err(per_store[0], per_event[0]) <= 2e-5 and P.rel_err(per_store[1], per_event[1]) <= 2e-5
+    assert not np.array_equal(per_store[1], per_event[1])
+    err_store = max(P.rel_err(per_store[0], chk.plain.X), P.rel_err(per_store[1], chk.plain.Xt))
+    err_event = max(P.rel_err(per_event[0], chk.plain.X), P.rel_err(per_event[1], chk.plain.Xt))
+    print(f"{cfg.name}: per store {err_store:.2e}, per event {err_event:.2e}")
+    assert err_store <= P.TOL["f32"] and err_event <= P.TOL["f32"]
+    if name == "cfg4":  # alpha~ / alpha = 14.5: here the roundings of x dominate, and sparing them shows
+        assert err_store < err_event
+
+
+def test_round_per_store_launch_modes_flush_and_refusals():
+    cfg = W.CONFIGS["cfg4"].scaled(d=2_049, n_events=1500)
+    ev = W.config_events(cfg)
+    states = []
+    for mode in (B.A2_LAUNCH_PER_BATCH, B.A2_LAUNCH_COLUMN_SLICES):
+        eng, chk = P.make_small(cfg)
+        eng.set_rounding(B.A2_ROUND_PER_STORE)
+        eng.set_launch_mode(mode)
+        eng.apply_events(ev.times, ev.wi, ev.wj, ev.slot, flags=B.A2_SCHED_CHAIN)
+        t_end = float(ev.times[-1]) + 0.5
+        eng.flush(t_end)
+        states.append(eng.read_state())
+        if mode == B.A2_LAUNCH_PER_BATCH:
+            chk.plain.apply_stream(ev)
+            chk.plain.flush(t_end)
+            x, xt, t = states[0]
+            chk.compare(P.widen(x, "f32"), P.widen(xt, "f32"), t, where="per store, flushed")
+            c_ref = chk.plain.consensus()
+            assert abs(eng.consensus_distance() - c_ref) <= 1e-4 * c_ref
+            # the shared-memory-resident mode rounds at every event: refused, state untouched
+            with pytest.raises(B.A2Error) as e:
+                eng.apply_events([t_end + 1.0], [0], [1], [-1], flags=B.A2_SCHED_RESIDENT)
+            assert e.value.code == B.A2_EINVAL
+            assert all(np.array_equal(u, v) for u, v in zip(states[0], eng.read_state()))
+        eng.close()
+    assert all(np.array_equal(u, v) for u, v in zip(*states))  # the same schedule: the same bits in both launch modes
+    # rows that are only 16-byte aligned cannot take the mode: refused before any launch
+    odd = B.Engine(cfg.n, cfg.d, *B.config_params(cfg), cfg.gamma, n_grad_slots=cfg.n_grad_slots, rows_16B_only=True)
+    odd.set_rounding(B.A2_ROUND_PER_STORE)
+    with pytest.raises(B.A2Error) as e:
+        odd.apply_events(ev.times[:10], ev.wi[:10], ev.wj[:10], ev.slot[:10])
+    assert e.value.code == B.A2_ESTATE and "32-byte" in str(e.value)
+    odd.set_rounding(B.A2_ROUND_PER_EVENT)
+    odd.apply_events(ev.times[:10], ev.wi[:10], ev.wj[:10], ev.slot[:10])
+    odd.close()
+    bf = B.Engine(4, 64, 0.1, 0.5, 0.5, 0.1, storage="bf16")
+    with pytest.raises(B.A2Error) as e:
+        bf.set_rounding(B.A2_ROUND_PER_STORE)
+    assert e.value.code == B.A2_EINVAL
+    bf.close()
