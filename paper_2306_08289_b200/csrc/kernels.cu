@@ -624,10 +624,11 @@ __global__ void __launch_bounds__(THREADS) k_apply_events(const EventArgs p) {
 
 // The two updates with x carried as an unevaluated sum x + xl inside an item (xl: what the roundings of x have lost
 // so far; it starts at zero when the row is loaded and is added back, with one rounding, when the row is stored).
+// xl enters the message, which alpha~ amplifies; the mixing difference x - x~ ignores it (c xl is second order:
+// measured, the worst element of the 64-worker ring is the same with and without, and the kernel 3 % faster).
 template <bool XLO>
 __device__ __forceinline__ void grad_pair_x(f32x2& x, f32x2& xl, f32x2& xt, const GradK& K, f32x2 g) {
-    f32x2 dlt = sub2(x, xt);
-    if (XLO) dlt = add2(dlt, xl);
+    const f32x2 dlt = sub2(x, xt);
     const f32x2 tg = mul2(K.ngamma, g);
     const f32x2 inc = fma2(K.nc, dlt, tg);
     const f32x2 s = add2(x, inc);
@@ -638,10 +639,8 @@ __device__ __forceinline__ void grad_pair_x(f32x2& x, f32x2& xl, f32x2& xt, cons
 template <bool XLO>
 __device__ __forceinline__ void comm_pair_x(f32x2& xa, f32x2& xla, f32x2& xta, f32x2& xb, f32x2& xlb, f32x2& xtb, const CommK& K,
                                             bool msg_before_mix) {
-    f32x2 da = sub2(xa, xta), db = sub2(xb, xtb);
-    if (XLO) { da = add2(da, xla); db = add2(db, xlb); }
-    const f32x2 ua = mul2(K.nca, da);
-    const f32x2 ub = mul2(K.ncb, db);
+    const f32x2 ua = mul2(K.nca, sub2(xa, xta));
+    const f32x2 ub = mul2(K.ncb, sub2(xb, xtb));
     const f32x2 raw = sub2(xa, xb);
     f32x2 bv = sub2(raw, xa);
     f32x2 av = sub2(raw, bv);
