@@ -44,7 +44,7 @@ pytestmark = pytest.mark.gpu
 
 CHUNK_COLS = 8192
 EVENTS_PER_STEP = 500
-BUDGET_S = 180.0
+BUDGET_S = 160.0
 
 
 def _threads():
